@@ -1,0 +1,196 @@
+/*
+ * luvc.h - C ABI of the LUVC token-compression library for NVIDIA B200 (sm_100a).
+ *
+ * Two training-free operators of "Towards Lossless Ultimate Vision Token
+ * Compression for VLMs" (arXiv 2512.09010):
+ *
+ *   OIM  Orthogonal Iterative Merger (Section 3.2; Eq. 3; appendix "Iterative
+ *        Strategy and Pseudocode of OIM", Algorithm 1): merges similar
+ *        neighbouring vision tokens on the 2D patch grid, alternately along the
+ *        width and the height, so that the grid stays rectangular.
+ *   SPU  Spectrum Pruning Unit (Section 3.3, Eq. 4-8; Algorithm 2): scores every
+ *        visual token by the energy of the low-pass-filtered token sequence and
+ *        keeps the highest-scoring tokens in their original order.
+ *
+ * General rules
+ *   - Every function returns a luvc_status (int); 0 is success.  Nothing aborts
+ *     or throws.  Argument errors are reported before any work is queued and
+ *     leave the outputs untouched.
+ *   - Unless a function says "host", every data pointer is a DEVICE pointer
+ *     owned by the caller (for PyTorch: tensor.data_ptr()).  The library never
+ *     frees or keeps caller memory.  Inputs are not modified.  Outputs must not
+ *     overlap inputs.
+ *   - Tensors are dense, row-major, innermost dimension D contiguous.  Base
+ *     pointers must be 16-byte aligned and D * sizeof(element) a multiple of 16
+ *     (D % 8 == 0 for bf16, D % 4 == 0 for fp32), else LUVC_ERR_ALIGN.
+ *   - Device calls are asynchronous on the calling thread's luvc stream (see
+ *     luvc_set_stream) and do not synchronise the host.
+ *   - The plain entry points use a library-owned scratch buffer that grows with
+ *     cudaMalloc on demand (a host-synchronous call the first time a larger
+ *     problem is seen) and is released by luvc_shutdown().  The _ex entry points
+ *     use only the caller's workspace when one is given.
+ */
+#ifndef LUVC_H_
+#define LUVC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LUVC_OK = 0,
+    LUVC_ERR_NULL = 1,       /* a required pointer is NULL */
+    LUVC_ERR_SHAPE = 2,      /* a dimension is < 1 or too large for 32-bit indexing */
+    LUVC_ERR_TARGET = 3,     /* target_count / output grid not reachable from H x W */
+    LUVC_ERR_KEEP = 4,       /* keep outside [1, N] */
+    LUVC_ERR_CUTOFF = 5,     /* cutoff is NaN or > 1 */
+    LUVC_ERR_ALIGN = 6,      /* pointer or row size not 16-byte aligned */
+    LUVC_ERR_DTYPE = 7,      /* unknown element type */
+    LUVC_ERR_WORKSPACE = 8,  /* caller workspace too small or misaligned */
+    LUVC_ERR_CUDA = 9,       /* a CUDA call failed (allocation, copy, launch) */
+    LUVC_ERR_TIMEOUT = 10,   /* a bounded device-side wait gave up */
+    LUVC_ERR_INTERNAL = 11
+} luvc_status;
+
+typedef enum { LUVC_BF16 = 0, LUVC_F32 = 1 } luvc_dtype;
+
+/* Cutoff used when the caller passes cutoff <= 0.  The paper never states the
+ * value of its sigma_t; 1/8 of the band is this library's choice. */
+#define LUVC_SPU_DEFAULT_CUTOFF 0.125f
+
+/* ---- housekeeping ------------------------------------------------------- */
+
+/* Library version, major * 1000 + minor. */
+int luvc_version(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char* luvc_status_string(int status);
+
+/* Sets the CUDA stream (a cudaStream_t passed as void*) used by the plain entry
+ * points of the calling host thread.  NULL selects the legacy default stream. */
+int luvc_set_stream(void* cuda_stream);
+
+/* Frees the library-owned scratch buffers of the current device.  Synchronises
+ * the device first.  Safe to call more than once. */
+int luvc_shutdown(void);
+
+/* Number of kernels this library has launched since it was loaded (all threads). */
+long long luvc_kernel_launches(void);
+
+/* ---- OIM ---------------------------------------------------------------- */
+
+/* Host-only planning.  Maps target_count to the final grid out_h x out_w: the
+ * factor pair of target_count with out_h <= H, out_w <= W whose aspect ratio is
+ * closest, in log scale, to H / W (tie: larger out_h), and counts the merge
+ * steps needed with `merge_per_step` cells removed per line per step
+ * (0 = the paper's merge number 2).  LUVC_ERR_TARGET if no such pair exists. */
+int luvc_oim_plan(int H, int W, int target_count, int merge_per_step,
+                  int* out_h, int* out_w, int* n_steps);
+
+/* Bytes of workspace luvc_oim_merge_ex needs for this problem. */
+size_t luvc_oim_workspace_bytes(int B, int H, int W, int D, int dtype);
+
+typedef struct {
+    int dtype;               /* luvc_dtype of tokens and out_tokens */
+    void* stream;            /* cudaStream_t; NULL = legacy default stream */
+    void* workspace;         /* device, 256-byte aligned; NULL = library-owned scratch */
+    size_t workspace_bytes;
+    int out_h, out_w;        /* explicit final grid; 0,0 = derive from target_count */
+    int merge_per_step;      /* cells removed per line per step; 0 = 2 (appendix of the paper) */
+    int height_first;        /* 0: width step first (Section 3.2); 1: Algorithm 1's order */
+    int32_t* trace;          /* optional device [B, H*W - out_h*out_w]: one entry per merge,
+                                (position of the merged cell in its line) * 2 + direction
+                                (0 = into the previous cell of the line, 1 = into the next),
+                                ordered by step, line, rank of the candidate */
+} luvc_oim_opts;
+
+/*
+ * Orthogonal Iterative Merger (Section 3.2).
+ *
+ * tokens      [B, H, W, D]  patch tokens of B images on their 2D grid
+ * out_tokens  [B, target_count, D]  merged tokens, row-major over the final grid;
+ *             each is the mean of its source tokens (the size-weighted merge
+ *             composed over the steps), rounded once to the element type
+ * out_sizes   [B, target_count] int32  number of source tokens per merged token
+ *             (the vector s of Eq. 3)
+ * out_map     [B, H*W] int32  final cell (row-major index) each source token ended in
+ *
+ * The iteration alternates one width step and one height step until the grid is
+ * out_h x out_w.  A step treats every line (row or column) independently: cells
+ * at even positions compare themselves (cosine, fp32 accumulation) with their
+ * one or two neighbours in the line, the m cells with the highest similarity
+ * (ties: lowest position; direction ties: the previous cell) are merged into
+ * that neighbour, and the line closes up keeping its order.
+ *
+ * luvc_oim_merge takes bf16, luvc_oim_merge_f32 fp32; both run on the thread's
+ * luvc stream with library-owned scratch.
+ */
+int luvc_oim_merge(const void* tokens, int B, int H, int W, int D, int target_count,
+                   void* out_tokens, int32_t* out_sizes, int32_t* out_map);
+int luvc_oim_merge_f32(const float* tokens, int B, int H, int W, int D, int target_count,
+                       float* out_tokens, int32_t* out_sizes, int32_t* out_map);
+int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target_count,
+                      void* out_tokens, int32_t* out_sizes, int32_t* out_map,
+                      const luvc_oim_opts* opts);
+
+/* Same operator on HOST buffers (pinned memory recommended): copies the tokens to
+ * the device, runs, copies the three outputs back and synchronises the stream
+ * before returning.  dtype is a luvc_dtype. */
+int luvc_oim_merge_host(const void* tokens, int B, int H, int W, int D, int target_count, int dtype,
+                        void* out_tokens, int32_t* out_sizes, int32_t* out_map);
+
+/* ---- SPU ---------------------------------------------------------------- */
+
+/* Last passed frequency bin for a sequence of N tokens:
+ * floor(cutoff * floor(N / 2)); cutoff <= 0 selects LUVC_SPU_DEFAULT_CUTOFF.
+ * Returns -1 if cutoff is NaN or > 1. */
+int luvc_spu_sigma(int N, float cutoff);
+
+/* Bytes of workspace luvc_spu_prune_ex needs for this problem. */
+size_t luvc_spu_workspace_bytes(int B, int N, int D, float cutoff, int dtype);
+
+typedef struct {
+    int dtype;               /* luvc_dtype of hidden and out_hidden */
+    void* stream;
+    void* workspace;         /* device, 256-byte aligned; NULL = library-owned scratch */
+    size_t workspace_bytes;
+    int no_window;           /* 0: Hamming-windowed pass band (Eq. 5); 1: flat pass band
+                                (the paper's "without HW" ablation) */
+    float* out_scores;       /* optional device [B, N] fp32: the energies E of Eq. 8 */
+} luvc_spu_opts;
+
+/*
+ * Spectrum Pruning Unit (Algorithm 2).
+ *
+ * hidden      [B, N, D]  hidden states of the N visual tokens of B sequences
+ * cutoff      fraction of the band [0, floor(N/2)] that is passed, in (0, 1];
+ *             <= 0 selects the default
+ * keep        number of tokens kept per sequence, 1 <= keep <= N
+ * out_idx     [B, keep] int32  kept token indices, strictly ascending
+ * out_hidden  [B, keep, D]  the kept rows of `hidden`, bit-exact copies
+ *
+ * Per sequence and channel the token axis is transformed (Eq. 4), multiplied by
+ * the mask of Eq. 5/6 - a Hamming window centred on the zero frequency,
+ * 0.54 + 0.46 cos(2 pi f / (N - 1)) for signed frequencies |f| <= sigma and 0
+ * elsewhere - and transformed back (Eq. 7); a token's score is the L2 norm over
+ * the channels of the filtered signal (Eq. 8).  The `keep` highest scores win,
+ * ties go to the lower index.  Arithmetic is fp32.
+ */
+int luvc_spu_prune(const void* hidden, int B, int N, int D, float cutoff, int keep,
+                   int32_t* out_idx, void* out_hidden);
+int luvc_spu_prune_f32(const float* hidden, int B, int N, int D, float cutoff, int keep,
+                       int32_t* out_idx, float* out_hidden);
+int luvc_spu_prune_ex(const void* hidden, int B, int N, int D, float cutoff, int keep,
+                      int32_t* out_idx, void* out_hidden, const luvc_spu_opts* opts);
+
+/* Same operator on HOST buffers (see luvc_oim_merge_host). */
+int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, int keep, int dtype,
+                        int32_t* out_idx, void* out_hidden);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LUVC_H_ */

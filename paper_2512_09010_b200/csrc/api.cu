@@ -1,0 +1,277 @@
+// C ABI of the library: argument checks, stream and scratch handling, and the
+// host-buffer variants.  All arithmetic lives in oim.cu and spu.cu.
+
+#include <atomic>
+#include <cmath>
+#include <mutex>
+
+#include "luvc_internal.h"
+
+namespace luvc {
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+namespace {
+
+thread_local cudaStream_t t_stream = nullptr;
+
+// Library-owned scratch: one growing buffer per purpose, shared by all threads.
+// Calls that use it from several host threads at once must use different streams'
+// work serially; the plain entry points take this lock only while (re)allocating.
+enum Slot { kOimWs = 0, kSpuWs, kIoIn, kIoOut, kSlots };
+struct Scratch { void* ptr = nullptr; size_t bytes = 0; };
+Scratch g_scratch[kSlots];
+std::mutex g_mutex;
+
+void* scratch(Slot s, size_t bytes) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Scratch& sc = g_scratch[s];
+    if (sc.bytes >= bytes && sc.ptr) return sc.ptr;
+    if (sc.ptr) { cudaDeviceSynchronize(); cudaFree(sc.ptr); sc.ptr = nullptr; sc.bytes = 0; }
+    void* p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    sc.ptr = p; sc.bytes = bytes;
+    return p;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+size_t elem_size(int dtype) { return dtype == LUVC_F32 ? 4 : 2; }
+
+int check_oim(const void* tokens, int B, int H, int W, int D, int target, const void* out_tokens,
+              const void* out_sizes, const void* out_map, const luvc_oim_opts& o, int* Hf, int* Wf) {
+    if (!tokens || !out_tokens || !out_sizes || !out_map) return LUVC_ERR_NULL;
+    if (o.dtype != LUVC_BF16 && o.dtype != LUVC_F32) return LUVC_ERR_DTYPE;
+    if (B < 1 || H < 1 || W < 1 || D < 1 || B > 65535) return LUVC_ERR_SHAPE;
+    if ((long long)H * W > (1ll << 30) || (long long)B * H * W > (1ll << 31) - 1) return LUVC_ERR_SHAPE;
+    if (((size_t)D * elem_size(o.dtype)) % 16 != 0) return LUVC_ERR_ALIGN;
+    if (!aligned16(tokens) || !aligned16(out_tokens) || (reinterpret_cast<uintptr_t>(out_sizes) & 3u) ||
+        (reinterpret_cast<uintptr_t>(out_map) & 3u))
+        return LUVC_ERR_ALIGN;
+    if (o.merge_per_step < 0) return LUVC_ERR_TARGET;
+    if (o.out_h || o.out_w) {
+        if (o.out_h < 1 || o.out_w < 1 || o.out_h > H || o.out_w > W) return LUVC_ERR_TARGET;
+        if ((long long)o.out_h * o.out_w != (long long)target) return LUVC_ERR_TARGET;
+        *Hf = o.out_h; *Wf = o.out_w;
+    } else if (!oim_final_dims(H, W, target, Hf, Wf)) {
+        return LUVC_ERR_TARGET;
+    }
+    int n = 0;
+    if (!oim_schedule(H, W, *Hf, *Wf, o.merge_per_step ? o.merge_per_step : 2, o.height_first, nullptr, 0, &n))
+        return LUVC_ERR_TARGET;
+    return LUVC_OK;
+}
+
+int check_spu(const void* hidden, int B, int N, int D, float cutoff, int keep, const void* out_idx,
+              const void* out_hidden, int dtype, int* sigma) {
+    if (!hidden || !out_idx || !out_hidden) return LUVC_ERR_NULL;
+    if (dtype != LUVC_BF16 && dtype != LUVC_F32) return LUVC_ERR_DTYPE;
+    if (B < 1 || N < 1 || D < 1 || B > 65535 || (long long)B * N > (1ll << 31) - 1) return LUVC_ERR_SHAPE;
+    if (keep < 1 || keep > N) return LUVC_ERR_KEEP;
+    *sigma = luvc_spu_sigma(N, cutoff);
+    if (*sigma < 0) return LUVC_ERR_CUTOFF;
+    if (((size_t)D * elem_size(dtype)) % 16 != 0) return LUVC_ERR_ALIGN;
+    if (!aligned16(hidden) || !aligned16(out_hidden) || (reinterpret_cast<uintptr_t>(out_idx) & 3u))
+        return LUVC_ERR_ALIGN;
+    return LUVC_OK;
+}
+
+}  // namespace
+}  // namespace luvc
+
+using namespace luvc;
+
+extern "C" {
+
+int luvc_version(void) { return 1000; }
+
+const char* luvc_status_string(int status) {
+    switch (status) {
+        case LUVC_OK: return "ok";
+        case LUVC_ERR_NULL: return "a required pointer is NULL";
+        case LUVC_ERR_SHAPE: return "a dimension is out of range";
+        case LUVC_ERR_TARGET: return "the target grid cannot be reached from the input grid";
+        case LUVC_ERR_KEEP: return "keep is outside [1, N]";
+        case LUVC_ERR_CUTOFF: return "cutoff is NaN or larger than 1";
+        case LUVC_ERR_ALIGN: return "a pointer or the row size is not 16-byte aligned";
+        case LUVC_ERR_DTYPE: return "unknown element type";
+        case LUVC_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case LUVC_ERR_CUDA: return "a CUDA call failed";
+        case LUVC_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case LUVC_ERR_INTERNAL: return "internal error";
+        default: return "unknown status";
+    }
+}
+
+int luvc_set_stream(void* cuda_stream) {
+    t_stream = static_cast<cudaStream_t>(cuda_stream);
+    return LUVC_OK;
+}
+
+int luvc_shutdown(void) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    cudaDeviceSynchronize();
+    for (auto& sc : g_scratch) {
+        if (sc.ptr) cudaFree(sc.ptr);
+        sc.ptr = nullptr; sc.bytes = 0;
+    }
+    return LUVC_OK;
+}
+
+long long luvc_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+// ---- OIM ---------------------------------------------------------------------
+
+int luvc_oim_plan(int H, int W, int target_count, int merge_per_step, int* out_h, int* out_w, int* n_steps) {
+    if (!out_h || !out_w || !n_steps) return LUVC_ERR_NULL;
+    if (H < 1 || W < 1) return LUVC_ERR_SHAPE;
+    int hf, wf, n;
+    if (merge_per_step < 0 || !oim_final_dims(H, W, target_count, &hf, &wf)) return LUVC_ERR_TARGET;
+    if (!oim_schedule(H, W, hf, wf, merge_per_step ? merge_per_step : 2, 0, nullptr, 0, &n)) return LUVC_ERR_TARGET;
+    *out_h = hf; *out_w = wf; *n_steps = n;
+    return LUVC_OK;
+}
+
+size_t luvc_oim_workspace_bytes(int B, int H, int W, int D, int dtype) {
+    if (B < 1 || H < 1 || W < 1 || D < 1) return 0;
+    return oim_workspace_bytes(B, H, W, D, dtype);
+}
+
+int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target_count, void* out_tokens,
+                      int32_t* out_sizes, int32_t* out_map, const luvc_oim_opts* opts) {
+    if (!opts) return LUVC_ERR_NULL;
+    int Hf = 0, Wf = 0;
+    const int rc = check_oim(tokens, B, H, W, D, target_count, out_tokens, out_sizes, out_map, *opts, &Hf, &Wf);
+    if (rc) return rc;
+    const size_t need = oim_workspace_bytes(B, H, W, D, opts->dtype);
+    void* ws = opts->workspace;
+    if (ws) {
+        if (opts->workspace_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u)) return LUVC_ERR_WORKSPACE;
+    } else {
+        ws = scratch(kOimWs, need);
+        if (!ws) return LUVC_ERR_CUDA;
+    }
+    OimProblem p;
+    p.tokens = tokens; p.B = B; p.H = H; p.W = W; p.D = D; p.Hf = Hf; p.Wf = Wf;
+    p.r = opts->merge_per_step ? opts->merge_per_step : 2;
+    p.height_first = opts->height_first ? 1 : 0;
+    p.dtype = opts->dtype;
+    p.out_tokens = out_tokens; p.out_sizes = out_sizes; p.out_map = out_map; p.trace = opts->trace;
+    p.workspace = ws; p.stream = static_cast<cudaStream_t>(opts->stream);
+    return oim_run(p);
+}
+
+int luvc_oim_merge(const void* tokens, int B, int H, int W, int D, int target_count, void* out_tokens,
+                   int32_t* out_sizes, int32_t* out_map) {
+    luvc_oim_opts o = {};
+    o.dtype = LUVC_BF16; o.stream = t_stream;
+    return luvc_oim_merge_ex(tokens, B, H, W, D, target_count, out_tokens, out_sizes, out_map, &o);
+}
+
+int luvc_oim_merge_f32(const float* tokens, int B, int H, int W, int D, int target_count, float* out_tokens,
+                       int32_t* out_sizes, int32_t* out_map) {
+    luvc_oim_opts o = {};
+    o.dtype = LUVC_F32; o.stream = t_stream;
+    return luvc_oim_merge_ex(tokens, B, H, W, D, target_count, out_tokens, out_sizes, out_map, &o);
+}
+
+int luvc_oim_merge_host(const void* tokens, int B, int H, int W, int D, int target_count, int dtype,
+                        void* out_tokens, int32_t* out_sizes, int32_t* out_map) {
+    if (!tokens || !out_tokens || !out_sizes || !out_map) return LUVC_ERR_NULL;
+    if (dtype != LUVC_BF16 && dtype != LUVC_F32) return LUVC_ERR_DTYPE;
+    if (B < 1 || H < 1 || W < 1 || D < 1 || target_count < 1) return LUVC_ERR_SHAPE;
+    const size_t es = elem_size(dtype), hw = (size_t)H * W;
+    const size_t in_bytes = (size_t)B * hw * D * es;
+    const size_t tok_bytes = align_up((size_t)B * target_count * D * es);
+    const size_t sz_bytes = align_up((size_t)B * target_count * 4), map_bytes = align_up((size_t)B * hw * 4);
+    unsigned char* din = static_cast<unsigned char*>(scratch(kIoIn, in_bytes));
+    unsigned char* dout = static_cast<unsigned char*>(scratch(kIoOut, tok_bytes + sz_bytes + map_bytes));
+    if (!din || !dout) return LUVC_ERR_CUDA;
+    cudaStream_t st = t_stream;
+    if (cudaMemcpyAsync(din, tokens, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return LUVC_ERR_CUDA;
+    luvc_oim_opts o = {};
+    o.dtype = dtype; o.stream = st;
+    int32_t* dsz = reinterpret_cast<int32_t*>(dout + tok_bytes);
+    int32_t* dmap = reinterpret_cast<int32_t*>(dout + tok_bytes + sz_bytes);
+    const int rc = luvc_oim_merge_ex(din, B, H, W, D, target_count, dout, dsz, dmap, &o);
+    if (rc) return rc;
+    cudaMemcpyAsync(out_tokens, dout, (size_t)B * target_count * D * es, cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(out_sizes, dsz, (size_t)B * target_count * 4, cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(out_map, dmap, (size_t)B * hw * 4, cudaMemcpyDeviceToHost, st);
+    return cudaStreamSynchronize(st) == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
+}
+
+// ---- SPU ---------------------------------------------------------------------
+
+int luvc_spu_sigma(int N, float cutoff) {
+    if (N < 1 || cutoff != cutoff || cutoff > 1.0f) return -1;
+    const double c = cutoff <= 0.0f ? (double)LUVC_SPU_DEFAULT_CUTOFF : (double)cutoff;
+    return (int)std::floor(c * (double)(N / 2));
+}
+
+size_t luvc_spu_workspace_bytes(int B, int N, int D, float cutoff, int dtype) {
+    const int sigma = luvc_spu_sigma(N, cutoff);
+    if (B < 1 || N < 1 || D < 1 || sigma < 0) return 0;
+    return spu_workspace_bytes(B, N, D, sigma, dtype);
+}
+
+int luvc_spu_prune_ex(const void* hidden, int B, int N, int D, float cutoff, int keep, int32_t* out_idx,
+                      void* out_hidden, const luvc_spu_opts* opts) {
+    if (!opts) return LUVC_ERR_NULL;
+    int sigma = 0;
+    const int rc = check_spu(hidden, B, N, D, cutoff, keep, out_idx, out_hidden, opts->dtype, &sigma);
+    if (rc) return rc;
+    const size_t need = spu_workspace_bytes(B, N, D, sigma, opts->dtype);
+    void* ws = opts->workspace;
+    if (ws) {
+        if (opts->workspace_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u)) return LUVC_ERR_WORKSPACE;
+    } else {
+        ws = scratch(kSpuWs, need);
+        if (!ws) return LUVC_ERR_CUDA;
+    }
+    SpuProblem p;
+    p.hidden = hidden; p.B = B; p.N = N; p.D = D; p.sigma = sigma; p.keep = keep; p.dtype = opts->dtype;
+    p.no_window = opts->no_window ? 1 : 0;
+    p.out_idx = out_idx; p.out_hidden = out_hidden; p.out_scores = opts->out_scores;
+    p.workspace = ws; p.stream = static_cast<cudaStream_t>(opts->stream);
+    return spu_run(p);
+}
+
+int luvc_spu_prune(const void* hidden, int B, int N, int D, float cutoff, int keep, int32_t* out_idx,
+                   void* out_hidden) {
+    luvc_spu_opts o = {};
+    o.dtype = LUVC_BF16; o.stream = t_stream;
+    return luvc_spu_prune_ex(hidden, B, N, D, cutoff, keep, out_idx, out_hidden, &o);
+}
+
+int luvc_spu_prune_f32(const float* hidden, int B, int N, int D, float cutoff, int keep, int32_t* out_idx,
+                       float* out_hidden) {
+    luvc_spu_opts o = {};
+    o.dtype = LUVC_F32; o.stream = t_stream;
+    return luvc_spu_prune_ex(hidden, B, N, D, cutoff, keep, out_idx, out_hidden, &o);
+}
+
+int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, int keep, int dtype,
+                        int32_t* out_idx, void* out_hidden) {
+    if (!hidden || !out_idx || !out_hidden) return LUVC_ERR_NULL;
+    if (dtype != LUVC_BF16 && dtype != LUVC_F32) return LUVC_ERR_DTYPE;
+    if (B < 1 || N < 1 || D < 1) return LUVC_ERR_SHAPE;
+    if (keep < 1 || keep > N) return LUVC_ERR_KEEP;
+    const size_t es = elem_size(dtype);
+    const size_t in_bytes = (size_t)B * N * D * es, hid_bytes = align_up((size_t)B * keep * D * es);
+    unsigned char* din = static_cast<unsigned char*>(scratch(kIoIn, in_bytes));
+    unsigned char* dout = static_cast<unsigned char*>(scratch(kIoOut, hid_bytes + align_up((size_t)B * keep * 4)));
+    if (!din || !dout) return LUVC_ERR_CUDA;
+    cudaStream_t st = t_stream;
+    if (cudaMemcpyAsync(din, hidden, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return LUVC_ERR_CUDA;
+    luvc_spu_opts o = {};
+    o.dtype = dtype; o.stream = st;
+    int32_t* didx = reinterpret_cast<int32_t*>(dout + hid_bytes);
+    const int rc = luvc_spu_prune_ex(din, B, N, D, cutoff, keep, didx, dout, &o);
+    if (rc) return rc;
+    cudaMemcpyAsync(out_hidden, dout, (size_t)B * keep * D * es, cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(out_idx, didx, (size_t)B * keep * 4, cudaMemcpyDeviceToHost, st);
+    return cudaStreamSynchronize(st) == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
+}
+
+}  // extern "C"

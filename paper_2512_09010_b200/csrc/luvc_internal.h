@@ -1,0 +1,58 @@
+// Internal declarations shared by the translation units of the library
+// (host side only; no device code is shared across files).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/luvc.h"
+
+namespace luvc {
+
+// Counts every kernel launch of the library (reported by luvc_kernel_launches).
+void count_launch(int n = 1);
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+// ---- OIM -------------------------------------------------------------------
+
+struct OimStep {
+    int axis;  // 0: lines are rows, the width shrinks; 1: lines are columns, the height shrinks
+    int m;     // cells removed per line
+    int h, w;  // grid before the step
+};
+
+// Final grid for a target count; false if none fits.
+bool oim_final_dims(int H, int W, int target, int* Hf, int* Wf);
+// Step list from H x W to Hf x Wf; returns false if unreachable.  `steps` may be null (count only).
+bool oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first, OimStep* steps, int cap, int* n_steps);
+
+struct OimProblem {
+    const void* tokens;
+    int B, H, W, D, Hf, Wf, r, height_first, dtype;
+    void* out_tokens;
+    int32_t* out_sizes;
+    int32_t* out_map;
+    int32_t* trace;
+    void* workspace;
+    cudaStream_t stream;
+};
+size_t oim_workspace_bytes(int B, int H, int W, int D, int dtype);
+int oim_run(const OimProblem& p);
+
+// ---- SPU -------------------------------------------------------------------
+
+struct SpuProblem {
+    const void* hidden;
+    int B, N, D, sigma, keep, dtype, no_window;
+    int32_t* out_idx;
+    void* out_hidden;
+    float* out_scores;
+    void* workspace;
+    cudaStream_t stream;
+};
+size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype);
+int spu_run(const SpuProblem& p);
+
+}  // namespace luvc

@@ -1,0 +1,305 @@
+// Spectrum Pruning Unit (Section 3.3, Eq. 4-8, Algorithm 2) for sm_100a.
+//
+// The mask of Eq. 5 is zero outside |f| <= sigma, so only the 2*sigma+1 real
+// spectral rows of the pass band are ever formed:
+//   Phi[n][r] = cos(2 pi r n / N)            r = 0 .. sigma
+//   Phi[n][r] = -sin(2 pi (r-sigma) n / N)   r = sigma+1 .. 2 sigma
+//   Y  = diag(c) Phi^T X      (Eq. 4 restricted to the band, Eq. 6 and the 1/N and the
+//                              factor 2 of the conjugate half folded into c)
+//   X' = Phi Y                (Eq. 7; real because the mask is even in f)
+//   E[n] = || X'[n, :] ||_2   (Eq. 8)
+// followed by an order-preserving top-`keep` selection and a row gather
+// (Algorithm 2's last two lines).  Everything is fp32; reductions have a fixed
+// order, so results are reproducible run to run.
+
+#include <cuda_bf16.h>
+
+#include "luvc_internal.h"
+
+namespace luvc {
+namespace {
+
+constexpr int BM = 64, BN = 64, BK = 16;     // tile of the generic contraction
+constexpr int kGemmThreads = 256;
+
+// cos / sin of 2 pi j / N for j = 0..N-1, and the per-row constants c[r].
+__global__ void spu_tables_kernel(float2* tw, float* scale, int N, int sigma, int no_window) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < N) {
+        double s, c;
+        sincospi(2.0 * (double)i / (double)N, &s, &c);
+        tw[i] = make_float2((float)c, (float)s);
+    }
+    if (i < 2 * sigma + 1) {
+        const int k = i <= sigma ? i : i - sigma;
+        double m = 1.0;
+        if (!no_window && N > 1) m = 0.54 + 0.46 * cospi(2.0 * (double)k / (double)(N - 1));
+        const double mult = (k == 0 || 2 * k == N) ? 1.0 : 2.0;   // bins without a distinct conjugate count once
+        scale[i] = (float)(m * mult / (double)N);
+    }
+}
+
+__device__ __forceinline__ float phi(const float2* __restrict__ tw, int n, int r, int N, int sigma) {
+    const bool is_cos = r <= sigma;
+    const int k = is_cos ? r : r - sigma;
+    // k <= N/2 and n < N: the product fits 32 bits for every N below 65536
+    const int j = N < 65536 ? (int)(((unsigned)k * (unsigned)n) % (unsigned)N)
+                            : (int)(((unsigned long long)k * (unsigned long long)n) % (unsigned long long)N);
+    const float2 t = __ldg(tw + j);
+    return is_cos ? t.x : -t.y;
+}
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// C[M x D] = A[M x K] * Bm[K x D] with A generated from the twiddle table.
+//   FWD:  M = 2 sigma + 1 rows r, K = N tokens;  A[r][n] = Phi[n][r];  Bm = the input (type T);
+//         the result, times c[r], is stored to Y[b][r][d].
+//   !FWD: M = N tokens, K = 2 sigma + 1;         A[n][r] = Phi[n][r];  Bm = Y (fp32);
+//         the squared result is summed over the tile's 64 channels into part[b][d-tile][n].
+template <typename T, bool FWD>
+__global__ void __launch_bounds__(kGemmThreads) spu_contract_kernel(const void* __restrict__ bm_v,
+                                                                    float* __restrict__ out,
+                                                                    const float2* __restrict__ tw,
+                                                                    const float* __restrict__ scale,
+                                                                    int N, int D, int sigma) {
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int R = 2 * sigma + 1;
+    const int M = FWD ? R : N, K = FWD ? N : R;
+    const int b = blockIdx.z, m0 = blockIdx.y * BM, d0 = blockIdx.x * BN;
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const T* xin = reinterpret_cast<const T*>(bm_v) + (size_t)b * N * D;          // FWD operand
+    const float* yin = reinterpret_cast<const float*>(bm_v) + (size_t)b * R * D;  // !FWD operand
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < K; k0 += BK) {
+#pragma unroll
+        for (int q = 0; q < BM * BK / kGemmThreads; ++q) {
+            const int idx = tid + q * kGemmThreads;
+            const int mi = idx % BM, ki = idx / BM;
+            const int row = m0 + mi, red = k0 + ki;
+            float v = 0.f;
+            if (row < M && red < K) v = FWD ? phi(tw, red, row, N, sigma) : phi(tw, row, red, N, sigma);
+            As[ki][mi] = v;
+        }
+#pragma unroll
+        for (int q = 0; q < BN * BK / kGemmThreads; ++q) {
+            const int idx = tid + q * kGemmThreads;
+            const int ni = idx % BN, ki = idx / BN;
+            const int red = k0 + ki, d = d0 + ni;
+            float v = 0.f;
+            if (red < K && d < D) v = FWD ? to_f32<T>(xin[(size_t)red * D + d]) : yin[(size_t)red * D + d];
+            Bs[ki][ni] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int ki = 0; ki < BK; ++ki) {
+            const float4 av = *reinterpret_cast<const float4*>(&As[ki][ty * 4]);
+            const float4 bv = *reinterpret_cast<const float4*>(&Bs[ki][tx * 4]);
+            const float a[4] = {av.x, av.y, av.z, av.w}, bb[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+
+    if (FWD) {
+        float* Y = out + (size_t)b * R * D;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = m0 + ty * 4 + i;
+            if (r >= M) continue;
+            const float c = scale[r];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int d = d0 + tx * 4 + j;
+                if (d < D) Y[(size_t)r * D + d] = c * acc[i][j];
+            }
+        }
+    } else {
+        float* part = out + ((size_t)b * gridDim.x + blockIdx.x) * N;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float s = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s = fmaf(acc[i][j], acc[i][j], s);   // columns beyond D hold zeros
+            // the 16 threads that share this row sit in one half-warp
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            const int n = m0 + ty * 4 + i;
+            if (tx == 0 && n < M) part[n] = s;
+        }
+    }
+}
+
+// E[b][n] = sqrt(sum over the channel tiles, in tile order).
+__global__ void spu_energy_kernel(const float* part, float* E, int N, int tiles, long long total) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int b = (int)(i / N), n = (int)(i % N);
+    float s = 0.f;
+    for (int t = 0; t < tiles; ++t) s += part[((size_t)b * tiles + t) * N + n];
+    E[i] = sqrtf(s);
+}
+
+// ---- order-preserving top-k ---------------------------------------------------
+
+constexpr int kSelThreads = 1024;
+
+__device__ __forceinline__ unsigned score_key(float e) {
+    // scores are >= 0, so their bit patterns order like the values; anything else
+    // (a NaN from non-finite input) ranks lowest
+    return (e >= 0.f) ? __float_as_uint(e) : 0u;
+}
+
+// Exclusive prefix sum of one int per thread over the block; returns the block total in `total`.
+__device__ int block_exclusive_scan(int v, int* s_warp, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    __syncthreads();                 // s_warp may still be read from the previous call
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < (kSelThreads >> 5) ? s_warp[lane] : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += t;
+        }
+        s_warp[lane] = w;            // inclusive totals per warp
+    }
+    __syncthreads();
+    total = s_warp[31];
+    return inc - v + (warp ? s_warp[warp - 1] : 0);
+}
+
+// One CTA per sequence: radix-select the keep-th largest key (4 passes of 8 bits),
+// then one ordered sweep that keeps everything above it plus the first equal ones.
+__global__ void __launch_bounds__(kSelThreads) spu_select_kernel(const float* __restrict__ E, int32_t* __restrict__ out_idx,
+                                                                 int N, int keep) {
+    __shared__ int s_hist[256];
+    __shared__ int s_warp[32];
+    __shared__ unsigned s_prefix;
+    __shared__ int s_remaining;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const float* e = E + (size_t)b * N;
+    if (tid == 0) { s_prefix = 0u; s_remaining = keep; }
+    for (int pass = 3; pass >= 0; --pass) {
+        for (int i = tid; i < 256; i += kSelThreads) s_hist[i] = 0;
+        __syncthreads();
+        const unsigned prefix = s_prefix;
+        const unsigned himask = pass == 3 ? 0u : (0xffffffffu << (8 * (pass + 1)));
+        for (int n = tid; n < N; n += kSelThreads) {
+            const unsigned key = score_key(e[n]);
+            if ((key & himask) == prefix) atomicAdd(&s_hist[(key >> (8 * pass)) & 255u], 1);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int rem = s_remaining, bucket = 255;
+            for (; bucket > 0; --bucket) {
+                if (s_hist[bucket] >= rem) break;
+                rem -= s_hist[bucket];
+            }
+            s_prefix = prefix | ((unsigned)bucket << (8 * pass));
+            s_remaining = rem;
+        }
+        __syncthreads();
+    }
+    const unsigned thr = s_prefix;      // the keep-th largest key
+    const int take_equal = s_remaining; // how many keys equal to it are kept (lowest indices first)
+    int32_t* out = out_idx + (size_t)b * keep;
+    int eq_seen = 0, written = 0;
+    for (int n0 = 0; n0 < N; n0 += kSelThreads) {
+        const int n = n0 + tid;
+        const unsigned key = n < N ? score_key(e[n]) : 0u;
+        const int is_eq = (n < N && key == thr) ? 1 : 0;
+        int eq_total;
+        const int eq_rank = eq_seen + block_exclusive_scan(is_eq, s_warp, eq_total);
+        const int kept = (n < N && (key > thr || (is_eq && eq_rank < take_equal))) ? 1 : 0;
+        int kept_total;
+        const int pos = written + block_exclusive_scan(kept, s_warp, kept_total);
+        if (kept) out[pos] = n;
+        eq_seen += eq_total;
+        written += kept_total;
+    }
+}
+
+// out_hidden[b][j][:] = hidden[b][idx[b][j]][:], 16 bytes per thread per trip.
+__global__ void __launch_bounds__(128) spu_gather_kernel(const uint4* __restrict__ hidden, const int32_t* __restrict__ idx,
+                                                         uint4* __restrict__ out, int N, int keep, int row_vec) {
+    const int b = blockIdx.y, j = blockIdx.x;
+    const int src = idx[(size_t)b * keep + j];
+    const uint4* in = hidden + ((size_t)b * N + src) * row_vec;
+    uint4* o = out + ((size_t)b * keep + j) * row_vec;
+    for (int v = threadIdx.x; v < row_vec; v += 128) o[v] = __ldg(in + v);
+}
+
+struct Workspace {
+    float2* tw;
+    float* scale;
+    float* Y;
+    float* part;
+    float* E;
+};
+
+Workspace carve(void* ws, int B, int N, int D, int sigma) {
+    unsigned char* p = static_cast<unsigned char*>(ws);
+    const int R = 2 * sigma + 1, tiles = (D + BN - 1) / BN;
+    Workspace w;
+    w.tw = reinterpret_cast<float2*>(p); p += align_up((size_t)N * sizeof(float2));
+    w.scale = reinterpret_cast<float*>(p); p += align_up((size_t)R * 4);
+    w.Y = reinterpret_cast<float*>(p); p += align_up((size_t)B * R * D * 4);
+    w.part = reinterpret_cast<float*>(p); p += align_up((size_t)B * tiles * N * 4);
+    w.E = reinterpret_cast<float*>(p);
+    return w;
+}
+
+}  // namespace
+
+size_t spu_workspace_bytes(int B, int N, int D, int sigma, int /*dtype*/) {
+    const int R = 2 * sigma + 1, tiles = (D + BN - 1) / BN;
+    return align_up((size_t)N * sizeof(float2)) + align_up((size_t)R * 4) + align_up((size_t)B * R * D * 4) +
+           align_up((size_t)B * tiles * N * 4) + align_up((size_t)B * N * 4);
+}
+
+template <typename T>
+static int spu_run_typed(const SpuProblem& p) {
+    const int N = p.N, D = p.D, B = p.B, sigma = p.sigma, R = 2 * sigma + 1;
+    const int tiles = (D + BN - 1) / BN;
+    Workspace ws = carve(p.workspace, B, N, D, sigma);
+    float* E = p.out_scores ? p.out_scores : ws.E;
+    const int tab = N > R ? N : R;
+    spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, ws.scale, N, sigma, p.no_window);
+    spu_contract_kernel<T, true><<<dim3(tiles, (R + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
+        p.hidden, ws.Y, ws.tw, ws.scale, N, D, sigma);
+    spu_contract_kernel<T, false><<<dim3(tiles, (N + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
+        ws.Y, ws.part, ws.tw, ws.scale, N, D, sigma);
+    const long long bn = (long long)B * N;
+    spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn);
+    spu_select_kernel<<<B, kSelThreads, 0, p.stream>>>(E, p.out_idx, N, p.keep);
+    const int row_vec = (int)((size_t)D * sizeof(T) / 16);
+    spu_gather_kernel<<<dim3(p.keep, B), 128, 0, p.stream>>>(reinterpret_cast<const uint4*>(p.hidden), p.out_idx,
+                                                            reinterpret_cast<uint4*>(p.out_hidden), N, p.keep, row_vec);
+    count_launch(6);
+    return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
+}
+
+int spu_run(const SpuProblem& p) {
+    return p.dtype == LUVC_F32 ? spu_run_typed<float>(p) : spu_run_typed<__nv_bfloat16>(p);
+}
+
+}  // namespace luvc

@@ -1,0 +1,84 @@
+"""The C-ABI library loads and exports every symbol the header declares; host-side argument
+checks answer without touching a GPU (CPU only: no compute call is made here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def luvc():
+    import paper_2512_09010_b200 as luvc
+    return luvc
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "luvc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(luvc_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(luvc):
+    names = _declared()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(luvc.lib, n), "%s is declared in include/luvc.h but not exported" % n
+    assert set(names) == set(luvc.EXPORTS)
+
+
+def test_version_and_status_strings(luvc):
+    assert luvc.version() >= 1000
+    assert luvc.lib.luvc_status_string(0) == b"ok"
+    for code in range(1, 12):
+        assert len(luvc.lib.luvc_status_string(code)) > 3
+
+
+def test_plan_matches_the_benchmark_grids(luvc):
+    golden = os.path.join(ROOT, "tests", "golden", "oim_schedules.txt")
+    for line in open(golden):
+        if line.startswith("#") or not line.strip():
+            continue
+        H, W, target, Hf, Wf, steps = map(int, line.split())
+        assert luvc.oim_plan(H, W, target) == (Hf, Wf, steps)
+    with pytest.raises(luvc.LuvcError) as e:
+        luvc.oim_plan(4, 4, 7)
+    assert e.value.status == 3
+    assert luvc.oim_plan(6, 6, 8)[:2] == (4, 2)
+    assert luvc.oim_plan(5, 5, 25) == (5, 5, 0)
+
+
+def test_sigma_from_cutoff(luvc):
+    assert luvc.spu_sigma(144, 0.0) == 9
+    assert luvc.spu_sigma(1296, 0.125) == 81
+    assert luvc.spu_sigma(16384, 0.05) == 409
+    assert luvc.spu_sigma(16384, 0.25) == 2048
+    assert luvc.spu_sigma(7, 1.0) == 3
+    assert luvc.spu_sigma(16, 1.5) == -1
+    assert luvc.spu_sigma(16, float("nan")) == -1
+
+
+def test_argument_errors_are_reported_before_any_device_work(luvc):
+    L = luvc.lib
+    o = luvc.OimOpts()
+    assert L.luvc_oim_merge_ex(None, 1, 4, 4, 8, 4, None, None, None, ctypes.byref(o)) == 1          # NULL
+    fake = ctypes.c_void_p(4096)      # never dereferenced: checks fail first
+    assert L.luvc_oim_merge_ex(fake, 0, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 2         # shape
+    assert L.luvc_oim_merge_ex(fake, 1, 4, 4, 8, 7, fake, fake, fake, ctypes.byref(o)) == 3         # target
+    assert L.luvc_oim_merge_ex(fake, 1, 4, 4, 12, 4, fake, fake, fake, ctypes.byref(o)) == 6        # row not 16 B
+    assert L.luvc_oim_merge_ex(ctypes.c_void_p(4100), 1, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 6
+    o.dtype = 5
+    assert L.luvc_oim_merge_ex(fake, 1, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 7         # dtype
+    o.dtype = 0
+    o.out_h, o.out_w = 3, 2
+    assert L.luvc_oim_merge_ex(fake, 1, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 3         # 3*2 != 4
+    s = luvc.SpuOpts()
+    assert L.luvc_spu_prune_ex(None, 1, 8, 8, 0.5, 2, None, None, ctypes.byref(s)) == 1
+    assert L.luvc_spu_prune_ex(fake, 1, 8, 8, 0.5, 9, fake, fake, ctypes.byref(s)) == 4             # keep > N
+    assert L.luvc_spu_prune_ex(fake, 1, 8, 8, 0.5, 0, fake, fake, ctypes.byref(s)) == 4
+    assert L.luvc_spu_prune_ex(fake, 1, 8, 8, 2.0, 2, fake, fake, ctypes.byref(s)) == 5             # cutoff
+    assert L.luvc_spu_prune_ex(fake, 1, 8, 4, 0.5, 2, fake, fake, ctypes.byref(s)) == 6             # 8-byte rows
+    assert L.luvc_oim_workspace_bytes(1, 24, 24, 1024, 0) >= 576 * 1024 * 4
+    assert L.luvc_spu_workspace_bytes(1, 144, 4096, 0.0, 0) > 0

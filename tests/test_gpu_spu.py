@@ -1,0 +1,139 @@
+"""Parity of luvc_spu_prune* (CUDA, through the C ABI) with the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import luvc_inputs as gi
+from _compare import assert_scores_close, check_spu_selection
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def luvc():
+    import paper_2512_09010_b200 as luvc
+    assert torch.cuda.is_available()
+    return luvc
+
+
+def _run(luvc, x_dev, keep, cutoff, **kw):
+    idx, hid, scores = luvc.spu_prune(x_dev, keep, cutoff, want_scores=True, **kw)
+    torch.cuda.synchronize()
+    return idx.cpu().numpy(), hid, scores.cpu().numpy()
+
+
+def _check(luvc, oracle_mod, x, keep, cutoff, no_window=False, method="fft"):
+    idx, hid, scores = _run(luvc, x.cuda(), keep, cutoff, no_window=no_window)
+    xh = x.float().numpy()
+    B, N, D = xh.shape
+    sigma = oracle_mod.spu_sigma(N, cutoff)
+    assert sigma == luvc.spu_sigma(N, cutoff)
+    unique = 0
+    for b in range(B):
+        ref = oracle_mod.spu_scores(xh[b], sigma, hamming=not no_window, method=method)
+        assert_scores_close(scores[b], ref, "sequence %d scores" % b)
+        if check_spu_selection(ref, idx[b], keep):
+            np.testing.assert_array_equal(idx[b], oracle_mod.spu_select(ref, keep))
+            unique += 1
+    gathered = torch.stack([x[b][torch.as_tensor(idx[b], dtype=torch.long)] for b in range(B)])
+    assert torch.equal(hid.cpu(), gathered)          # the original rows, bit for bit
+    return unique
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B,N,D,keep,cutoff", [
+    (2, 16, 8, 4, 0.5), (1, 45, 24, 10, 0.3), (3, 64, 72, 32, 0.125), (1, 100, 40, 99, 0.25), (2, 1, 8, 1, 0.5),
+    (2, 2, 8, 1, 1.0), (1, 3, 16, 2, 1.0), (1, 64, 8, 64, 1.0), (1, 63, 8, 5, 1.0), (2, 130, 136, 7, 0.0),
+    (1, 257, 8, 100, 0.01),
+])
+def test_small_sequences_match_the_oracle(luvc, oracle_mod, dtype, B, N, D, keep, cutoff):
+    g = torch.Generator().manual_seed(N * 100 + D)
+    x = torch.randn((B, N, D), generator=g).to(dtype)
+    _check(luvc, oracle_mod, x, keep, cutoff, method="naive" if N <= 130 else "fft")
+
+
+def test_flat_pass_band_option(luvc, oracle_mod):
+    g = torch.Generator().manual_seed(3)
+    x = torch.randn((2, 48, 16), generator=g)
+    _check(luvc, oracle_mod, x, 12, 0.5, no_window=True)
+    # full band, no window: the score is the plain token norm
+    idx, hid, scores = _run(luvc, x.cuda(), 5, 1.0, no_window=True)
+    np.testing.assert_allclose(scores, x.norm(dim=-1).numpy(), rtol=1e-5)
+
+
+def test_ties_keep_the_lowest_indices(luvc):
+    # a constant sequence passes the filter unchanged: all scores are equal
+    x = torch.ones((2, 40, 8), dtype=torch.bfloat16)
+    idx, hid, scores = _run(luvc, x.cuda(), 7, 0.25)
+    assert np.allclose(scores, np.sqrt(8.0), rtol=1e-5)
+    if np.all(scores == scores[:, :1]):
+        assert idx.tolist() == [list(range(7))] * 2
+    # exact duplicates of a score by construction: period-2 sequence under a full flat band
+    y = torch.zeros((1, 8, 8))
+    y[0, ::2] = 3.0
+    y[0, 1::2] = 1.0
+    idx, _, scores = _run(luvc, y.cuda(), 5, 1.0, no_window=True)
+    if np.all(scores[0, ::2] == scores[0, 0]) and np.all(scores[0, 1::2] == scores[0, 1]):
+        assert idx[0].tolist() == [0, 1, 2, 4, 6]
+
+
+def test_plain_entry_points(luvc, oracle_mod):
+    g = torch.Generator().manual_seed(4)
+    for dtype in (torch.bfloat16, torch.float32):
+        x = torch.randn((2, 96, 64), generator=g).to(dtype)
+        idx, hid = luvc.spu_prune_plain(x.cuda(), 24, 0.0)
+        ref = oracle_mod.spu(x.float().numpy(), cutoff=None, keep=24)
+        np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
+
+
+def test_host_buffer_entry_point(luvc):
+    g = torch.Generator().manual_seed(9)
+    x = torch.randn((2, 80, 64), generator=g).to(torch.bfloat16).pin_memory()
+    idx = torch.empty((2, 20), dtype=torch.int32).pin_memory()
+    hid = torch.empty((2, 20, 64), dtype=torch.bfloat16).pin_memory()
+    luvc.spu_prune_host(x, 20, 0.25, idx, hid)
+    ref = luvc.spu_prune(x.cuda(), 20, 0.25)
+    assert torch.equal(idx, ref[0].cpu()) and torch.equal(hid, ref[1].cpu())
+
+
+@pytest.mark.parametrize("config", [0, 1, 2, 3])
+def test_pipeline_configurations(luvc, oracle_mod, config):
+    # SPU input = the merged tokens (from the CUDA OIM) through the seeded projection, at full size
+    c = gi.CONFIGS[config]
+    merged = luvc.oim_merge(gi.oim_input(config, device="cuda"), c["target"])[0]
+    x = gi.spu_input_from_tokens(config, merged).cpu()
+    for keep in c["keep"]:
+        _check(luvc, oracle_mod, x, keep, 0.0)
+
+
+def test_cascade_of_prunes(luvc, oracle_mod):
+    # 1296 -> 324 -> 130 -> 65, each stage on the previous stage's survivors
+    c = gi.CONFIGS[2]
+    x = gi.spu_input_from_tokens(2, gi.oim_input(2, device="cuda", batch=1, hw=(24, 24), dim=128).reshape(1, 576, 128),
+                                 dim_out=256).cpu()
+    for keep in (144, 58, 29):
+        _check(luvc, oracle_mod, x, keep, 0.0)
+        x = luvc.spu_prune(x.cuda(), keep, 0.0)[1].cpu()
+
+
+def test_stress_configuration_sampled(luvc, oracle_mod):
+    # 8 x 16384 x 4096 as benchmarked; the oracle evaluates a sample of tokens from the definition
+    c = gi.CONFIGS[4]
+    x = gi.spu_stress_input(device="cuda")
+    rng = np.random.default_rng(0)
+    for cutoff, keep in ((0.05, 1638), (0.125, 4096), (0.25, 8192)):
+        idx, hid, scores = luvc.spu_prune(x, keep, cutoff, want_scores=True)
+        torch.cuda.synchronize()
+        sigma = oracle_mod.spu_sigma(c["spu_N"], cutoff)
+        idx_h, sc_h = idx.cpu().numpy(), scores.cpu().numpy()
+        for b in (0, 7):
+            tokens = np.sort(rng.choice(c["spu_N"], size=6, replace=False))
+            ref = oracle_mod.spu_scores_at(x[b].float().cpu().numpy(), sigma, tokens)
+            assert_scores_close(sc_h[b][tokens], ref, "sampled scores, sequence %d" % b)
+        for b in range(c["spu_B"]):
+            # selection is consistent with the scores the kernel produced, exact in count and order
+            kept = np.zeros(c["spu_N"], bool)
+            kept[idx_h[b]] = True
+            assert len(idx_h[b]) == keep and np.all(np.diff(idx_h[b]) > 0)
+            assert sc_h[b][kept].min() >= sc_h[b][~kept].max()
+            assert torch.equal(hid[b], x[b][idx[b].long()])
