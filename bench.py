@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the LUVC hot path (OIM + SPU) on B200.
+
+One step = one pass of the whole path over one batch of a configuration: luvc_oim_merge on the
+visual-encoder grid, then luvc_spu_prune on the LLM-side hidden states of the merged tokens
+(configurations 2 and 3; the seeded projection between the two stands in for the projector and
+is not timed), or the two stress operators back to back (configuration 4).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is vision tokens per second with inputs resident in HBM,
+timed with CUDA events on the launching stream; `e2e` is the same metric through the host-buffer
+C-ABI entry points (host->device and device->host copies inside the timed region); `roofline`
+describes the dominant kernel (the OIM merge-step kernel) against the measured HBM copy rate;
+`cpu_baseline` is the CPU oracle timed on this machine's host cores on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "vision tokens/sec through OIM+SPU"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+HBM_NOMINAL_GBS = 8000.0      # the figure the metric's "% of 8 TB/s" divides by
+HBM_FALLBACK_GBS = 6650.0     # used only if MEASURED_PEAKS.json is absent
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (null until a capture for that workload exists).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4])
+    ap.add_argument("--impl", default="luvc", choices=["luvc", "reference"])
+    ap.add_argument("--cpu-sample", type=int, default=0, help="units of the batch the CPU oracle is timed on (0 = auto)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+# ----------------------------------------------------------------------------- workloads
+
+
+def workload_spec(k):
+    import luvc_inputs as gi
+
+    c = gi.CONFIGS[k]
+    spec = dict(id=k, oim=(c["B"], c["H"], c["W"], c["D"]), target=c["target"], keep=c["keep"][0], cutoff=0.0)
+    if k == 4:
+        spec["spu"] = (c["spu_B"], c["spu_N"], c["D_llm"])
+        spec["cutoff"] = c["cutoffs"][0]
+        spec["tokens"] = c["B"] * c["H"] * c["W"] + c["spu_B"] * c["spu_N"]
+    else:
+        T = c["target"]
+        spec["spu"] = (c["B"] // c.get("frames", 1), T * c.get("frames", 1), c["D_llm"])
+        spec["tokens"] = c["B"] * c["H"] * c["W"]
+    return spec
+
+
+def workload_name(spec):
+    B, H, W, D = spec["oim"]
+    sb, sn, sd = spec["spu"]
+    cut = spec["cutoff"] if spec["cutoff"] > 0 else 0.125
+    return ("configs[%d]: OIM %dx%dx%dx%d -> %d tokens/grid, then SPU %dx%dx%d keep %d at cutoff %g%s" % (
+        spec["id"], B, H, W, D, spec["target"], sb, sn, sd, spec["keep"], cut,
+        " (independent stress inputs)" if spec["id"] == 4 else " (merged tokens through the seeded projection)"))
+
+
+def oim_iter_bytes(luvc, B, H, W, D, target, e=2):
+    """Algorithmic bytes of the OIM chain: every step reads its grid and writes the compacted one,
+    tokens plus the int32 size per token."""
+    Hf, Wf, n_steps = luvc.oim_plan(H, W, target)
+    h, w, total = H, W, 0
+    while (h, w) != (Hf, Wf):
+        for axis in (0, 1):
+            ln, goal = (w, Wf) if axis == 0 else (h, Hf)
+            m = min(2, ln - goal, (ln + 1) // 2)
+            if ln < 2 or m <= 0:
+                continue
+            nh, nw = (h, w - m) if axis == 0 else (h - m, w)
+            total += B * (h * w + nh * nw) * (D * e + 4)
+            h, w = nh, nw
+    return total, n_steps
+
+
+def make_inputs(spec, device, sets):
+    """`sets` independent input sets (different seeds via batch rolls) so that consecutive steps do
+    not find their inputs in L2."""
+    import torch
+
+    import luvc_inputs as gi
+    import paper_2512_09010_b200 as luvc
+
+    k = spec["id"]
+    x0 = gi.oim_input(k, device=device)
+    xs = [x0] + [torch.roll(x0, shifts=(s, 3 * s, 5 * s), dims=(0, 1, 2)).contiguous() for s in range(1, sets)]
+    if k == 4:
+        y0 = gi.spu_stress_input(device=device)
+        ys = [y0] + [torch.roll(y0, shifts=(s, 17 * s), dims=(0, 1)).contiguous() for s in range(1, sets)]
+    else:
+        ys = []
+        for x in xs:
+            merged = luvc.oim_merge(x, spec["target"])[0]
+            ys.append(gi.spu_input_from_tokens(k, merged))
+    torch.cuda.synchronize()
+    return xs, ys
+
+
+# ----------------------------------------------------------------------------- clocks
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, device_index):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as exc:  # no NVML: report that clocks were not sampled
+            self.err = str(exc)
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for name, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop_evt.wait(0.01)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+
+
+def cpu_oracle_pass(spec, sample_units, x_host, y_host, min_seconds=0.0):
+    """Times the CPU oracle (as it stands) on `sample_units` images and the matching sequences."""
+    import oracle
+
+    B = spec["oim"][0]
+    sb = spec["spu"][0]
+    n_img = max(1, min(sample_units, B))
+    n_seq = n_img if spec["id"] == 4 else max(1, min(sb, (n_img * sb + B - 1) // B))
+    n_seq = min(n_seq, len(y_host))
+    cores = oracle.hardware_threads()
+    sigma = oracle.spu_sigma(spec["spu"][1], spec["cutoff"])
+    t_oim = t_spu = 0.0
+    reps = 0
+    while reps < 1 or (t_oim + t_spu < min_seconds and reps < 50):   # repeat the sample until the clock is steady
+        t0 = time.perf_counter()
+        oracle.oim(x_host[:n_img], target=spec["target"])
+        t1 = time.perf_counter()
+        for b in range(n_seq):
+            e = oracle.spu_scores(y_host[b], sigma)
+            idx = oracle.spu_select(e, spec["keep"])
+            _ = y_host[b][idx]
+        t2 = time.perf_counter()
+        t_oim += t1 - t0
+        t_spu += t2 - t1
+        reps += 1
+    if spec["id"] == 4:
+        tokens = n_img * spec["oim"][1] * spec["oim"][2] + n_seq * spec["spu"][1]
+    else:
+        tokens = n_img * spec["oim"][1] * spec["oim"][2]      # the sequences are those same grids, merged
+    return dict(seconds=t_oim + t_spu, oim_seconds=t_oim, spu_seconds=t_spu, tokens=tokens * reps, cores=cores,
+                sample="%d of %d grids through the OIM oracle, %d of %d sequences through the SPU oracle (FFT method), "
+                       "repeated %d times" % (n_img, B, n_seq, sb, reps))
+
+
+def auto_cpu_sample(spec):
+    return {1: 32, 2: 8, 3: 16, 4: 1}[spec["id"]]
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+
+    import luvc_inputs as gi
+    import oracle
+
+    spec = workload_spec(args.workload)
+    k = spec["id"]
+    sample = args.cpu_sample or max(1, auto_cpu_sample(spec) // 4)
+    B = spec["oim"][0]
+    n_img = min(sample, B)
+    x = gi.oim_input(k, batch=n_img).float().numpy()
+    if k == 4:
+        y = gi.spu_stress_input(batch=1).float().numpy()
+    else:
+        merged = torch.from_numpy(oracle.oim(x, target=spec["target"])["tokens"]).float()
+        y = gi.spu_input_from_tokens(k, merged).float().numpy()
+    for _ in range(min(args.warmup, 1)):
+        cpu_oracle_pass(spec, n_img, x, y)
+    steps = max(1, min(args.steps, 3))
+    secs, tokens, info = 0.0, 0.0, None
+    for _ in range(steps):
+        info = cpu_oracle_pass(spec, n_img, x, y)
+        secs += info["seconds"]
+        tokens += info["tokens"]
+    value = tokens / secs
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * secs / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(spec), "note": "CPU oracle on a bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": info["cores"], "kind": "oracle", "sample": info["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- the GPU arm
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2512_09010_b200 as luvc
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    spec = workload_spec(args.workload)
+    k = spec["id"]
+    B, H, W, D = spec["oim"]
+    sb, sn, sd = spec["spu"]
+    e = 2
+    oim_in_bytes = B * H * W * D * e
+    spu_in_bytes = sb * sn * sd * e
+    sets = max(2, -(-3 * L2_BYTES // max(1, oim_in_bytes + spu_in_bytes)) if k != 4 else 2)
+    sets = min(sets, 8)
+    xs, ys = make_inputs(spec, device, sets)
+
+    def step(i):
+        x, y = xs[i % sets], ys[i % sets]
+        a = luvc.oim_merge(x, spec["target"])
+        b = luvc.spu_prune(y, spec["keep"], spec["cutoff"])
+        return a, b
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+
+    # ---- timed region: K steps back to back, CUDA events on the launching stream
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = luvc.kernel_launches()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = luvc.kernel_launches() - launches0
+    clocks = sampler.stop()
+    t = torch.tensor([ms_total], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * spec["tokens"] / (ms_per_step * 1e-3)
+
+    # ---- per-phase pass: the library's own events around its phases, one step at a time
+    luvc.profile_enable(True)
+    phases = {name: 0.0 for name in luvc.PHASES}
+    reps = min(args.steps, 20)
+    for i in range(reps):
+        step(i)
+        got = luvc.profile_read()
+        for name in phases:
+            phases[name] += got[name] / reps
+    luvc.profile_enable(False)
+
+    # ---- end to end: host buffers through the C ABI, copies inside the timed region
+    x_host = xs[0].cpu().pin_memory()
+    y_host = ys[0].cpu().pin_memory()
+    T = spec["target"]
+    o_tok = torch.empty((B, T, D), dtype=xs[0].dtype).pin_memory()
+    o_sz = torch.empty((B, T), dtype=torch.int32).pin_memory()
+    o_map = torch.empty((B, H * W), dtype=torch.int32).pin_memory()
+    o_idx = torch.empty((sb, spec["keep"]), dtype=torch.int32).pin_memory()
+    o_hid = torch.empty((sb, spec["keep"], sd), dtype=ys[0].dtype).pin_memory()
+
+    def e2e_step():
+        luvc.oim_merge_host(x_host, T, o_tok, o_sz, o_map)
+        luvc.spu_prune_host(y_host, spec["keep"], spec["cutoff"], o_idx, o_hid)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e2e_reps = max(3, min(args.steps, 20))
+    ev0.record()
+    for _ in range(e2e_reps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    t = torch.tensor([ev0.elapsed_time(ev1) / e2e_reps], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item())
+    h2d = x_host.numel() * 2 + y_host.numel() * 2
+    d2h = sum(t_.numel() * t_.element_size() for t_ in (o_tok, o_sz, o_map, o_idx, o_hid))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = HBM_FALLBACK_GBS, "fallback"
+    iter_bytes, n_steps = oim_iter_bytes(luvc, B, H, W, D, spec["target"], e)
+    floor_bytes = B * H * W * D * e + B * T * (D * e + 4) + B * H * W * 4
+    steps_ms = phases["oim_steps"]
+    achieved = iter_bytes / (steps_ms * 1e-3) / 1e9 if steps_ms > 0 else None
+    spu_bytes = spu_in_bytes + sb * sn * 4 + 2 * sb * spec["keep"] * sd * e + sb * spec["keep"] * 4
+    spu_ms = phases["spu_transform"] + phases["spu_select"] + phases["spu_gather"]
+    roofline = {
+        "kernel": "oim_step_kernel (%d launches per step)" % n_steps,
+        "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak if achieved else None, "peak_source": peak_src,
+        "frac_of_8TBs": achieved / HBM_NOMINAL_GBS if achieved else None,
+        "algorithmic_bytes_per_launch": iter_bytes / n_steps, "avg_launch_ms": steps_ms / n_steps,
+        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(k),
+        "floor_bytes": floor_bytes,
+        "spu": {"algorithmic_bytes": spu_bytes, "ms": spu_ms,
+                "achieved": spu_bytes / (spu_ms * 1e-3) / 1e9 if spu_ms > 0 else None,
+                "frac": spu_bytes / (spu_ms * 1e-3) / 1e9 / peak if spu_ms > 0 else None},
+    }
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        sample = args.cpu_sample or auto_cpu_sample(spec)
+        info = cpu_oracle_pass(spec, sample, xs[0][:sample].float().cpu().numpy(),
+                               ys[0][: max(1, sample)].float().cpu().numpy(), min_seconds=10.0)
+        cpu = {"value": info["tokens"] / info["seconds"], "unit": UNIT, "cores": info["cores"], "kind": "oracle",
+               "sample": info["sample"], "seconds": info["seconds"]}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 arithmetic on bf16 I/O", "data": "synthetic",
+        "config": {"workload": workload_name(spec), "l2": "inputs rotate over %d distinct sets (%.0f MB) > L2" % (
+            sets, sets * (oim_in_bytes + spu_in_bytes) / 1e6), "parallelism": "batch split, no collective" if world > 1 else "1 GPU"},
+        "clocks": clocks,
+        "e2e": {"value": world * spec["tokens"] / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "phases_ms": phases,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

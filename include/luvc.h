@@ -80,6 +80,22 @@ int luvc_shutdown(void);
 /* Number of kernels this library has launched since it was loaded (all threads). */
 long long luvc_kernel_launches(void);
 
+/* Phase timing for benchmarks.  While enabled, every operator call records CUDA
+ * events on its stream around its phases (two event records per phase, nothing
+ * else changes).  luvc_profile_read synchronises those events and returns the
+ * elapsed milliseconds of the most recent call's phases, indexed by luvc_phase;
+ * phases that did not run since the last read are reported as 0. */
+typedef enum {
+    LUVC_PHASE_OIM_STEPS = 0,      /* all merge-step launches of one luvc_oim_merge* call */
+    LUVC_PHASE_OIM_TOTAL = 1,      /* the whole call: init, steps, emit, map */
+    LUVC_PHASE_SPU_TRANSFORM = 2,  /* tables, forward band DFT, inverse, energies */
+    LUVC_PHASE_SPU_SELECT = 3,
+    LUVC_PHASE_SPU_GATHER = 4,
+    LUVC_PHASE_COUNT = 5
+} luvc_phase;
+int luvc_profile_enable(int on);
+int luvc_profile_read(float* ms, int count);
+
 /* ---- OIM ---------------------------------------------------------------- */
 
 /* Host-only planning.  Maps target_count to the final grid out_h x out_w: the

@@ -26,6 +26,7 @@ STATUS_NAMES = {
 # every symbol include/luvc.h declares
 EXPORTS = (
     "luvc_version", "luvc_status_string", "luvc_set_stream", "luvc_shutdown", "luvc_kernel_launches",
+    "luvc_profile_enable", "luvc_profile_read",
     "luvc_oim_plan", "luvc_oim_workspace_bytes", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
     "luvc_oim_merge_host", "luvc_spu_sigma", "luvc_spu_workspace_bytes", "luvc_spu_prune",
     "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host",
@@ -69,6 +70,8 @@ def _load() -> ctypes.CDLL:
     L.luvc_status_string.argtypes = [i]
     L.luvc_set_stream.argtypes = [p]
     L.luvc_kernel_launches.restype = ctypes.c_longlong
+    L.luvc_profile_enable.argtypes = [i]
+    L.luvc_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), i]
     L.luvc_oim_plan.argtypes = [i, i, i, i, ctypes.POINTER(i), ctypes.POINTER(i), ctypes.POINTER(i)]
     L.luvc_oim_workspace_bytes.restype = sz
     L.luvc_oim_workspace_bytes.argtypes = [i, i, i, i, i]
@@ -116,6 +119,20 @@ def kernel_launches() -> int:
 
 def shutdown() -> None:
     _check(lib.luvc_shutdown(), "luvc_shutdown")
+
+
+PHASES = ("oim_steps", "oim_total", "spu_transform", "spu_select", "spu_gather")
+
+
+def profile_enable(on: bool) -> None:
+    _check(lib.luvc_profile_enable(int(bool(on))), "luvc_profile_enable")
+
+
+def profile_read() -> dict:
+    """Elapsed milliseconds of the phases of the most recent calls (synchronises their events)."""
+    buf = (ctypes.c_float * len(PHASES))()
+    _check(lib.luvc_profile_read(buf, len(PHASES)), "luvc_profile_read")
+    return {name: float(buf[k]) for k, name in enumerate(PHASES)}
 
 
 def oim_plan(H: int, W: int, target_count: int, merge_per_step: int = 0):

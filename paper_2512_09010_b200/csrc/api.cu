@@ -12,6 +12,29 @@ namespace luvc {
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+static std::atomic<int> g_profile{0};
+static cudaEvent_t g_ev[LUVC_PHASE_COUNT][2];
+static bool g_ev_made = false, g_ev_used[LUVC_PHASE_COUNT];
+static std::mutex g_ev_mutex;
+
+void phase_begin(int phase, cudaStream_t stream) {
+    if (!g_profile.load(std::memory_order_relaxed)) return;
+    std::lock_guard<std::mutex> lock(g_ev_mutex);
+    if (!g_ev_made) {
+        for (auto& pair : g_ev) { cudaEventCreate(&pair[0]); cudaEventCreate(&pair[1]); }
+        g_ev_made = true;
+    }
+    cudaEventRecord(g_ev[phase][0], stream);
+}
+
+void phase_end(int phase, cudaStream_t stream) {
+    if (!g_profile.load(std::memory_order_relaxed)) return;
+    std::lock_guard<std::mutex> lock(g_ev_mutex);
+    if (!g_ev_made) return;
+    cudaEventRecord(g_ev[phase][1], stream);
+    g_ev_used[phase] = true;
+}
+
 namespace {
 
 thread_local cudaStream_t t_stream = nullptr;
@@ -119,6 +142,24 @@ int luvc_shutdown(void) {
 }
 
 long long luvc_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int luvc_profile_enable(int on) {
+    g_profile.store(on ? 1 : 0, std::memory_order_relaxed);
+    return LUVC_OK;
+}
+
+int luvc_profile_read(float* ms, int count) {
+    if (!ms) return LUVC_ERR_NULL;
+    std::lock_guard<std::mutex> lock(g_ev_mutex);
+    for (int i = 0; i < count; ++i) {
+        ms[i] = 0.f;
+        if (i >= LUVC_PHASE_COUNT || !g_ev_made || !g_ev_used[i]) continue;
+        if (cudaEventSynchronize(g_ev[i][1]) != cudaSuccess) return LUVC_ERR_CUDA;
+        if (cudaEventElapsedTime(&ms[i], g_ev[i][0], g_ev[i][1]) != cudaSuccess) return LUVC_ERR_CUDA;
+        g_ev_used[i] = false;
+    }
+    return LUVC_OK;
+}
 
 // ---- OIM ---------------------------------------------------------------------
 

@@ -13,6 +13,10 @@ namespace luvc {
 // Counts every kernel launch of the library (reported by luvc_kernel_launches).
 void count_launch(int n = 1);
 
+// Phase timing (luvc_profile_*): no-ops unless enabled.
+void phase_begin(int phase, cudaStream_t stream);
+void phase_end(int phase, cudaStream_t stream);
+
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 // ---- OIM -------------------------------------------------------------------

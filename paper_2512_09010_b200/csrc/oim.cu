@@ -82,8 +82,56 @@ struct StepArgs {
     int h, w, axis, m, D, HW;
 };
 
-template <typename T>
-__global__ void __launch_bounds__(kStepThreads) oim_step_kernel(const StepArgs a) {
+// |x|^2 and <x, y> over one lane's share of two vectors.  NCHUNK > 0: D == NCHUNK * 32 * kVec and
+// the loop is fully unrolled so that all of a lane's loads are in flight together.
+template <typename T, int NCHUNK>
+__device__ __forceinline__ void pair_stats(const T* __restrict__ t0, const float* __restrict__ a0, bool m0,
+                                           const T* __restrict__ t1, const float* __restrict__ a1, bool m1,
+                                           bool has_next, int lane, int D, float& nn, float& dd) {
+    constexpr int V = Elem<T>::kVec;
+    if (has_next) {
+        if constexpr (NCHUNK > 0) {
+#pragma unroll
+            for (int c = 0; c < NCHUNK; ++c) {
+                float x[V], y[V];
+                load_vec<T>(t0, a0, m0, (c * 32 + lane) * V, x);
+                load_vec<T>(t1, a1, m1, (c * 32 + lane) * V, y);
+#pragma unroll
+                for (int q = 0; q < V; ++q) { nn = fmaf(x[q], x[q], nn); dd = fmaf(x[q], y[q], dd); }
+            }
+        } else {
+#pragma unroll 2
+            for (int e = lane * V; e < D; e += 32 * V) {
+                float x[V], y[V];
+                load_vec<T>(t0, a0, m0, e, x);
+                load_vec<T>(t1, a1, m1, e, y);
+#pragma unroll
+                for (int q = 0; q < V; ++q) { nn = fmaf(x[q], x[q], nn); dd = fmaf(x[q], y[q], dd); }
+            }
+        }
+    } else {
+        if constexpr (NCHUNK > 0) {
+#pragma unroll
+            for (int c = 0; c < NCHUNK; ++c) {
+                float x[V];
+                load_vec<T>(t0, a0, m0, (c * 32 + lane) * V, x);
+#pragma unroll
+                for (int q = 0; q < V; ++q) nn = fmaf(x[q], x[q], nn);
+            }
+        } else {
+#pragma unroll 2
+            for (int e = lane * V; e < D; e += 32 * V) {
+                float x[V];
+                load_vec<T>(t0, a0, m0, e, x);
+#pragma unroll
+                for (int q = 0; q < V; ++q) nn = fmaf(x[q], x[q], nn);
+            }
+        }
+    }
+}
+
+template <typename T, int NCHUNK>
+__global__ void __launch_bounds__(kStepThreads, 3) oim_step_kernel(const StepArgs a) {
     constexpr int V = Elem<T>::kVec;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int len = a.axis == 0 ? a.w : a.h;
@@ -122,24 +170,7 @@ __global__ void __launch_bounds__(kStepThreads) oim_step_kernel(const StepArgs a
         const bool m1 = r1 & kMergedBit;
         const size_t o1 = (size_t)(r1 & ~kMergedBit) * D;
         float nn = 0.f, dd = 0.f;
-        if (has_next) {
-#pragma unroll 2
-            for (int e = lane * V; e < D; e += 32 * V) {
-                float x[V], y[V];
-                load_vec<T>(tokens + o0, acc + o0, m0, e, x);
-                load_vec<T>(tokens + o1, acc + o1, m1, e, y);
-#pragma unroll
-                for (int q = 0; q < V; ++q) { nn = fmaf(x[q], x[q], nn); dd = fmaf(x[q], y[q], dd); }
-            }
-        } else {
-#pragma unroll 2
-            for (int e = lane * V; e < D; e += 32 * V) {
-                float x[V];
-                load_vec<T>(tokens + o0, acc + o0, m0, e, x);
-#pragma unroll
-                for (int q = 0; q < V; ++q) nn = fmaf(x[q], x[q], nn);
-            }
-        }
+        pair_stats<T, NCHUNK>(tokens + o0, acc + o0, m0, tokens + o1, acc + o1, m1, has_next, lane, D, nn, dd);
         nn = warp_sum(nn);
         dd = warp_sum(dd);
         if (lane == 0) { s_nrm[j] = nn; s_dot[j] = dd; }
@@ -393,8 +424,10 @@ static int oim_run_typed(const OimProblem& p) {
         delete[] steps;
         return LUVC_ERR_TARGET;
     }
+    phase_begin(LUVC_PHASE_OIM_TOTAL, p.stream);
     oim_init_kernel<<<(unsigned)((n + 255) / 256), 256, 0, p.stream>>>(ws.cell_a, ws.size, ws.parent, HW, n);
     count_launch();
+    phase_begin(LUVC_PHASE_OIM_STEPS, p.stream);
     int32_t *cin = ws.cell_a, *cout = ws.cell_b;
     long long trace_off = 0;
     for (int s = 0; s < n_steps; ++s) {
@@ -407,18 +440,28 @@ static int oim_run_typed(const OimProblem& p) {
         a.trace_stride = (long long)HW - target;
         a.h = st.h; a.w = st.w; a.axis = st.axis; a.m = st.m; a.D = p.D; a.HW = HW;
         const size_t smem = (size_t)(3 * len + 2 * ((len + 1) / 2) + st.m + 8) * 4;
-        oim_step_kernel<T><<<dim3(lines, p.B), kStepThreads, smem, p.stream>>>(a);
+        const int chunk = 32 * Elem<T>::kVec;
+        const int nchunk = p.D % chunk == 0 ? p.D / chunk : 0;
+        const dim3 grid(lines, p.B);
+        switch (nchunk) {
+            case 4: oim_step_kernel<T, 4><<<grid, kStepThreads, smem, p.stream>>>(a); break;
+            case 5: oim_step_kernel<T, 5><<<grid, kStepThreads, smem, p.stream>>>(a); break;
+            case 8: oim_step_kernel<T, 8><<<grid, kStepThreads, smem, p.stream>>>(a); break;
+            default: oim_step_kernel<T, 0><<<grid, kStepThreads, smem, p.stream>>>(a); break;
+        }
         count_launch();
         trace_off += (long long)lines * st.m;
         int32_t* t = cin; cin = cout; cout = t;
     }
     delete[] steps;
+    phase_end(LUVC_PHASE_OIM_STEPS, p.stream);
     const long long cells = (long long)p.B * target;
     oim_emit_kernel<T><<<(unsigned)((cells * 32 + 255) / 256), 256, 0, p.stream>>>(
         p.tokens, ws.acc, cin, ws.size, ws.cellpos, p.out_tokens, p.out_sizes, HW, target, p.D, cells);
     count_launch();
     oim_map_kernel<<<(unsigned)((n + 255) / 256), 256, 0, p.stream>>>(ws.parent, ws.cellpos, p.out_map, HW, n);
     count_launch();
+    phase_end(LUVC_PHASE_OIM_TOTAL, p.stream);
     return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
 

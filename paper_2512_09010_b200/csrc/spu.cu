@@ -283,6 +283,7 @@ static int spu_run_typed(const SpuProblem& p) {
     Workspace ws = carve(p.workspace, B, N, D, sigma);
     float* E = p.out_scores ? p.out_scores : ws.E;
     const int tab = N > R ? N : R;
+    phase_begin(LUVC_PHASE_SPU_TRANSFORM, p.stream);
     spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, ws.scale, N, sigma, p.no_window);
     spu_contract_kernel<T, true><<<dim3(tiles, (R + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
         p.hidden, ws.Y, ws.tw, ws.scale, N, D, sigma);
@@ -290,10 +291,15 @@ static int spu_run_typed(const SpuProblem& p) {
         ws.Y, ws.part, ws.tw, ws.scale, N, D, sigma);
     const long long bn = (long long)B * N;
     spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn);
+    phase_end(LUVC_PHASE_SPU_TRANSFORM, p.stream);
+    phase_begin(LUVC_PHASE_SPU_SELECT, p.stream);
     spu_select_kernel<<<B, kSelThreads, 0, p.stream>>>(E, p.out_idx, N, p.keep);
+    phase_end(LUVC_PHASE_SPU_SELECT, p.stream);
+    phase_begin(LUVC_PHASE_SPU_GATHER, p.stream);
     const int row_vec = (int)((size_t)D * sizeof(T) / 16);
     spu_gather_kernel<<<dim3(p.keep, B), 128, 0, p.stream>>>(reinterpret_cast<const uint4*>(p.hidden), p.out_idx,
                                                             reinterpret_cast<uint4*>(p.out_hidden), N, p.keep, row_vec);
+    phase_end(LUVC_PHASE_SPU_GATHER, p.stream);
     count_launch(6);
     return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
