@@ -73,6 +73,13 @@ const char* luvc_status_string(int status);
  * points of the calling host thread.  NULL selects the legacy default stream. */
 int luvc_set_stream(void* cuda_stream);
 
+/* Device-side conditions (a bounded wait inside a kernel that gave up) are written
+ * to a status word in device memory instead of trapping.  This call synchronises
+ * the given stream, returns that word as a luvc_status (LUVC_OK if nothing was
+ * reported) and clears it.  While the word is set, later operator calls stop early;
+ * their outputs are then undefined. */
+int luvc_check_status(void* cuda_stream);
+
 /* Frees the library-owned scratch buffers of the current device.  Synchronises
  * the device first.  Safe to call more than once. */
 int luvc_shutdown(void);

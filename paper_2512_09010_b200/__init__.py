@@ -26,7 +26,7 @@ STATUS_NAMES = {
 # every symbol include/luvc.h declares
 EXPORTS = (
     "luvc_version", "luvc_status_string", "luvc_set_stream", "luvc_shutdown", "luvc_kernel_launches",
-    "luvc_profile_enable", "luvc_profile_read",
+    "luvc_profile_enable", "luvc_profile_read", "luvc_check_status",
     "luvc_oim_plan", "luvc_oim_workspace_bytes", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
     "luvc_oim_merge_host", "luvc_spu_sigma", "luvc_spu_workspace_bytes", "luvc_spu_prune",
     "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host",
@@ -70,6 +70,7 @@ def _load() -> ctypes.CDLL:
     L.luvc_status_string.argtypes = [i]
     L.luvc_set_stream.argtypes = [p]
     L.luvc_kernel_launches.restype = ctypes.c_longlong
+    L.luvc_check_status.argtypes = [p]
     L.luvc_profile_enable.argtypes = [i]
     L.luvc_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), i]
     L.luvc_oim_plan.argtypes = [i, i, i, i, ctypes.POINTER(i), ctypes.POINTER(i), ctypes.POINTER(i)]
@@ -119,6 +120,11 @@ def kernel_launches() -> int:
 
 def shutdown() -> None:
     _check(lib.luvc_shutdown(), "luvc_shutdown")
+
+
+def check_status(device=None) -> int:
+    """Synchronises the current torch stream and returns (and clears) the device status word."""
+    return int(lib.luvc_check_status(_stream_ptr(device)))
 
 
 PHASES = ("oim_steps", "oim_total", "spu_transform", "spu_select", "spu_gather")

@@ -42,7 +42,7 @@ thread_local cudaStream_t t_stream = nullptr;
 // Library-owned scratch: one growing buffer per purpose, shared by all threads.
 // Calls that use it from several host threads at once must use different streams'
 // work serially; the plain entry points take this lock only while (re)allocating.
-enum Slot { kOimWs = 0, kSpuWs, kIoIn, kIoOut, kSlots };
+enum Slot { kOimWs = 0, kSpuWs, kIoIn, kIoOut, kStatus, kSlots };
 struct Scratch { void* ptr = nullptr; size_t bytes = 0; };
 Scratch g_scratch[kSlots];
 std::mutex g_mutex;
@@ -56,6 +56,17 @@ void* scratch(Slot s, size_t bytes) {
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
     sc.ptr = p; sc.bytes = bytes;
     return p;
+}
+
+// The device status word: 256 bytes allocated once and zeroed, never freed before luvc_shutdown.
+int* status_word() {
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (g_scratch[kStatus].ptr) return static_cast<int*>(g_scratch[kStatus].ptr);
+    }
+    void* p = scratch(kStatus, 256);
+    if (p && cudaMemset(p, 0, 256) != cudaSuccess) return nullptr;
+    return static_cast<int*>(p);
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -141,6 +152,16 @@ int luvc_shutdown(void) {
     return LUVC_OK;
 }
 
+int luvc_check_status(void* cuda_stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return LUVC_ERR_CUDA;
+    int* word = status_word();
+    if (!word) return LUVC_ERR_CUDA;
+    int host = 0;
+    if (cudaMemcpy(&host, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return LUVC_ERR_CUDA;
+    if (host != 0 && cudaMemset(word, 0, sizeof(int)) != cudaSuccess) return LUVC_ERR_CUDA;
+    return host;
+}
+
 long long luvc_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int luvc_profile_enable(int on) {
@@ -199,6 +220,8 @@ int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target
     p.dtype = opts->dtype;
     p.out_tokens = out_tokens; p.out_sizes = out_sizes; p.out_map = out_map; p.trace = opts->trace;
     p.workspace = ws; p.stream = static_cast<cudaStream_t>(opts->stream);
+    p.status = status_word();
+    if (!p.status) return LUVC_ERR_CUDA;
     return oim_run(p);
 }
 

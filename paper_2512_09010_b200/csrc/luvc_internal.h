@@ -40,6 +40,7 @@ struct OimProblem {
     int32_t* out_map;
     int32_t* trace;
     void* workspace;
+    int* status;   // device status word shared by all calls (0 = ok, else a luvc_status)
     cudaStream_t stream;
 };
 size_t oim_workspace_bytes(int B, int H, int W, int D, int dtype);

@@ -6,15 +6,27 @@
 // input row; a cell that has absorbed others keeps the fp32 SUM of its sources
 // in row `root` of a scratch matrix acc[B][H*W][D] (cosines are scale-free, so
 // sums serve for the similarity; the mean is formed once, at the end).  The
-// grid itself is a small int32 matrix of roots that is compacted every step.
-// A step therefore reads every live vector once (that is the algorithm: all
-// neighbour similarities along the axis change when the orthogonal axis was
-// compacted) and writes only the merged rows.
+// grid itself is a small int32 matrix of (root | merged-bit) that is compacted
+// every step.  A step therefore reads every live vector once (that is the
+// algorithm: all neighbour similarities along the axis change when the
+// orthogonal axis was compacted) and writes only the merged rows.
 //
-// One CTA owns one line (row or column) of one image for one step: its warps
-// stream the line's vectors with 128-bit loads and fp32 accumulation, warp 0
-// ranks the even-position cells, then the warps apply the merges and close the
-// line up.  Lines are independent inside a step, so a step is one launch.
+// Execution.  The whole chain of steps of one call is ONE persistent kernel.
+// Its work items are the lines (rows or columns) of every image at every step,
+// numbered step-major, and handed out through an atomic counter.  A line of
+// image b at step s needs only image b's lines of step s-1, so each image has a
+// counter of finished lines per step and an item waits (bounded spin) on its
+// image's previous counter: images drift apart and one image's ranking and
+// merging overlaps another's streaming; there is no grid-wide barrier and no
+// launch between steps.  Items are claimed only by running CTAs and depend
+// only on lower-numbered items, so the lowest unfinished item can always run
+// and no co-residency guarantee is needed.
+//
+// One CTA owns one line: its warps stream the line's vectors with 128-bit
+// loads and fp32 accumulation (norm of each cell and dot with its successor),
+// warp 0 ranks the even-position cells, then the warps apply the merges and
+// close the line up.  Data written inside the kernel by other CTAs (grid,
+// sizes, fp32 sums) is read with L1-bypassing loads.
 
 #include <cuda_bf16.h>
 #include <float.h>
@@ -24,8 +36,10 @@
 namespace luvc {
 namespace {
 
-constexpr int kStepThreads = 256;
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
 constexpr unsigned kMergedBit = 0x80000000u;
+constexpr int kSpinLimit = 1 << 20;        // about a microsecond per probe: gives up after roughly a second
 
 template <typename T> struct Elem;
 template <> struct Elem<__nv_bfloat16> { static constexpr int kVec = 8; };   // elements per 16 bytes
@@ -35,15 +49,16 @@ __device__ __forceinline__ float bf16lo(unsigned u) { return __uint_as_float(u <
 __device__ __forceinline__ float bf16hi(unsigned u) { return __uint_as_float(u & 0xffff0000u); }
 
 // Loads kVec consecutive elements starting at element e of a cell's vector as fp32:
-// from the fp32 sum row when the cell is merged, else from the caller's input row.
+// from the fp32 sum row when the cell is merged (written during this kernel: L2 only),
+// else from the caller's read-only input row.
 template <typename T>
-__device__ __forceinline__ void load_vec(const T* __restrict__ tok_row, const float* __restrict__ acc_row,
-                                         bool merged, int e, float (&v)[Elem<T>::kVec]) {
+__device__ __forceinline__ void load_vec(const T* __restrict__ tok_row, const float* acc_row, bool merged, int e,
+                                         float (&v)[Elem<T>::kVec]) {
     constexpr int V = Elem<T>::kVec;
     if (merged) {
 #pragma unroll
         for (int q = 0; q < V; q += 4) {
-            const float4 f = *reinterpret_cast<const float4*>(acc_row + e + q);
+            const float4 f = __ldcg(reinterpret_cast<const float4*>(acc_row + e + q));
             v[q] = f.x; v[q + 1] = f.y; v[q + 2] = f.z; v[q + 3] = f.w;
         }
     } else if constexpr (sizeof(T) == 4) {
@@ -62,32 +77,12 @@ __device__ __forceinline__ float warp_sum(float x) {
     return x;
 }
 
-__global__ void oim_init_kernel(int32_t* cell, int32_t* size, int32_t* parent, int HW, long long total) {
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    cell[i] = (int32_t)(i % HW);
-    size[i] = 1;
-    parent[i] = -1;
-}
-
-struct StepArgs {
-    const void* tokens;   // [B][HW][D] caller input
-    float* acc;           // [B][HW][D] fp32 sums of merged cells
-    const int32_t* cell_in;
-    int32_t* cell_out;
-    int32_t* size;        // [B][HW] by root
-    int32_t* parent;      // [B][HW] by root: the root this one was merged into, or -1
-    int32_t* trace;       // this step's slice of image 0, or null
-    long long trace_stride;  // ints per image in the trace
-    int h, w, axis, m, D, HW;
-};
-
 // |x|^2 and <x, y> over one lane's share of two vectors.  NCHUNK > 0: D == NCHUNK * 32 * kVec and
 // the loop is fully unrolled so that all of a lane's loads are in flight together.
 template <typename T, int NCHUNK>
-__device__ __forceinline__ void pair_stats(const T* __restrict__ t0, const float* __restrict__ a0, bool m0,
-                                           const T* __restrict__ t1, const float* __restrict__ a1, bool m1,
-                                           bool has_next, int lane, int D, float& nn, float& dd) {
+__device__ __forceinline__ void pair_stats(const T* __restrict__ t0, const float* a0, bool m0,
+                                           const T* __restrict__ t1, const float* a1, bool m1, bool has_next,
+                                           int lane, int D, float& nn, float& dd) {
     constexpr int V = Elem<T>::kVec;
     if (has_next) {
         if constexpr (NCHUNK > 0) {
@@ -130,158 +125,266 @@ __device__ __forceinline__ void pair_stats(const T* __restrict__ t0, const float
     }
 }
 
+// One entry per merge step, built on the device by the set-up kernel.
+struct StepDesc {
+    int axis;        // 0: lines are rows, the width shrinks; 1: lines are columns, the height shrinks
+    int m;           // cells removed per line
+    int h, w;        // grid before the step
+    int item_begin;  // first work item of the step (items are step-major, then image, then line)
+    int trace_off;   // offset of the step's decisions inside one image's trace
+};
+
+struct ChainArgs {
+    const void* tokens;   // [B][HW][D] caller input
+    float* acc;           // [B][HW][D] fp32 sums of merged cells
+    int32_t* cell[2];     // [B][HW] grid of (root | merged bit), ping-pong by step parity
+    int32_t* size;        // [B][HW] by root
+    int32_t* parent;      // [B][HW] by root: the root this one was merged into, or -1
+    int32_t* trace;       // [B][HW - target] or null
+    const StepDesc* steps;
+    int* done;            // [n_steps][B] finished lines
+    int* next_item;       // work counter
+    int* status;          // device status word (0 = ok)
+    int B, HW, D, n_steps, total_items, trace_stride;
+};
+
+// Set-up: identity grid, unit sizes, no parents, zeroed counters, and the step table
+// (the same rule the host uses to validate the request).
+__global__ void oim_setup_kernel(int32_t* cell, int32_t* size, int32_t* parent, int HW, long long total,
+                                 StepDesc* steps, int* done, int* next_item, int B, int H, int W, int Hf, int Wf,
+                                 int r, int height_first, int n_steps) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < total) {
+        cell[i] = (int32_t)(i % HW);
+        size[i] = 1;
+        parent[i] = -1;
+    }
+    if (i < (long long)n_steps * B) done[i] = 0;
+    if (i == 0) {
+        *next_item = 0;
+        int h = H, w = W, n = 0, item = 0, toff = 0;
+        while ((h != Hf || w != Wf) && n < n_steps) {
+            for (int turn = 0; turn < 2 && n < n_steps; ++turn) {
+                const int axis = height_first ? 1 - turn : turn;
+                const int len = axis == 0 ? w : h, goal = axis == 0 ? Wf : Hf;
+                int m = len - goal < r ? len - goal : r;
+                if (m > (len + 1) / 2) m = (len + 1) / 2;
+                if (len < 2 || m <= 0) continue;
+                const int lines = axis == 0 ? h : w;
+                steps[n] = StepDesc{axis, m, h, w, item, toff};
+                item += lines * B;
+                toff += lines * m;
+                ++n;
+                if (axis == 0) w -= m; else h -= m;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ int load_acquire(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Thread 0 of a CTA waits until *ctr reaches `target`.  Gives up after kSpinLimit probes (or as soon
+// as another CTA has reported a failure) and records LUVC_ERR_TIMEOUT in the status word.
+__device__ bool wait_for_count(const int* ctr, int target, int* status) {
+    for (int it = 0; it < kSpinLimit; ++it) {
+        if (load_acquire(ctr) >= target) return true;
+        if (load_acquire(status) != 0) return false;
+        __nanosleep(it < 64 ? 32 : 256);
+    }
+    atomicCAS(status, 0, (int)LUVC_ERR_TIMEOUT);
+    return false;
+}
+
 template <typename T, int NCHUNK>
-__global__ void __launch_bounds__(kStepThreads, 3) oim_step_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) oim_chain_kernel(const ChainArgs a) {
     constexpr int V = Elem<T>::kVec;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int len = a.axis == 0 ? a.w : a.h;
-    const int ncand = (len + 1) >> 1;
-    float* s_dot = reinterpret_cast<float*>(smem_raw);          // <v_j, v_{j+1}>
-    float* s_nrm = s_dot + len;                                  // |v_j|^2
-    float* s_score = s_nrm + len;                                // best cosine of even cell 2c
-    unsigned* s_root = reinterpret_cast<unsigned*>(s_score + ncand);   // root | merged bit
-    int* s_dir = reinterpret_cast<int*>(s_root + len);           // best direction of even cell 2c
-    int* s_sel = s_dir + ncand;                                  // chosen (pos * 2 + dir), m entries
+    __shared__ int s_item;
+    __shared__ int s_ok;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int D = a.D, B = a.B;
+    int step = 0;
+    StepDesc st = a.steps[0];
+    int step_end = a.n_steps > 1 ? a.steps[1].item_begin : a.total_items;
 
-    const int b = blockIdx.y, line = blockIdx.x;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = kStepThreads >> 5;
-    const int base = a.axis == 0 ? line * a.w : line;
-    const int stride = a.axis == 0 ? 1 : a.w;
-    const size_t img = (size_t)b * a.HW;
-    const int32_t* cell_in = a.cell_in + img;
-    int32_t* size = a.size + img;
-    const T* tokens = reinterpret_cast<const T*>(a.tokens) + img * a.D;
-    float* acc = a.acc + img * a.D;
-    const int D = a.D;
-
-    for (int j = tid; j < len; j += kStepThreads) {
-        const unsigned r = (unsigned)cell_in[base + j * stride];
-        s_root[j] = r | (size[r] > 1 ? kMergedBit : 0u);
-    }
-    __syncthreads();
-
-    // ---- similarity pass: one warp per cell, norm of v_j and dot with its successor
-    for (int j = warp; j < len; j += nwarps) {
-        const unsigned r0 = s_root[j];
-        const bool m0 = r0 & kMergedBit;
-        const size_t o0 = (size_t)(r0 & ~kMergedBit) * D;
-        const bool has_next = j + 1 < len;
-        const unsigned r1 = has_next ? s_root[j + 1] : r0;
-        const bool m1 = r1 & kMergedBit;
-        const size_t o1 = (size_t)(r1 & ~kMergedBit) * D;
-        float nn = 0.f, dd = 0.f;
-        pair_stats<T, NCHUNK>(tokens + o0, acc + o0, m0, tokens + o1, acc + o1, m1, has_next, lane, D, nn, dd);
-        nn = warp_sum(nn);
-        dd = warp_sum(dd);
-        if (lane == 0) { s_nrm[j] = nn; s_dot[j] = dd; }
-    }
-    __syncthreads();
-
-    // ---- ranking: warp 0 scores the even cells and takes the m best
-    if (warp == 0) {
-        for (int c = lane; c < ncand; c += 32) {
-            const int j = 2 * c;
-            const float nj = sqrtf(s_nrm[j]);
-            float cl = -FLT_MAX, cr = -FLT_MAX;
-            if (j >= 1) {
-                const float nb = sqrtf(s_nrm[j - 1]);
-                cl = (nj == 0.f || nb == 0.f) ? 0.f : s_dot[j - 1] / (nj * nb);
-                if (!(cl == cl)) cl = -FLT_MAX;
-            }
-            if (j + 1 < len) {
-                const float nb = sqrtf(s_nrm[j + 1]);
-                cr = (nj == 0.f || nb == 0.f) ? 0.f : s_dot[j] / (nj * nb);
-                if (!(cr == cr)) cr = -FLT_MAX;
-            }
-            const bool right = (j < 1) || (j + 1 < len && cr > cl);   // ties stay with the previous cell
-            s_dir[c] = right ? 1 : 0;
-            s_score[c] = right ? cr : cl;
+    for (;;) {
+        __syncthreads();                       // the previous item's shared memory is no longer read
+        if (tid == 0) s_item = atomicAdd(a.next_item, 1);
+        __syncthreads();
+        const int item = s_item;
+        if (item >= a.total_items) break;
+        while (item >= step_end) {             // items only grow: walk the step table forward
+            ++step;
+            st = a.steps[step];
+            step_end = step + 1 < a.n_steps ? a.steps[step + 1].item_begin : a.total_items;
         }
-        __syncwarp();
-        for (int k = 0; k < a.m; ++k) {
-            float best = -INFINITY;
-            int best_c = 0x7fffffff;
+        const int len = st.axis == 0 ? st.w : st.h;
+        const int lines = st.axis == 0 ? st.h : st.w;
+        const int local = item - st.item_begin;
+        const int b = local / lines, line = local - b * lines;
+
+        if (step > 0) {                        // every line of this image's previous step must be finished
+            if (tid == 0) {
+                const StepDesc prev = a.steps[step - 1];
+                const int need = prev.axis == 0 ? prev.h : prev.w;
+                s_ok = wait_for_count(a.done + (size_t)(step - 1) * B + b, need, a.status) ? 1 : 0;
+            }
+            __syncthreads();
+            if (!s_ok) break;
+        }
+
+        const int ncand = (len + 1) >> 1;
+        float* s_dot = reinterpret_cast<float*>(smem_raw);          // <v_j, v_{j+1}>
+        float* s_nrm = s_dot + len;                                  // |v_j|^2
+        float* s_score = s_nrm + len;                                // best cosine of even cell 2c
+        unsigned* s_root = reinterpret_cast<unsigned*>(s_score + ncand);   // root | merged bit
+        int* s_dir = reinterpret_cast<int*>(s_root + len);           // best direction of even cell 2c
+        int* s_sel = s_dir + ncand;                                  // chosen (pos * 2 + dir), m entries
+
+        const int base = st.axis == 0 ? line * st.w : line;
+        const int stride = st.axis == 0 ? 1 : st.w;
+        const size_t img = (size_t)b * a.HW;
+        const int32_t* cell_in = a.cell[step & 1] + img;
+        int32_t* cell_out = a.cell[(step + 1) & 1] + img;
+        int32_t* size = a.size + img;
+        const T* tokens = reinterpret_cast<const T*>(a.tokens) + img * D;
+        float* acc = a.acc + img * D;
+
+        for (int j = tid; j < len; j += kThreads) s_root[j] = (unsigned)__ldcg(cell_in + base + j * stride);
+        __syncthreads();
+
+        // ---- similarity pass: one warp per cell, norm of v_j and dot with its successor
+        for (int j = warp; j < len; j += kWarps) {
+            const unsigned r0 = s_root[j];
+            const bool has_next = j + 1 < len;
+            const unsigned r1 = has_next ? s_root[j + 1] : r0;
+            const size_t o0 = (size_t)(r0 & ~kMergedBit) * D, o1 = (size_t)(r1 & ~kMergedBit) * D;
+            float nn = 0.f, dd = 0.f;
+            pair_stats<T, NCHUNK>(tokens + o0, acc + o0, r0 & kMergedBit, tokens + o1, acc + o1, r1 & kMergedBit,
+                                  has_next, lane, D, nn, dd);
+            nn = warp_sum(nn);
+            dd = warp_sum(dd);
+            if (lane == 0) { s_nrm[j] = nn; s_dot[j] = dd; }
+        }
+        __syncthreads();
+
+        // ---- ranking: warp 0 scores the even cells and takes the m best
+        if (warp == 0) {
             for (int c = lane; c < ncand; c += 32) {
-                const float s = s_score[c];
-                if (s > best) { best = s; best_c = c; }   // ascending c: the first maximum stays
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-                const int oc = __shfl_xor_sync(0xffffffffu, best_c, o);
-                if (ob > best || (ob == best && oc < best_c)) { best = ob; best_c = oc; }
-            }
-            if (lane == 0) {
-                s_sel[k] = (2 * best_c) * 2 + s_dir[best_c];
-                s_score[best_c] = -INFINITY;             // taken
+                const int j = 2 * c;
+                const float nj = sqrtf(s_nrm[j]);
+                float cl = -FLT_MAX, cr = -FLT_MAX;
+                if (j >= 1) {
+                    const float nb = sqrtf(s_nrm[j - 1]);
+                    cl = (nj == 0.f || nb == 0.f) ? 0.f : s_dot[j - 1] / (nj * nb);
+                    if (!(cl == cl)) cl = -FLT_MAX;
+                }
+                if (j + 1 < len) {
+                    const float nb = sqrtf(s_nrm[j + 1]);
+                    cr = (nj == 0.f || nb == 0.f) ? 0.f : s_dot[j] / (nj * nb);
+                    if (!(cr == cr)) cr = -FLT_MAX;
+                }
+                const bool right = (j < 1) || (j + 1 < len && cr > cl);   // ties stay with the previous cell
+                s_dir[c] = right ? 1 : 0;
+                s_score[c] = right ? cr : cl;
             }
             __syncwarp();
-        }
-        if (a.trace != nullptr)
-            for (int k = lane; k < a.m; k += 32)
-                a.trace[(size_t)b * a.trace_stride + (size_t)line * a.m + k] = s_sel[k];
-    }
-    __syncthreads();
-
-    // ---- close the line up: surviving cells keep their order
-    {
-        int32_t* cell_out = a.cell_out + img;
-        const int out_w = a.axis == 0 ? a.w - a.m : a.w;
-        for (int j = tid; j < len; j += kStepThreads) {
-            int before = 0;
-            bool removed = false;
-            for (int k = 0; k < a.m; ++k) {
-                const int p = s_sel[k] >> 1;   // position of the merged cell
-                removed |= p == j;
-                before += p < j;
-            }
-            if (!removed) {
-                const int nj = j - before;
-                const int dst = a.axis == 0 ? line * out_w + nj : nj * out_w + line;
-                cell_out[dst] = (int32_t)(s_root[j] & ~kMergedBit);
-            }
-        }
-    }
-
-    // ---- merges: one warp per destination cell; its new sum is written as fp32
-    for (int k = warp; k < a.m; k += nwarps) {
-        const int pos = s_sel[k] >> 1, dst = pos + ((s_sel[k] & 1) ? 1 : -1);
-        bool first = true;          // the lowest rank that targets this destination does the work
-        int other = -1;             // a second source of the same destination, if any
-        for (int q = 0; q < a.m; ++q) {
-            if (q == k) continue;
-            const int qpos = s_sel[q] >> 1, qdst = qpos + ((s_sel[q] & 1) ? 1 : -1);
-            if (qdst == dst) { if (q < k) first = false; else other = qpos; }
-        }
-        if (!first) continue;
-        const unsigned rd = s_root[dst], ra = s_root[pos], rb = other >= 0 ? s_root[other] : 0u;
-        const size_t od = (size_t)(rd & ~kMergedBit) * D, oa = (size_t)(ra & ~kMergedBit) * D,
-                     ob = (size_t)(rb & ~kMergedBit) * D;
-        for (int e = lane * V; e < D; e += 32 * V) {
-            float x[V], y[V];
-            load_vec<T>(tokens + od, acc + od, rd & kMergedBit, e, x);
-            load_vec<T>(tokens + oa, acc + oa, ra & kMergedBit, e, y);
+            for (int k = 0; k < st.m; ++k) {
+                float best = -INFINITY;
+                int best_c = 0x7fffffff;
+                for (int c = lane; c < ncand; c += 32) {
+                    const float s = s_score[c];
+                    if (s > best) { best = s; best_c = c; }   // ascending c: the first maximum stays
+                }
 #pragma unroll
-            for (int q = 0; q < V; ++q) x[q] += y[q];
-            if (other >= 0) {
-                load_vec<T>(tokens + ob, acc + ob, rb & kMergedBit, e, y);
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+                    const int oc = __shfl_xor_sync(0xffffffffu, best_c, o);
+                    if (ob > best || (ob == best && oc < best_c)) { best = ob; best_c = oc; }
+                }
+                if (lane == 0) {
+                    s_sel[k] = (2 * best_c) * 2 + s_dir[best_c];
+                    s_score[best_c] = -INFINITY;             // taken
+                }
+                __syncwarp();
+            }
+            if (a.trace != nullptr)
+                for (int k = lane; k < st.m; k += 32)
+                    a.trace[(size_t)b * a.trace_stride + st.trace_off + (size_t)line * st.m + k] = s_sel[k];
+        }
+        __syncthreads();
+
+        // ---- close the line up: surviving cells keep their order; receivers get the merged bit
+        {
+            const int out_w = st.axis == 0 ? st.w - st.m : st.w;
+            for (int j = tid; j < len; j += kThreads) {
+                int before = 0;
+                bool removed = false, receives = false;
+                for (int k = 0; k < st.m; ++k) {
+                    const int p = s_sel[k] >> 1;   // position of the merged cell
+                    removed |= p == j;
+                    before += p < j;
+                    receives |= p + ((s_sel[k] & 1) ? 1 : -1) == j;
+                }
+                if (!removed) {
+                    const int nj = j - before;
+                    const int dst = st.axis == 0 ? line * out_w + nj : nj * out_w + line;
+                    cell_out[dst] = (int32_t)(s_root[j] | (receives ? kMergedBit : 0u));
+                }
+            }
+        }
+
+        // ---- merges: one warp per destination cell; its new sum is written as fp32
+        for (int k = warp; k < st.m; k += kWarps) {
+            const int pos = s_sel[k] >> 1, dst = pos + ((s_sel[k] & 1) ? 1 : -1);
+            bool first = true;          // the lowest rank that targets this destination does the work
+            int other = -1;             // a second source of the same destination, if any
+            for (int q = 0; q < st.m; ++q) {
+                if (q == k) continue;
+                const int qpos = s_sel[q] >> 1, qdst = qpos + ((s_sel[q] & 1) ? 1 : -1);
+                if (qdst == dst) { if (q < k) first = false; else other = qpos; }
+            }
+            if (!first) continue;
+            const unsigned rd = s_root[dst], ra = s_root[pos], rb = other >= 0 ? s_root[other] : 0u;
+            const size_t od = (size_t)(rd & ~kMergedBit) * D, oa = (size_t)(ra & ~kMergedBit) * D,
+                         ob = (size_t)(rb & ~kMergedBit) * D;
+            for (int e = lane * V; e < D; e += 32 * V) {
+                float x[V], y[V];
+                load_vec<T>(tokens + od, acc + od, rd & kMergedBit, e, x);
+                load_vec<T>(tokens + oa, acc + oa, ra & kMergedBit, e, y);
 #pragma unroll
                 for (int q = 0; q < V; ++q) x[q] += y[q];
-            }
+                if (other >= 0) {
+                    load_vec<T>(tokens + ob, acc + ob, rb & kMergedBit, e, y);
 #pragma unroll
-            for (int q = 0; q < V; q += 4)
-                *reinterpret_cast<float4*>(acc + od + e + q) = make_float4(x[q], x[q + 1], x[q + 2], x[q + 3]);
-        }
-        if (lane == 0) {
-            const int id = rd & ~kMergedBit, ia = ra & ~kMergedBit;
-            int s = size[id] + size[ia];
-            a.parent[img + ia] = id;
-            if (other >= 0) {
-                const int ib = rb & ~kMergedBit;
-                s += size[ib];
-                a.parent[img + ib] = id;
+                    for (int q = 0; q < V; ++q) x[q] += y[q];
+                }
+#pragma unroll
+                for (int q = 0; q < V; q += 4)
+                    *reinterpret_cast<float4*>(acc + od + e + q) = make_float4(x[q], x[q + 1], x[q + 2], x[q + 3]);
             }
-            size[id] = s;
+            if (lane == 0) {
+                const int id = rd & ~kMergedBit, ia = ra & ~kMergedBit;
+                int s = __ldcg(size + id) + __ldcg(size + ia);
+                a.parent[img + ia] = id;
+                if (other >= 0) {
+                    const int ib = rb & ~kMergedBit;
+                    s += __ldcg(size + ib);
+                    a.parent[img + ib] = id;
+                }
+                size[id] = s;
+            }
+        }
+
+        // ---- publish: every write of this line is ordered before the counter increment
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            atomicAdd(a.done + (size_t)step * B + b, 1);
         }
     }
 }
@@ -299,7 +402,7 @@ __global__ void __launch_bounds__(256) oim_emit_kernel(const void* tokens_v, con
     if (gw >= total_cells) return;
     const int b = (int)(gw / target), c = (int)(gw % target);
     const size_t img = (size_t)b * HW;
-    const int root = cell[img + c];
+    const int root = (int)((unsigned)cell[img + c] & ~kMergedBit);
     const int s = size[img + root];
     const T* tok = reinterpret_cast<const T*>(tokens_v) + (img + root) * D;
     const float* arow = acc + (img + root) * D;
@@ -348,18 +451,26 @@ __global__ void oim_map_kernel(const int32_t* parent, const int32_t* cellpos, in
 struct Workspace {
     float* acc;
     int32_t *cell_a, *cell_b, *size, *parent, *cellpos;
+    StepDesc* steps;
+    int* done;
+    int* counters;   // [0] next item, [1] status
 };
 
-Workspace carve(void* ws, int B, int HW, int D) {
+size_t max_steps(int H, int W) { return (size_t)H + W + 2; }
+
+Workspace carve(void* ws, int B, int H, int W, int D) {
     unsigned char* p = static_cast<unsigned char*>(ws);
     Workspace w;
-    const size_t n = (size_t)B * HW;
+    const size_t n = (size_t)B * H * W;
     w.acc = reinterpret_cast<float*>(p); p += align_up(n * D * sizeof(float));
     w.cell_a = reinterpret_cast<int32_t*>(p); p += align_up(n * 4);
     w.cell_b = reinterpret_cast<int32_t*>(p); p += align_up(n * 4);
     w.size = reinterpret_cast<int32_t*>(p); p += align_up(n * 4);
     w.parent = reinterpret_cast<int32_t*>(p); p += align_up(n * 4);
-    w.cellpos = reinterpret_cast<int32_t*>(p);
+    w.cellpos = reinterpret_cast<int32_t*>(p); p += align_up(n * 4);
+    w.steps = reinterpret_cast<StepDesc*>(p); p += align_up(max_steps(H, W) * sizeof(StepDesc));
+    w.done = reinterpret_cast<int*>(p); p += align_up(max_steps(H, W) * B * sizeof(int));
+    w.counters = reinterpret_cast<int*>(p);
     return w;
 }
 
@@ -409,55 +520,78 @@ bool oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first, OimStep
 
 size_t oim_workspace_bytes(int B, int H, int W, int D, int /*dtype*/) {
     const size_t n = (size_t)B * H * W;
-    return align_up(n * D * sizeof(float)) + 5 * align_up(n * 4);
+    return align_up(n * D * sizeof(float)) + 5 * align_up(n * 4) + align_up(max_steps(H, W) * sizeof(StepDesc)) +
+           align_up(max_steps(H, W) * B * sizeof(int)) + 256;
+}
+
+template <typename T, int NCHUNK>
+static cudaError_t launch_chain(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
+    static int blocks_per_sm = 0, sms = 0;      // per kernel instantiation
+    const size_t smem = (size_t)(3 * max_len + 2 * ((max_len + 1) / 2) + r + 8) * 4;
+    if (smem > 48 * 1024)
+        cudaFuncSetAttribute(oim_chain_kernel<T, NCHUNK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, oim_chain_kernel<T, NCHUNK>, kThreads, smem);
+    if (blocks_per_sm < 1) blocks_per_sm = 1;
+    int grid = blocks_per_sm * sms;
+    if (grid > a.total_items) grid = a.total_items;
+    oim_chain_kernel<T, NCHUNK><<<grid, kThreads, smem, stream>>>(a);
+    return cudaGetLastError();
 }
 
 template <typename T>
 static int oim_run_typed(const OimProblem& p) {
     const int HW = p.H * p.W, target = p.Hf * p.Wf;
     const long long n = (long long)p.B * HW;
-    Workspace ws = carve(p.workspace, p.B, HW, p.D);
-    int n_steps = 0;
-    const int cap = 2 * (p.H + p.W) + 4;
+    Workspace ws = carve(p.workspace, p.B, p.H, p.W, p.D);
+    const int cap = (int)max_steps(p.H, p.W);
     OimStep* steps = new OimStep[cap];
-    if (!oim_schedule(p.H, p.W, p.Hf, p.Wf, p.r, p.height_first, steps, cap, &n_steps)) {
+    int n_steps = 0;
+    if (!oim_schedule(p.H, p.W, p.Hf, p.Wf, p.r, p.height_first, steps, cap, &n_steps) || n_steps > cap) {
         delete[] steps;
         return LUVC_ERR_TARGET;
     }
+    long long total_items = 0;
+    for (int s = 0; s < n_steps; ++s) total_items += (long long)p.B * (steps[s].axis == 0 ? steps[s].h : steps[s].w);
+    delete[] steps;
+    if (total_items > 0x7fffffffll) return LUVC_ERR_SHAPE;
+
     phase_begin(LUVC_PHASE_OIM_TOTAL, p.stream);
-    oim_init_kernel<<<(unsigned)((n + 255) / 256), 256, 0, p.stream>>>(ws.cell_a, ws.size, ws.parent, HW, n);
+    long long setup_threads = n > (long long)n_steps * p.B ? n : (long long)n_steps * p.B;
+    oim_setup_kernel<<<(unsigned)((setup_threads + 255) / 256), 256, 0, p.stream>>>(
+        ws.cell_a, ws.size, ws.parent, HW, n, ws.steps, ws.done, ws.counters, p.B, p.H, p.W, p.Hf, p.Wf, p.r,
+        p.height_first, n_steps);
     count_launch();
     phase_begin(LUVC_PHASE_OIM_STEPS, p.stream);
-    int32_t *cin = ws.cell_a, *cout = ws.cell_b;
-    long long trace_off = 0;
-    for (int s = 0; s < n_steps; ++s) {
-        const OimStep& st = steps[s];
-        const int len = st.axis == 0 ? st.w : st.h, lines = st.axis == 0 ? st.h : st.w;
-        StepArgs a;
-        a.tokens = p.tokens; a.acc = ws.acc; a.cell_in = cin; a.cell_out = cout;
-        a.size = ws.size; a.parent = ws.parent;
-        a.trace = p.trace ? p.trace + trace_off : nullptr;
-        a.trace_stride = (long long)HW - target;
-        a.h = st.h; a.w = st.w; a.axis = st.axis; a.m = st.m; a.D = p.D; a.HW = HW;
-        const size_t smem = (size_t)(3 * len + 2 * ((len + 1) / 2) + st.m + 8) * 4;
+    if (n_steps > 0) {
+        ChainArgs a;
+        a.tokens = p.tokens; a.acc = ws.acc; a.cell[0] = ws.cell_a; a.cell[1] = ws.cell_b;
+        a.size = ws.size; a.parent = ws.parent; a.trace = p.trace; a.steps = ws.steps; a.done = ws.done;
+        a.next_item = ws.counters; a.status = p.status;
+        a.B = p.B; a.HW = HW; a.D = p.D; a.n_steps = n_steps; a.total_items = (int)total_items;
+        a.trace_stride = HW - target;
         const int chunk = 32 * Elem<T>::kVec;
         const int nchunk = p.D % chunk == 0 ? p.D / chunk : 0;
-        const dim3 grid(lines, p.B);
+        const int max_len = p.H > p.W ? p.H : p.W;
+        cudaError_t err;
         switch (nchunk) {
-            case 4: oim_step_kernel<T, 4><<<grid, kStepThreads, smem, p.stream>>>(a); break;
-            case 5: oim_step_kernel<T, 5><<<grid, kStepThreads, smem, p.stream>>>(a); break;
-            case 8: oim_step_kernel<T, 8><<<grid, kStepThreads, smem, p.stream>>>(a); break;
-            default: oim_step_kernel<T, 0><<<grid, kStepThreads, smem, p.stream>>>(a); break;
+            case 4: err = launch_chain<T, 4>(a, max_len, p.r, p.stream); break;
+            case 5: err = launch_chain<T, 5>(a, max_len, p.r, p.stream); break;
+            case 8: err = launch_chain<T, 8>(a, max_len, p.r, p.stream); break;
+            default: err = launch_chain<T, 0>(a, max_len, p.r, p.stream); break;
         }
         count_launch();
-        trace_off += (long long)lines * st.m;
-        int32_t* t = cin; cin = cout; cout = t;
+        if (err != cudaSuccess) return LUVC_ERR_CUDA;
     }
-    delete[] steps;
     phase_end(LUVC_PHASE_OIM_STEPS, p.stream);
+    const int32_t* final_cell = (n_steps & 1) ? ws.cell_b : ws.cell_a;
     const long long cells = (long long)p.B * target;
     oim_emit_kernel<T><<<(unsigned)((cells * 32 + 255) / 256), 256, 0, p.stream>>>(
-        p.tokens, ws.acc, cin, ws.size, ws.cellpos, p.out_tokens, p.out_sizes, HW, target, p.D, cells);
+        p.tokens, ws.acc, final_cell, ws.size, ws.cellpos, p.out_tokens, p.out_sizes, HW, target, p.D, cells);
     count_launch();
     oim_map_kernel<<<(unsigned)((n + 255) / 256), 256, 0, p.stream>>>(ws.parent, ws.cellpos, p.out_map, HW, n);
     count_launch();
