@@ -298,6 +298,8 @@ int luvc_spu_prune_ex(const void* hidden, int B, int N, int D, float cutoff, int
     p.no_window = opts->no_window ? 1 : 0;
     p.out_idx = out_idx; p.out_hidden = out_hidden; p.out_scores = opts->out_scores;
     p.workspace = ws; p.stream = static_cast<cudaStream_t>(opts->stream);
+    p.status = status_word();
+    if (!p.status) return LUVC_ERR_CUDA;
     return spu_run(p);
 }
 

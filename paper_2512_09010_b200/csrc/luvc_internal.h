@@ -55,9 +55,29 @@ struct SpuProblem {
     void* out_hidden;
     float* out_scores;
     void* workspace;
+    int* status;   // device status word (see OimProblem)
     cudaStream_t stream;
 };
 size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype);
 int spu_run(const SpuProblem& p);
+
+// Tensor-core contraction of the bf16 path (spu_tc.cu).
+struct SpuTcPlan {
+    int r_pad;          // band rows 2 sigma + 1, padded to a multiple of 64
+    int n_pad;          // tokens padded to a multiple of 128
+    int tiles2;         // 256-channel tiles of the second pass
+    size_t phi_elems;   // bf16 elements of each half of the band matrix
+    size_t yt_elems;    // bf16 elements of each half of the spectrum
+    size_t part_elems;  // floats of the per-tile energy partials
+};
+struct SpuTcBuffers {
+    void *phi_hi, *phi_lo, *yt_hi, *yt_lo;
+    float* part;
+};
+SpuTcPlan spu_tc_plan(int B, int N, int D, int sigma);
+// Fills part[b][2 * tiles2][N] with per-tile sums of squares of the filtered signal.
+// `scale` must hold r_pad entries (zero beyond 2 sigma + 1).
+int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float* scale, int B, int N, int D,
+               int sigma, int* status, cudaStream_t stream);
 
 }  // namespace luvc

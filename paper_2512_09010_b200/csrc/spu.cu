@@ -9,8 +9,10 @@
 //   X' = Phi Y                (Eq. 7; real because the mask is even in f)
 //   E[n] = || X'[n, :] ||_2   (Eq. 8)
 // followed by an order-preserving top-`keep` selection and a row gather
-// (Algorithm 2's last two lines).  Everything is fp32; reductions have a fixed
-// order, so results are reproducible run to run.
+// (Algorithm 2's last two lines).  fp32 tokens run both contractions on the CUDA
+// cores in this file; bf16 tokens run them on the tensor cores (spu_tc.cu) with the
+// band matrix and the spectrum held as bf16 pairs and fp32 accumulation.  Reductions
+// have a fixed order, so results are reproducible run to run.
 
 #include <cuda_bf16.h>
 
@@ -23,13 +25,15 @@ constexpr int BM = 64, BN = 64, BK = 16;     // tile of the generic contraction
 constexpr int kGemmThreads = 256;
 
 // cos / sin of 2 pi j / N for j = 0..N-1, and the per-row constants c[r].
-__global__ void spu_tables_kernel(float2* tw, float* scale, int N, int sigma, int no_window) {
+// scale has `scale_len` >= 2 sigma + 1 entries; the extra ones are zero.
+__global__ void spu_tables_kernel(float2* tw, float* scale, int N, int sigma, int scale_len, int no_window) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < N) {
         double s, c;
         sincospi(2.0 * (double)i / (double)N, &s, &c);
         tw[i] = make_float2((float)c, (float)s);
     }
+    if (i >= 2 * sigma + 1 && i < scale_len) scale[i] = 0.f;
     if (i < 2 * sigma + 1) {
         const int k = i <= sigma ? i : i - sigma;
         double m = 1.0;
@@ -251,46 +255,75 @@ __global__ void __launch_bounds__(128) spu_gather_kernel(const uint4* __restrict
 struct Workspace {
     float2* tw;
     float* scale;
+    float* E;
+    // fp32 path (CUDA cores)
     float* Y;
     float* part;
-    float* E;
+    // bf16 path (tensor cores)
+    SpuTcBuffers tc;
 };
 
-Workspace carve(void* ws, int B, int N, int D, int sigma) {
+// Both paths share the twiddle table, the row constants and the scores; the rest differs.
+Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path) {
     unsigned char* p = static_cast<unsigned char*>(ws);
     const int R = 2 * sigma + 1, tiles = (D + BN - 1) / BN;
-    Workspace w;
+    const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
+    Workspace w = {};
     w.tw = reinterpret_cast<float2*>(p); p += align_up((size_t)N * sizeof(float2));
-    w.scale = reinterpret_cast<float*>(p); p += align_up((size_t)R * 4);
-    w.Y = reinterpret_cast<float*>(p); p += align_up((size_t)B * R * D * 4);
-    w.part = reinterpret_cast<float*>(p); p += align_up((size_t)B * tiles * N * 4);
-    w.E = reinterpret_cast<float*>(p);
+    w.scale = reinterpret_cast<float*>(p); p += align_up((size_t)pl.r_pad * 4);
+    w.E = reinterpret_cast<float*>(p); p += align_up((size_t)B * N * 4);
+    if (!tensor_path) {
+        w.Y = reinterpret_cast<float*>(p); p += align_up((size_t)B * R * D * 4);
+        w.part = reinterpret_cast<float*>(p);
+    } else {
+        w.tc.phi_hi = p; p += align_up(pl.phi_elems * 2);
+        w.tc.phi_lo = p; p += align_up(pl.phi_elems * 2);
+        w.tc.yt_hi = p; p += align_up(pl.yt_elems * 2);
+        w.tc.yt_lo = p; p += align_up(pl.yt_elems * 2);
+        w.tc.part = reinterpret_cast<float*>(p);
+    }
     return w;
 }
 
 }  // namespace
 
-size_t spu_workspace_bytes(int B, int N, int D, int sigma, int /*dtype*/) {
+size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype) {
     const int R = 2 * sigma + 1, tiles = (D + BN - 1) / BN;
-    return align_up((size_t)N * sizeof(float2)) + align_up((size_t)R * 4) + align_up((size_t)B * R * D * 4) +
-           align_up((size_t)B * tiles * N * 4) + align_up((size_t)B * N * 4);
+    const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
+    size_t bytes = align_up((size_t)N * sizeof(float2)) + align_up((size_t)pl.r_pad * 4) + align_up((size_t)B * N * 4);
+    if (dtype == LUVC_F32)
+        bytes += align_up((size_t)B * R * D * 4) + align_up((size_t)B * tiles * N * 4);
+    else
+        bytes += 2 * align_up(pl.phi_elems * 2) + 2 * align_up(pl.yt_elems * 2) + align_up(pl.part_elems * 4);
+    return bytes;
 }
 
 template <typename T>
 static int spu_run_typed(const SpuProblem& p) {
+    constexpr bool kTensor = sizeof(T) == 2;     // bf16 tokens go through the tensor cores
     const int N = p.N, D = p.D, B = p.B, sigma = p.sigma, R = 2 * sigma + 1;
-    const int tiles = (D + BN - 1) / BN;
-    Workspace ws = carve(p.workspace, B, N, D, sigma);
+    const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
+    Workspace ws = carve(p.workspace, B, N, D, sigma, kTensor);
     float* E = p.out_scores ? p.out_scores : ws.E;
-    const int tab = N > R ? N : R;
-    phase_begin(LUVC_PHASE_SPU_TRANSFORM, p.stream);
-    spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, ws.scale, N, sigma, p.no_window);
-    spu_contract_kernel<T, true><<<dim3(tiles, (R + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
-        p.hidden, ws.Y, ws.tw, ws.scale, N, D, sigma);
-    spu_contract_kernel<T, false><<<dim3(tiles, (N + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
-        ws.Y, ws.part, ws.tw, ws.scale, N, D, sigma);
+    const int tab = N > pl.r_pad ? N : pl.r_pad;
     const long long bn = (long long)B * N;
-    spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn);
+    phase_begin(LUVC_PHASE_SPU_TRANSFORM, p.stream);
+    spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, ws.scale, N, sigma, pl.r_pad, p.no_window);
+    count_launch();
+    if constexpr (kTensor) {
+        const int rc = spu_tc_run(ws.tc, p.hidden, ws.tw, ws.scale, B, N, D, sigma, p.status, p.stream);
+        if (rc != LUVC_OK) return rc;
+        spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, E, N, 2 * pl.tiles2, bn);
+        count_launch();
+    } else {
+        const int tiles = (D + BN - 1) / BN;
+        spu_contract_kernel<T, true><<<dim3(tiles, (R + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
+            p.hidden, ws.Y, ws.tw, ws.scale, N, D, sigma);
+        spu_contract_kernel<T, false><<<dim3(tiles, (N + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
+            ws.Y, ws.part, ws.tw, ws.scale, N, D, sigma);
+        spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn);
+        count_launch(3);
+    }
     phase_end(LUVC_PHASE_SPU_TRANSFORM, p.stream);
     phase_begin(LUVC_PHASE_SPU_SELECT, p.stream);
     spu_select_kernel<<<B, kSelThreads, 0, p.stream>>>(E, p.out_idx, N, p.keep);
@@ -300,7 +333,7 @@ static int spu_run_typed(const SpuProblem& p) {
     spu_gather_kernel<<<dim3(p.keep, B), 128, 0, p.stream>>>(reinterpret_cast<const uint4*>(p.hidden), p.out_idx,
                                                             reinterpret_cast<uint4*>(p.out_hidden), N, p.keep, row_vec);
     phase_end(LUVC_PHASE_SPU_GATHER, p.stream);
-    count_launch(6);
+    count_launch(2);
     return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
 
