@@ -35,7 +35,7 @@ HBM_FALLBACK_GBS = 6650.0     # used only if MEASURED_PEAKS.json is absent
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (null until a capture for that workload exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {2: 1.152e9 + 0.159e9}     # profiles/oim_chain_kernel_configs2.txt
 
 
 def parse_args():
@@ -392,11 +392,11 @@ def main():
     spu_bytes = spu_in_bytes + sb * sn * 4 + 2 * sb * spec["keep"] * sd * e + sb * spec["keep"] * 4
     spu_ms = phases["spu_transform"] + phases["spu_select"] + phases["spu_gather"]
     roofline = {
-        "kernel": "oim_step_kernel (%d launches per step)" % n_steps,
+        "kernel": "oim_chain_kernel (one launch runs the %d merge steps of a call)" % n_steps,
         "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak if achieved else None, "peak_source": peak_src,
         "frac_of_8TBs": achieved / HBM_NOMINAL_GBS if achieved else None,
-        "algorithmic_bytes_per_launch": iter_bytes / n_steps, "avg_launch_ms": steps_ms / n_steps,
+        "algorithmic_bytes_per_launch": iter_bytes, "avg_launch_ms": steps_ms, "merge_steps_per_launch": n_steps,
         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(k),
         "floor_bytes": floor_bytes,
         "spu": {"algorithmic_bytes": spu_bytes, "ms": spu_ms,
