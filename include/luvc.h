@@ -213,6 +213,46 @@ int luvc_spu_prune_ex(const void* hidden, int B, int N, int D, float cutoff, int
 int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, int keep, int dtype,
                         int32_t* out_idx, void* out_hidden);
 
+/* ---- SPU without any allocation ------------------------------------------- */
+
+/* Largest workspace (luvc_spu_workspace_bytes) luvc_spu_prune_static accepts: 32 MiB. */
+#define LUVC_SPU_STATIC_MAX_BYTES (32u * 1024u * 1024u)
+
+/*
+ * luvc_spu_prune with a fixed, built-in workspace.  (The paper has no counterpart:
+ * this is a deployment variant of the same operator, not another method.)
+ *
+ * For callers that cannot allocate device memory when they prune: a server whose
+ * own allocator already owns the device's memory, a loop that cannot afford the
+ * device-wide synchronisation an allocation may cause, a process under a fixed
+ * memory budget.  This call never calls cudaMalloc, cudaFree or any routine that
+ * allocates, and needs no caller workspace.  Its workspace is an array of
+ * LUVC_SPU_STATIC_MAX_BYTES (+256) bytes that is part of the library's device
+ * image: every GPU that loads the library holds it from load until exit.
+ *
+ * Arguments and results are those of luvc_spu_prune_ex with default options
+ * (Hamming-windowed pass band, no score export): hidden [B,N,D], out_idx [B,keep],
+ * out_hidden [B,keep,D] are DEVICE pointers owned by the caller, dtype is a
+ * luvc_dtype, cuda_stream a cudaStream_t (NULL = legacy default stream); the work
+ * is queued on that stream and the host is not synchronised.
+ *
+ * Errors: those of luvc_spu_prune_ex, and LUVC_ERR_WORKSPACE when
+ * luvc_spu_workspace_bytes(B, N, D, cutoff, dtype) exceeds LUVC_SPU_STATIC_MAX_BYTES
+ * (nothing is queued; use the other entry points for such sizes).
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.  All calls on
+ * a device share the one array and it keeps the previous call's contents: the
+ * call clears the part that must start at zero, but two calls whose GPU work
+ * overlaps (different streams, or several host threads) race on it - run them on
+ * one stream or order them with events.  A bounded device-side wait that gives up
+ * is recorded inside the array, not in the word luvc_check_status reads; the
+ * outputs of such a call are undefined.  With luvc_profile_enable(1) the first
+ * call creates CUDA events; leave profiling off where that matters.
+ */
+int luvc_spu_prune_static(const void* hidden, int B, int N, int D, float cutoff, int keep, int dtype,
+                          void* cuda_stream, int32_t* out_idx, void* out_hidden);
+
 #ifdef __cplusplus
 }
 #endif

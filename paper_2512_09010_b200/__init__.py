@@ -29,7 +29,7 @@ EXPORTS = (
     "luvc_profile_enable", "luvc_profile_read", "luvc_check_status",
     "luvc_oim_plan", "luvc_oim_workspace_bytes", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
     "luvc_oim_merge_host", "luvc_spu_sigma", "luvc_spu_workspace_bytes", "luvc_spu_prune",
-    "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host",
+    "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host", "luvc_spu_prune_static",
 )
 
 
@@ -87,6 +87,7 @@ def _load() -> ctypes.CDLL:
     L.luvc_spu_prune_f32.argtypes = [p, i, i, i, f, i, p, p]
     L.luvc_spu_prune_ex.argtypes = [p, i, i, i, f, i, p, p, ctypes.POINTER(SpuOpts)]
     L.luvc_spu_prune_host.argtypes = [p, i, i, i, f, i, i, p, p]
+    L.luvc_spu_prune_static.argtypes = [p, i, i, i, f, i, i, p, p, p]
     return L
 
 
@@ -242,6 +243,28 @@ def spu_prune_plain(hidden: torch.Tensor, keep: int, cutoff: float = 0.0):
         fn = lib.luvc_spu_prune if _dtype_code(hidden) == BF16 else lib.luvc_spu_prune_f32
         _check(fn(hidden.data_ptr(), B, N, D, float(cutoff), int(keep), out_idx.data_ptr(), out_hidden.data_ptr()),
                "luvc_spu_prune")
+    return out_idx, out_hidden
+
+
+SPU_STATIC_MAX_BYTES = 32 * 1024 * 1024
+
+
+def spu_prune_static(hidden: torch.Tensor, keep: int, cutoff: float = 0.0):
+    """luvc_spu_prune_static: the prune for callers that cannot allocate device memory.  The library
+    call allocates nothing (its workspace is a fixed array inside the library, at most
+    SPU_STATIC_MAX_BYTES); this wrapper still creates the two output tensors, which a caller with
+    such a constraint would own beforehand.  Returns (out_idx [B,keep] int32, out_hidden [B,keep,D])."""
+    if not hidden.is_cuda:
+        raise ValueError("hidden must live on a CUDA device")
+    hidden = hidden.contiguous()
+    B, N, D = hidden.shape
+    dev = hidden.device
+    with torch.cuda.device(dev):
+        out_idx = torch.empty((B, max(int(keep), 0)), dtype=torch.int32, device=dev)
+        out_hidden = torch.empty((B, max(int(keep), 0), D), dtype=hidden.dtype, device=dev)
+        _check(lib.luvc_spu_prune_static(hidden.data_ptr(), B, N, D, float(cutoff), int(keep), _dtype_code(hidden),
+                                         _stream_ptr(dev), out_idx.data_ptr(), out_hidden.data_ptr()),
+               "luvc_spu_prune_static")
     return out_idx, out_hidden
 
 

@@ -1,0 +1,46 @@
+"""luvc_spu_prune_static, the prune for callers that cannot allocate device memory (a server whose
+allocator already owns the GPU's memory, a loop that cannot take an allocation's synchronisation):
+its workspace is a fixed array inside the library.  Checked through the C ABI against
+luvc_spu_prune_ex on the same inputs, twice in a row, because every call reuses that one array and
+finds the previous call's contents in it.  This file sorts last on purpose: a run that stops at the
+first failure has then already run every other test."""
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def luvc():
+    import paper_2512_09010_b200 as luvc
+    assert torch.cuda.is_available()
+    return luvc
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_two_calls_in_a_row_match_the_allocating_entry_point(luvc, dtype):
+    g = torch.Generator().manual_seed(2512)
+    # the second problem is smaller and differently shaped, so stale bytes of the first stay in the array
+    for B, N, D, keep, cutoff in ((3, 200, 264, 50, 0.25), (2, 96, 136, 31, 0.0)):
+        x = torch.randn((B, N, D), generator=g).to(dtype).cuda()
+        assert luvc.lib.luvc_spu_workspace_bytes(B, N, D, cutoff, luvc._dtype_code(x)) <= luvc.SPU_STATIC_MAX_BYTES
+        ref_idx, ref_hid = luvc.spu_prune(x, keep, cutoff)
+        idx, hid = luvc.spu_prune_static(x, keep, cutoff)
+        torch.cuda.synchronize()
+        # same kernels on the same inputs: indices are integers, kept rows are copies -> exact
+        assert torch.equal(idx, ref_idx)
+        assert torch.equal(hid, ref_hid)
+        assert torch.equal(hid, torch.stack([x[b][idx[b].long()] for b in range(B)]))
+    assert luvc.check_status() == 0
+
+
+def test_sizes_beyond_the_fixed_array_are_refused(luvc):
+    B, N, D = 8, 16384, 4096
+    x = torch.zeros((1, 8, 8), dtype=torch.bfloat16, device="cuda")     # never read: the size check comes first
+    assert luvc.lib.luvc_spu_workspace_bytes(B, N, D, 0.0, luvc.BF16) > luvc.SPU_STATIC_MAX_BYTES
+    out_idx = torch.full((B, 4), -7, dtype=torch.int32, device="cuda")
+    rc = luvc.lib.luvc_spu_prune_static(x.data_ptr(), B, N, D, 0.0, 4, luvc.BF16, None, out_idx.data_ptr(),
+                                        x.data_ptr())
+    assert rc == 8                                                       # LUVC_ERR_WORKSPACE, nothing queued
+    torch.cuda.synchronize()
+    assert bool((out_idx == -7).all())
