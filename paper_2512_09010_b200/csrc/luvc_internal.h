@@ -66,18 +66,23 @@ struct SpuTcPlan {
     int r_pad;          // band rows 2 sigma + 1, padded to a multiple of 64
     int n_pad;          // tokens padded to a multiple of 128
     int tiles2;         // 256-channel tiles of the second pass
+    int coarse;         // 1: the inverse is evaluated on L < N uniform points t_j = j N / L of the period
+    int L;              // points of the inverse (N when not coarse; a multiple of 128 >= 4 sigma + 2 otherwise)
+    int l_pad;          // L padded to a multiple of 128
     size_t phi_elems;   // bf16 elements of each half of the band matrix
+    size_t phi2_elems;  // bf16 elements of each half of the coarse band matrix (0 when not coarse)
     size_t yt_elems;    // bf16 elements of each half of the spectrum
     size_t part_elems;  // floats of the per-tile energy partials
 };
 struct SpuTcBuffers {
-    void *phi_hi, *phi_lo, *yt_hi, *yt_lo;
+    void *phi_hi, *phi_lo, *phi2_hi, *phi2_lo, *yt_hi, *yt_lo;
     float* part;
 };
 SpuTcPlan spu_tc_plan(int B, int N, int D, int sigma);
-// Fills part[b][2 * tiles2][N] with per-tile sums of squares of the filtered signal.
-// `scale` must hold r_pad entries (zero beyond 2 sigma + 1).
-int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float* scale, int B, int N, int D,
-               int sigma, int* status, cudaStream_t stream);
+// Fills part[b][2 * tiles2][L] with per-tile sums of squares of the filtered signal at the L points
+// of the plan.  `scale` must hold r_pad entries (zero beyond 2 sigma + 1); `tw2` is the table of
+// cos / sin of 2 pi j / L (used when the plan is coarse).
+int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float2* tw2, const float* scale,
+               int B, int N, int D, int sigma, int* status, cudaStream_t stream);
 
 }  // namespace luvc

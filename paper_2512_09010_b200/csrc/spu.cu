@@ -26,12 +26,19 @@ constexpr int kGemmThreads = 256;
 
 // cos / sin of 2 pi j / N for j = 0..N-1, and the per-row constants c[r].
 // scale has `scale_len` >= 2 sigma + 1 entries; the extra ones are zero.
-__global__ void spu_tables_kernel(float2* tw, float* scale, int N, int sigma, int scale_len, int no_window) {
+// tw2 (may be null) is the same table for a period of L points.
+__global__ void spu_tables_kernel(float2* tw, float2* tw2, float* scale, int N, int L, int sigma, int scale_len,
+                                  int no_window) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < N) {
         double s, c;
         sincospi(2.0 * (double)i / (double)N, &s, &c);
         tw[i] = make_float2((float)c, (float)s);
+    }
+    if (tw2 != nullptr && i < L) {
+        double s, c;
+        sincospi(2.0 * (double)i / (double)L, &s, &c);
+        tw2[i] = make_float2((float)c, (float)s);
     }
     if (i >= 2 * sigma + 1 && i < scale_len) scale[i] = 0.f;
     if (i < 2 * sigma + 1) {
@@ -145,14 +152,92 @@ __global__ void __launch_bounds__(kGemmThreads) spu_contract_kernel(const void* 
     }
 }
 
-// E[b][n] = sqrt(sum over the channel tiles, in tile order).
-__global__ void spu_energy_kernel(const float* part, float* E, int N, int tiles, long long total) {
+// E[b][n] = sqrt(sum over the channel tiles, in tile order); with `squared` the sum itself.
+__global__ void spu_energy_kernel(const float* part, float* E, int N, int tiles, long long total, int squared) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total) return;
     const int b = (int)(i / N), n = (int)(i % N);
     float s = 0.f;
     for (int t = 0; t < tiles; ++t) s += part[((size_t)b * tiles + t) * N + n];
-    E[i] = sqrtf(s);
+    E[i] = squared ? s : sqrtf(s);
+}
+
+// ---- squared energies from L uniform samples of the period to the N tokens --------------------
+//
+// S(t) = sum_d x'_d(t)^2 is a real trigonometric polynomial of degree F = 2 sigma, so its L > 2 F
+// samples S(j N / L) fix its coefficients g_f = (1/L) sum_j S_j e^{-2 pi i f j / L} exactly, and
+// S(n) = g_0 + 2 sum_{f=1..F} Re(g_f e^{2 pi i f n / N}) on the tokens.
+
+constexpr int kSpecChunk = 256;    // samples per partial sum of a coefficient
+constexpr int kReseed = 32;        // steps of the rotation recurrence between exact restarts
+
+__device__ __forceinline__ float2 unit_root(long long num, int den) {   // e^{2 pi i num / den}
+    const int m = (int)(num % den);
+    float s, c;
+    sincospif(2.0f * (float)m / (float)den, &s, &c);
+    return make_float2(c, s);
+}
+
+// gpart[b][chunk][f] = sum over the chunk's samples of S_j e^{-2 pi i f j / L}
+__global__ void __launch_bounds__(128) spu_coarse_spectrum_kernel(const float* __restrict__ S, float2* __restrict__ gpart,
+                                                                  int L, int F) {
+    __shared__ float s_val[kSpecChunk];
+    const int b = blockIdx.z, chunk = blockIdx.y, f = blockIdx.x * 128 + threadIdx.x;
+    const int j0 = chunk * kSpecChunk, cnt = min(kSpecChunk, L - j0);
+    for (int j = threadIdx.x; j < cnt; j += 128) s_val[j] = S[(size_t)b * L + j0 + j];
+    __syncthreads();
+    if (f > F) return;
+    const float2 step = unit_root(f, L);
+    float gr = 0.f, gi = 0.f;
+    float2 w = make_float2(1.f, 0.f);
+    for (int j = 0; j < cnt; ++j) {
+        if ((j % kReseed) == 0) w = unit_root((long long)f * (j0 + j), L);
+        const float v = s_val[j];
+        gr = fmaf(v, w.x, gr);
+        gi = fmaf(-v, w.y, gi);                       // conjugate: e^{-i theta}
+        const float nx = w.x * step.x - w.y * step.y;
+        w.y = fmaf(w.x, step.y, w.y * step.x);
+        w.x = nx;
+    }
+    gpart[((size_t)b * gridDim.y + chunk) * (F + 1) + f] = make_float2(gr, gi);
+}
+
+// E[b][n] = sqrt(max(0, S(n))), the coefficient partials summed in chunk order.
+constexpr int kSynthTile = 2048;   // coefficients staged in shared memory at a time
+__global__ void __launch_bounds__(256) spu_coarse_synthesis_kernel(const float2* __restrict__ gpart, float* __restrict__ E,
+                                                                   int N, int L, int F, int chunks) {
+    __shared__ float2 s_g[kSynthTile];
+    const int b = blockIdx.y, n = blockIdx.x * 256 + threadIdx.x;
+    const float inv_l = 1.0f / (float)L;
+    const float2 step = unit_root(n < N ? n : 0, N);
+    float acc = 0.f;
+    for (int f0 = 0; f0 <= F; f0 += kSynthTile) {
+        const int cnt = min(kSynthTile, F + 1 - f0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < cnt; i += 256) {
+            float gr = 0.f, gi = 0.f;
+            for (int c = 0; c < chunks; ++c) {
+                const float2 v = gpart[((size_t)b * chunks + c) * (F + 1) + f0 + i];
+                gr += v.x; gi += v.y;
+            }
+            const float m = (f0 + i == 0) ? inv_l : 2.0f * inv_l;
+            s_g[i] = make_float2(gr * m, gi * m);
+        }
+        __syncthreads();
+        if (n < N) {
+            float2 w = make_float2(1.f, 0.f);
+            for (int i = 0; i < cnt; ++i) {
+                if ((i % kReseed) == 0) w = unit_root((long long)(f0 + i) * n, N);
+                const float2 g = s_g[i];
+                acc = fmaf(g.x, w.x, acc);
+                acc = fmaf(-g.y, w.y, acc);
+                const float nx = w.x * step.x - w.y * step.y;
+                w.y = fmaf(w.x, step.y, w.y * step.x);
+                w.x = nx;
+            }
+        }
+    }
+    if (n < N) E[(size_t)b * N + n] = sqrtf(fmaxf(acc, 0.f));
 }
 
 // ---- order-preserving top-k ---------------------------------------------------
@@ -254,6 +339,9 @@ __global__ void __launch_bounds__(128) spu_gather_kernel(const uint4* __restrict
 
 struct Workspace {
     float2* tw;
+    float2* tw2;     // table for the coarse period (tensor path)
+    float* S;        // squared energies at the coarse points [B][L]
+    float2* gpart;   // their spectrum, partial sums [B][chunks][2 sigma * 2 + 1]
     float* scale;
     float* E;
     // fp32 path (CUDA cores)
@@ -262,6 +350,10 @@ struct Workspace {
     // bf16 path (tensor cores)
     SpuTcBuffers tc;
 };
+
+size_t coarse_gpart_elems(int B, int L, int sigma) {
+    return (size_t)B * ((L + kSpecChunk - 1) / kSpecChunk) * (4 * (size_t)sigma + 1);
+}
 
 // Both paths share the twiddle table, the row constants and the scores; the rest differs.
 Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path) {
@@ -278,6 +370,11 @@ Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path) {
     } else {
         w.tc.phi_hi = p; p += align_up(pl.phi_elems * 2);
         w.tc.phi_lo = p; p += align_up(pl.phi_elems * 2);
+        w.tc.phi2_hi = p; p += align_up(pl.phi2_elems * 2);
+        w.tc.phi2_lo = p; p += align_up(pl.phi2_elems * 2);
+        w.tw2 = reinterpret_cast<float2*>(p); p += align_up((size_t)pl.L * sizeof(float2));
+        w.S = reinterpret_cast<float*>(p); p += align_up((size_t)B * pl.L * 4);
+        w.gpart = reinterpret_cast<float2*>(p); p += align_up(coarse_gpart_elems(B, pl.L, sigma) * sizeof(float2));
         w.tc.yt_hi = p; p += align_up(pl.yt_elems * 2);
         w.tc.yt_lo = p; p += align_up(pl.yt_elems * 2);
         w.tc.part = reinterpret_cast<float*>(p);
@@ -294,7 +391,10 @@ size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype) {
     if (dtype == LUVC_F32)
         bytes += align_up((size_t)B * R * D * 4) + align_up((size_t)B * tiles * N * 4);
     else
-        bytes += 2 * align_up(pl.phi_elems * 2) + 2 * align_up(pl.yt_elems * 2) + align_up(pl.part_elems * 4);
+        bytes += 2 * align_up(pl.phi_elems * 2) + 2 * align_up(pl.phi2_elems * 2) +
+                 align_up((size_t)pl.L * sizeof(float2)) + align_up((size_t)B * pl.L * 4) +
+                 align_up(coarse_gpart_elems(B, pl.L, sigma) * sizeof(float2)) + 2 * align_up(pl.yt_elems * 2) +
+                 align_up(pl.part_elems * 4);
     return bytes;
 }
 
@@ -305,23 +405,34 @@ static int spu_run_typed(const SpuProblem& p) {
     const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
     Workspace ws = carve(p.workspace, B, N, D, sigma, kTensor);
     float* E = p.out_scores ? p.out_scores : ws.E;
-    const int tab = N > pl.r_pad ? N : pl.r_pad;
+    const int tab = max(max(N, pl.r_pad), pl.L);
     const long long bn = (long long)B * N;
     phase_begin(LUVC_PHASE_SPU_TRANSFORM, p.stream);
-    spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, ws.scale, N, sigma, pl.r_pad, p.no_window);
+    const bool coarse = kTensor && pl.coarse;
+    spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, coarse ? ws.tw2 : nullptr, ws.scale, N, pl.L, sigma,
+                                                               pl.r_pad, p.no_window);
     count_launch();
     if constexpr (kTensor) {
-        const int rc = spu_tc_run(ws.tc, p.hidden, ws.tw, ws.scale, B, N, D, sigma, p.status, p.stream);
+        const int rc = spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status, p.stream);
         if (rc != LUVC_OK) return rc;
-        spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, E, N, 2 * pl.tiles2, bn);
-        count_launch();
+        if (!coarse) {
+            spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, E, N, 2 * pl.tiles2, bn, 0);
+            count_launch();
+        } else {
+            const int L = pl.L, F = 2 * sigma, chunks = (L + kSpecChunk - 1) / kSpecChunk;
+            const long long bl = (long long)B * L;
+            spu_energy_kernel<<<(unsigned)((bl + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, ws.S, L, 2 * pl.tiles2, bl, 1);
+            spu_coarse_spectrum_kernel<<<dim3((F + 128) / 128, chunks, B), 128, 0, p.stream>>>(ws.S, ws.gpart, L, F);
+            spu_coarse_synthesis_kernel<<<dim3((N + 255) / 256, B), 256, 0, p.stream>>>(ws.gpart, E, N, L, F, chunks);
+            count_launch(3);
+        }
     } else {
         const int tiles = (D + BN - 1) / BN;
         spu_contract_kernel<T, true><<<dim3(tiles, (R + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
             p.hidden, ws.Y, ws.tw, ws.scale, N, D, sigma);
         spu_contract_kernel<T, false><<<dim3(tiles, (N + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
             ws.Y, ws.part, ws.tw, ws.scale, N, D, sigma);
-        spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn);
+        spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn, 0);
         count_launch(3);
     }
     phase_end(LUVC_PHASE_SPU_TRANSFORM, p.stream);

@@ -314,20 +314,36 @@ SpuTcPlan spu_tc_plan(int B, int N, int D, int sigma) {
     p.r_pad = (R + 63) / 64 * 64;
     p.n_pad = (N + 127) / 128 * 128;
     p.tiles2 = (D + 255) / 256;
+    // The filtered signal has no frequency above sigma, so its squared row norm has none above
+    // 2 sigma: L > 4 sigma uniform samples of the period determine it on every token (Eq. 7 and 8
+    // evaluated off the token grid, then interpolated).  Used when it saves at least a quarter.
+    const long long need = 4ll * sigma + 2;
+    const long long lp = (need + 127) / 128 * 128;
+    p.coarse = (lp * 4 <= 3ll * p.n_pad) ? 1 : 0;
+    p.L = p.coarse ? (int)lp : N;
+    p.l_pad = p.coarse ? (int)lp : p.n_pad;
     p.phi_elems = (size_t)p.r_pad * p.n_pad;
+    p.phi2_elems = p.coarse ? (size_t)p.r_pad * p.l_pad : 0;
     p.yt_elems = (size_t)B * D * p.r_pad;
-    p.part_elems = (size_t)B * 2 * p.tiles2 * N;
+    p.part_elems = (size_t)B * 2 * p.tiles2 * p.L;
     return p;
 }
 
-int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float* scale, int B, int N, int D,
-               int sigma, int* status, cudaStream_t stream) {
+int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float2* tw2, const float* scale,
+               int B, int N, int D, int sigma, int* status, cudaStream_t stream) {
     const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
     const long long phi_n = (long long)pl.phi_elems;
     spu_phi_kernel<<<(unsigned)((phi_n + 255) / 256), 256, 0, stream>>>(
         tw, reinterpret_cast<__nv_bfloat16*>(w.phi_hi), reinterpret_cast<__nv_bfloat16*>(w.phi_lo), N, sigma,
         pl.r_pad, pl.n_pad);
     count_launch();
+    if (pl.coarse) {   // the same rows sampled at t_j = j N / L: angle 2 pi k t_j / N = 2 pi k j / L
+        const long long phi2_n = (long long)pl.phi2_elems;
+        spu_phi_kernel<<<(unsigned)((phi2_n + 255) / 256), 256, 0, stream>>>(
+            tw2, reinterpret_cast<__nv_bfloat16*>(w.phi2_hi), reinterpret_cast<__nv_bfloat16*>(w.phi2_lo), pl.L, sigma,
+            pl.r_pad, pl.l_pad);
+        count_launch();
+    }
 
     // pass 1: YT[d][r] = c[r] * sum_n X[n][d] PhiT[r][n]
     {
@@ -352,19 +368,19 @@ int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, cons
     // pass 2: part[n] = sum_d (sum_r PhiT[r][n] YT[d][r])^2
     {
         TcArgs g = {};
-        g.a[0] = reinterpret_cast<const __nv_bfloat16*>(w.phi_hi);
-        g.a[1] = reinterpret_cast<const __nv_bfloat16*>(w.phi_lo);
+        g.a[0] = reinterpret_cast<const __nv_bfloat16*>(pl.coarse ? w.phi2_hi : w.phi_hi);
+        g.a[1] = reinterpret_cast<const __nv_bfloat16*>(pl.coarse ? w.phi2_lo : w.phi_lo);
         g.b[0] = reinterpret_cast<const __nv_bfloat16*>(w.yt_hi);
         g.b[1] = reinterpret_cast<const __nv_bfloat16*>(w.yt_lo);
         g.a_batch = 0; g.b_batch = (long long)D * pl.r_pad;
-        g.lda = pl.n_pad; g.ldb = pl.r_pad;
-        g.m_total = pl.n_pad; g.n_total = D; g.k_a = pl.r_pad; g.k_blocks = pl.r_pad / TK;
+        g.lda = pl.l_pad; g.ldb = pl.r_pad;
+        g.m_total = pl.l_pad; g.n_total = D; g.k_a = pl.r_pad; g.k_blocks = pl.r_pad / TK;
         g.tn = 256;
-        g.part = w.part; g.part_n = N;
+        g.part = w.part; g.part_n = pl.L;
         g.status = status;
         const size_t smem = (size_t)kStages * (2 * kABytes + 2 * g.tn * TK * 2);
         cudaFuncSetAttribute(spu_tc_kernel<2, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        spu_tc_kernel<2, 2, true><<<dim3(pl.n_pad / TM, pl.tiles2, B), kThreads, smem, stream>>>(g);
+        spu_tc_kernel<2, 2, true><<<dim3(pl.l_pad / TM, pl.tiles2, B), kThreads, smem, stream>>>(g);
         count_launch();
     }
     return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
