@@ -82,7 +82,21 @@ SpuTcPlan spu_tc_plan(int B, int N, int D, int sigma);
 // Fills part[b][2 * tiles2][L] with per-tile sums of squares of the filtered signal at the L points
 // of the plan.  `scale` must hold r_pad entries (zero beyond 2 sigma + 1); `tw2` is the table of
 // cos / sin of 2 pi j / L (used when the plan is coarse).
+// With `have_yt` the spectrum (yt_hi / yt_lo) is already in place and only the inverse pass runs.
 int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float2* tw2, const float* scale,
-               int B, int N, int D, int sigma, int* status, cudaStream_t stream);
+               int B, int N, int D, int sigma, int* status, cudaStream_t stream, bool have_yt);
+
+// Two-stage forward transform of the bf16 path (spu_fwd2.cu): N = P * Q, P a multiple of 16.
+struct SpuFwd2Plan {
+    int ok;             // 0: N has no usable factor, use the dense contraction
+    int P, Q;
+    int KB, CH;         // kernel variant: band bins per frequency class and channels per thread
+    int slices;         // passes over the input, each covering KB values of k2
+    int n_ctiles, n_items;
+};
+SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma);
+// Y[b][r][d] = c[r] * (band spectrum); also its transposed bf16 pair [b][d][r_pad] when yt_hi is given.
+int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, void* yt_lo, int r_pad, int B, int N,
+                 int D, int sigma, int* status, cudaStream_t stream);
 
 }  // namespace luvc

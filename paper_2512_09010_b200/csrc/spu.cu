@@ -349,7 +349,12 @@ struct Workspace {
     float* part;
     // bf16 path (tensor cores)
     SpuTcBuffers tc;
+    float* Y2;       // band spectrum of the two-stage forward transform [B][2 sigma + 1][D]
 };
+
+size_t fwd2_y_bytes(int B, int N, int D, int sigma) {
+    return spu_fwd2_plan(B, N, D, sigma).ok ? (size_t)B * (2 * (size_t)sigma + 1) * D * sizeof(float) : 0;
+}
 
 size_t coarse_gpart_elems(int B, int L, int sigma) {
     return (size_t)B * ((L + kSpecChunk - 1) / kSpecChunk) * (4 * (size_t)sigma + 1);
@@ -375,6 +380,7 @@ Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path) {
         w.tw2 = reinterpret_cast<float2*>(p); p += align_up((size_t)pl.L * sizeof(float2));
         w.S = reinterpret_cast<float*>(p); p += align_up((size_t)B * pl.L * 4);
         w.gpart = reinterpret_cast<float2*>(p); p += align_up(coarse_gpart_elems(B, pl.L, sigma) * sizeof(float2));
+        w.Y2 = reinterpret_cast<float*>(p); p += align_up(fwd2_y_bytes(B, N, D, sigma));
         w.tc.yt_hi = p; p += align_up(pl.yt_elems * 2);
         w.tc.yt_lo = p; p += align_up(pl.yt_elems * 2);
         w.tc.part = reinterpret_cast<float*>(p);
@@ -393,7 +399,8 @@ size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype) {
     else
         bytes += 2 * align_up(pl.phi_elems * 2) + 2 * align_up(pl.phi2_elems * 2) +
                  align_up((size_t)pl.L * sizeof(float2)) + align_up((size_t)B * pl.L * 4) +
-                 align_up(coarse_gpart_elems(B, pl.L, sigma) * sizeof(float2)) + 2 * align_up(pl.yt_elems * 2) +
+                 align_up(coarse_gpart_elems(B, pl.L, sigma) * sizeof(float2)) +
+                 align_up(fwd2_y_bytes(B, N, D, sigma)) + 2 * align_up(pl.yt_elems * 2) +
                  align_up(pl.part_elems * 4);
     return bytes;
 }
@@ -413,7 +420,13 @@ static int spu_run_typed(const SpuProblem& p) {
                                                                pl.r_pad, p.no_window);
     count_launch();
     if constexpr (kTensor) {
-        const int rc = spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status, p.stream);
+        const bool two_stage = spu_fwd2_plan(B, N, D, sigma).ok;
+        if (two_stage) {
+            const int rc1 = spu_fwd2_run(p.hidden, ws.Y2, ws.scale, ws.tc.yt_hi, ws.tc.yt_lo, pl.r_pad, B, N, D, sigma,
+                                         p.status, p.stream);
+            if (rc1 != LUVC_OK) return rc1;
+        }
+        const int rc = spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status, p.stream, two_stage);
         if (rc != LUVC_OK) return rc;
         if (!coarse) {
             spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, E, N, 2 * pl.tiles2, bn, 0);

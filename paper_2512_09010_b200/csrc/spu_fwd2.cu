@@ -1,0 +1,420 @@
+// Two-stage forward transform of the Spectrum Pruning Unit for bf16 tokens (Eq. 4, restricted to
+// the pass band |f| <= sigma of Eq. 5), for sequence lengths N = P * Q with P a multiple of 16.
+//
+// Token n = p Q + q, frequency k = k1 + P k2:
+//   stage 1   A_q[k1] = sum_p x[p Q + q] e^{-2 pi i k1 p / P}        all k1: a dense P-point DFT over
+//                                                                    tokens that are Q apart
+//   stage 2   X[k]    = sum_q e^{-2 pi i q k / N} A_q[k mod P]       only the bins 0 <= k <= sigma
+// Stage 1 is a real P x P matrix (rows: A[0], A[P/2], then Re / Im of A[1 .. P/2-1]; the other half
+// follows from A[P-k1] = conj A[k1] because x is real) applied to a tile of Q-strided tokens: one
+// tcgen05 contraction per tile, the matrix held in shared memory as a bf16 pair (hi + lo) built
+// once per CTA, the token tile copied from global memory with 16-byte cp.async straight into the
+// no-swizzle operand layout, fp32 accumulators in TMEM (two buffers).  Stage 2 runs on the CUDA
+// cores straight out of TMEM: the thread that owns TMEM lane j owns the frequency pair
+// (k1, P - k1) of that row and keeps its band bins for a few channels in registers for the whole
+// sequence, so the input is read exactly once and nothing but the band spectrum is written:
+//   Y[b][r][d], r = k (cos rows, 0..sigma) and r = sigma + k (sin rows, k >= 1), times the row
+//   constants c[r] (mask of Eq. 5/6, 1/N and the weight of the conjugate half).
+//
+// Roles inside a CTA (persistent over work items = sequence x channel tile x bin slice):
+//   16 epilogue warps (stage 2), 3 copy warps, 1 thread issuing the MMAs; mbarrier rings between
+//   them, every wait bounded (on expiry: status word, drain, free TMEM, return).
+
+#include <cuda_bf16.h>
+
+#include "luvc_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace luvc {
+namespace {
+
+using namespace ptx;
+
+constexpr int kEpiWarps = 16;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kThreads = kEpiThreads + 128;   // plus copy warps 16, 18, 19 and MMA warp 17
+constexpr int kCopyLanes = 96;
+constexpr int kNmma = 256;                    // columns of a tile: QT tokens x C channels
+constexpr int kTmemCols = 512;                // two accumulator buffers
+constexpr int kSpin = 1 << 22;
+
+struct FwdArgs {
+    const __nv_bfloat16* x;   // [B][N][D]
+    float* Y;                 // [B][R][D]
+    const float* scale;       // c[r], r < R
+    int* status;
+    int B, N, D, P, Q, sigma, R;
+    int n_ctiles, n_slices, n_items;
+};
+
+// barriers: 0,1 stage full | 2,3 stage empty | 4,5 accumulator full | 6,7 accumulator empty | 8,9 table ready
+enum { kBarFull = 0, kBarEmpty = 2, kBarAccFull = 4, kBarAccEmpty = 6, kBarTab = 8, kBars = 10 };
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, int parity, volatile int* s_fail, int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer();
+    for (int it = 0; it < kSpin; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*s_fail) return false;
+        if ((it & 63) == 63 && global_timer() - t0 > 1000000000ull) break;   // one second
+    }
+    atomicCAS(status, 0, (int)LUVC_ERR_TIMEOUT);
+    *s_fail = 1;
+    return false;
+}
+
+__device__ __forceinline__ float2 cmul(float2 a, float2 b) {
+    return make_float2(a.x * b.x - a.y * b.y, fmaf(a.x, b.y, a.y * b.x));
+}
+// e^{-2 pi i num / den}, 0 <= num < den
+__device__ __forceinline__ float2 root_neg(int num, int den) {
+    float s, c;
+    sincospif(2.0f * (float)num / (float)den, &s, &c);
+    return make_float2(c, -s);
+}
+
+template <int NCOL> __device__ __forceinline__ void tmem_load(uint32_t addr, uint32_t (&v)[NCOL]) {
+    if constexpr (NCOL == 2) tmem_ld2(addr, v);
+    else if constexpr (NCOL == 4) tmem_ld4(addr, v);
+    else tmem_ld8(addr, v);
+}
+
+// KB: band bins per frequency class held by a thread; CH: channels per thread (C = 8 CH per item).
+template <int KB, int CH>
+__global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) {
+    constexpr int C = 8 * CH;
+    constexpr int QT = kNmma / C;
+    constexpr int LOG_CC = CH == 4 ? 2 : (CH == 2 ? 1 : 0);   // log2(C / 8)
+    constexpr int LOG_QT = 5 - LOG_CC;
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long s_bar[kBars];
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_fail;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int P = a.P, Q = a.Q, N = a.N, D = a.D, sigma = a.sigma;
+    const int f_bytes = P * 256;                 // one part of the stage-1 matrix: P/8 K chunks x 128 rows x 16 B
+    const int sbo_b = P * 16 + 16;               // distance between 8-column groups of a token tile (+16: bank spread)
+    const int stage_bytes = 32 * sbo_b;
+    unsigned char* s_fhi = smem;
+    unsigned char* s_flo = smem + f_bytes;
+    unsigned char* s_x = smem + 2 * f_bytes;
+    float2* s_tab = reinterpret_cast<float2*>(s_x + 2 * stage_bytes);   // [2][QT * KB]
+    const uint32_t bar0 = smem_u32(&s_bar[0]);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+    if (tid == 0) {
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(kBarFull + s), 3);
+            mbar_init(bar(kBarEmpty + s), 1);
+            mbar_init(bar(kBarAccFull + s), 1);
+            mbar_init(bar(kBarAccEmpty + s), kEpiWarps);
+            mbar_init(bar(kBarTab + s), kEpiWarps);
+        }
+        s_fail = 0;
+        mbar_fence_init();
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
+
+    // stage-1 matrix, K-major: element (row j, token p) at (j/8)*128 + (p/8)*2048 + (j%8)*16 + (p%8)*2
+    for (int idx = tid; idx < 128 * P; idx += kThreads) {
+        const int j = idx / P, p = idx - j * P;
+        float v = 0.f;
+        if (j == 0) v = 1.f;
+        else if (j == 1) v = (p & 1) ? -1.f : 1.f;
+        else if (j < P) {
+            const int m = ((j >> 1) * p) % P;
+            float s, c;
+            sincospif(2.0f * (float)m / (float)P, &s, &c);
+            v = (j & 1) ? -s : c;
+        }
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        const __nv_bfloat16 l = __float2bfloat16_rn(v - __bfloat162float(h));
+        const int off = (j >> 3) * 128 + (p >> 3) * 2048 + (j & 7) * 16 + (p & 7) * 2;
+        *reinterpret_cast<__nv_bfloat16*>(s_fhi + off) = h;
+        *reinterpret_cast<__nv_bfloat16*>(s_flo + off) = l;
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    volatile int* fail = &s_fail;
+    const int tiles_per_item = (Q + QT - 1) / QT;
+
+    if (warp < kEpiWarps) {
+        // ------------------------------------------------------------------ stage 2 (epilogue warps)
+        const int quarter = warp & 3, grp = warp >> 2;
+        const int j = quarter * 32 + lane;
+        const int i = j >> 1;
+        const bool odd = j & 1, special = i == 0;
+        const bool warp_active = quarter * 32 < P;
+        const int kA = special ? 0 : i, kB = special ? P / 2 : P - i;
+        const int my_c = grp * 2 * CH + (odd ? CH : 0);           // first of this thread's channels in the tile
+        const float2 stepA = root_neg(kA % N, N), stepB = root_neg(kB % N, N);
+        const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+        int u = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
+            const int slice = item % a.n_slices, rest = item / a.n_slices;
+            const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
+            const int k2_lo = slice * KB;
+            // bins of this thread in this slice: k = kA + P (k2_lo + t) <= sigma, likewise kB
+            int nA = (j < P && kA <= sigma) ? (sigma - kA) / P + 1 - k2_lo : 0;
+            int nB = (j < P && kB <= sigma) ? (sigma - kB) / P + 1 - k2_lo : 0;
+            nA = max(0, min(KB, nA));
+            nB = max(0, min(KB, nB));
+            const int nA_w = __reduce_max_sync(0xffffffffu, nA), nB_w = __reduce_max_sync(0xffffffffu, nB);
+            float yA[KB][CH][2], yB[KB][CH][2];
+#pragma unroll
+            for (int t = 0; t < KB; ++t)
+#pragma unroll
+                for (int c = 0; c < CH; ++c) { yA[t][c][0] = yA[t][c][1] = yB[t][c][0] = yB[t][c][1] = 0.f; }
+
+            for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
+                const int q0 = tile * QT, nq = min(QT, Q - q0), buf = u & 1, par = (u >> 1) & 1;
+                // table of e^{-2 pi i q k2 / Q} for the tile's tokens and the slice's k2
+                float2* tab = s_tab + buf * (QT * KB);
+                for (int e = tid; e < QT * KB; e += kEpiThreads) {
+                    const int ql = e / KB, k2 = k2_lo + (e - ql * KB);
+                    tab[e] = root_neg((int)(((long long)(q0 + ql) * k2) % Q), Q);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarTab + buf));
+                ok = wait_bar(bar(kBarTab + buf), par, fail, a.status);
+                ok = wait_bar(bar(kBarAccFull + buf), par, fail, a.status) && ok;
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                float2 rotA = root_neg((int)(((long long)q0 * kA) % N), N);
+                float2 rotB = root_neg((int)(((long long)q0 * kB) % N), N);
+                const uint32_t taddr = lane_addr + (uint32_t)(buf * kNmma + grp * 2 * CH);
+                for (int ql = 0; ql < nq; ++ql) {
+                    uint32_t v[2 * CH];
+                    tmem_load<2 * CH>(taddr + (uint32_t)(ql * C), v);
+                    tmem_ld_wait();
+                    if (ql == nq - 1) {          // this warp has read all it needs of the buffer
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kBarAccEmpty + buf));
+                    }
+                    if (warp_active) {
+                        const float2* trow = tab + ql * KB;
+#pragma unroll
+                        for (int c = 0; c < CH; ++c) {
+                            // the even lane owns the row of real parts, the odd lane the imaginary parts
+                            const float mine = __uint_as_float(odd ? v[CH + c] : v[c]);
+                            const float send = __uint_as_float(odd ? v[c] : v[CH + c]);
+                            const float got = __shfl_xor_sync(0xffffffffu, send, 1);
+                            const float re = odd ? got : mine, im = odd ? mine : got;
+                            // class A uses A[k1], class B its conjugate; the pair of row 0 / row 1 holds
+                            // the two real values A[0] and A[P/2]
+                            const float2 zA = special ? make_float2(re, 0.f) : make_float2(re, im);
+                            const float2 zB = special ? make_float2(im, 0.f) : make_float2(re, -im);
+                            const float2 wA = cmul(rotA, zA), wB = cmul(rotB, zB);
+#pragma unroll
+                            for (int t = 0; t < KB; ++t) {
+                                if (t < nA_w) {
+                                    const float2 g = trow[t];
+                                    yA[t][c][0] = fmaf(g.x, wA.x, fmaf(-g.y, wA.y, yA[t][c][0]));
+                                    yA[t][c][1] = fmaf(g.x, wA.y, fmaf(g.y, wA.x, yA[t][c][1]));
+                                }
+                                if (t < nB_w) {
+                                    const float2 g = trow[t];
+                                    yB[t][c][0] = fmaf(g.x, wB.x, fmaf(-g.y, wB.y, yB[t][c][0]));
+                                    yB[t][c][1] = fmaf(g.x, wB.y, fmaf(g.y, wB.x, yB[t][c][1]));
+                                }
+                            }
+                        }
+                        rotA = cmul(rotA, stepA);
+                        rotB = cmul(rotB, stepB);
+                    }
+                }
+            }
+            if (!ok) break;
+            // band spectrum of this thread's channels: cos row k, sin row sigma + k
+            const int ch0 = ctile * C + my_c;
+            if (ch0 < D) {
+                float* Yb = a.Y + (size_t)b * a.R * D + ch0;
+#pragma unroll
+                for (int cls = 0; cls < 2; ++cls) {
+                    const int kbase = cls == 0 ? kA : kB, cnt = cls == 0 ? nA : nB;
+#pragma unroll
+                    for (int t = 0; t < KB; ++t) {
+                        if (t >= cnt) continue;
+                        const int k = kbase + P * (k2_lo + t);
+                        const float cr = __ldg(a.scale + k);
+                        float* yr = Yb + (size_t)k * D;
+#pragma unroll
+                        for (int c = 0; c < CH; ++c) yr[c] = cr * (cls == 0 ? yA[t][c][0] : yB[t][c][0]);
+                        if (k >= 1) {
+                            const float ci = __ldg(a.scale + sigma + k);
+                            float* yi = Yb + (size_t)(sigma + k) * D;
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) yi[c] = ci * (cls == 0 ? yA[t][c][1] : yB[t][c][1]);
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == kEpiWarps + 1) {
+        // ------------------------------------------------------------------ MMA issue (one thread)
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(128, kNmma, false, true);
+            const uint32_t fhi = smem_u32(s_fhi), flo = smem_u32(s_flo), xs = smem_u32(s_x);
+            int u = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
+                for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
+                    const int buf = u & 1, par = (u >> 1) & 1;
+                    ok = wait_bar(bar(kBarFull + buf), par, fail, a.status) &&
+                         wait_bar(bar(kBarAccEmpty + buf), par ^ 1, fail, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t xb = xs + buf * stage_bytes, acc = tmem + (uint32_t)(buf * kNmma);
+                    for (int ks = 0; ks < P / 16; ++ks) {
+                        const uint64_t bd = make_desc(xb + ks * 256, 128, sbo_b);
+                        umma_bf16(acc, make_desc(fhi + ks * 4096, 2048, 128), bd, idesc, ks ? 1u : 0u);
+                        umma_bf16(acc, make_desc(flo + ks * 4096, 2048, 128), bd, idesc, 1u);
+                    }
+                    umma_commit(bar(kBarEmpty + buf));
+                    umma_commit(bar(kBarAccFull + buf));
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ copy warps
+        const int l = (warp == kEpiWarps ? 0 : warp - kEpiWarps - 1) * 32 + lane;   // 0 .. 95
+        const uint32_t xs = smem_u32(s_x);
+        int u = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
+            const int rest = item / a.n_slices;
+            const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
+            const int c0 = ctile * C;
+            const __nv_bfloat16* xb = a.x + (size_t)b * N * D + c0;
+            for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
+                const int q0 = tile * QT, buf = u & 1, par = (u >> 1) & 1;
+                ok = wait_bar(bar(kBarEmpty + buf), par ^ 1, fail, a.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t sbase = xs + buf * stage_bytes;
+                // chunk index bits: [channel chunk][token p mod 8][tile token ql][p / 8]
+                for (int idx = l; idx < 32 * P; idx += kCopyLanes) {
+                    const int cc = idx & ((1 << LOG_CC) - 1), pr = (idx >> LOG_CC) & 7;
+                    const int ql = (idx >> (LOG_CC + 3)) & (QT - 1), pg = idx >> (LOG_CC + 3 + LOG_QT);
+                    const bool valid = q0 + ql < Q && c0 + cc * 8 < D;
+                    const uint32_t dst = sbase + (uint32_t)((ql << LOG_CC) + cc) * sbo_b + pg * 128 + pr * 16;
+                    const __nv_bfloat16* src = xb + ((size_t)(pg * 8 + pr) * Q + q0 + ql) * D + cc * 8;
+                    cp_async16(dst, valid ? (const void*)src : (const void*)a.x, valid);
+                }
+                cp_async_commit();
+                if (u > 0) {      // the previous tile has landed: publish it
+                    cp_async_wait<1>();
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarFull + (buf ^ 1)));
+                }
+            }
+        }
+        cp_async_wait<0>();
+        fence_proxy_async();
+        __syncwarp();
+        if (ok && u > 0 && lane == 0) mbar_arrive(bar(kBarFull + ((u - 1) & 1)));
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// YT[b][d][r] (bf16 pair, r padded with zeros to r_pad) from Y[b][r][d]
+__global__ void __launch_bounds__(256) spu_y_transpose_kernel(const float* __restrict__ Y, __nv_bfloat16* __restrict__ hi,
+                                                              __nv_bfloat16* __restrict__ lo, int R, int r_pad, int D) {
+    __shared__ float tile[32][33];
+    const int b = blockIdx.z, r0 = blockIdx.x * 32, d0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int rr = ty; rr < 32; rr += 8) {
+        const int r = r0 + rr, d = d0 + tx;
+        tile[rr][tx] = (r < R && d < D) ? Y[((size_t)b * R + r) * D + d] : 0.f;
+    }
+    __syncthreads();
+    for (int dd = ty; dd < 32; dd += 8) {
+        const int d = d0 + dd, r = r0 + tx;
+        if (d < D && r < r_pad) {
+            const float v = tile[tx][dd];
+            const __nv_bfloat16 h = __float2bfloat16_rn(v);
+            const size_t o = ((size_t)b * D + d) * r_pad + r;
+            hi[o] = h;
+            lo[o] = __float2bfloat16_rn(v - __bfloat162float(h));
+        }
+    }
+}
+
+template <int KB, int CH>
+cudaError_t launch_fwd2(const FwdArgs& a, const SpuFwd2Plan& pl, cudaStream_t stream) {
+    constexpr int QT = kNmma / (8 * CH);
+    const size_t smem = (size_t)2 * a.P * 256 + (size_t)2 * 32 * (a.P * 16 + 16) + (size_t)2 * QT * KB * sizeof(float2);
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    cudaFuncSetAttribute(spu_fwd2_kernel<KB, CH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const int grid = pl.n_items < sms ? pl.n_items : sms;
+    spu_fwd2_kernel<KB, CH><<<grid, kThreads, smem, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma) {
+    SpuFwd2Plan pl = {};
+    for (int p = 128; p >= 16; p -= 16)
+        if (N % p == 0) { pl.P = p; break; }
+    if (!pl.P) return pl;
+    pl.Q = N / pl.P;
+    const int nk2 = sigma / pl.P + 1;                  // values of k2 that reach into the band
+    const int kbs[3] = {4, 9, 17}, chs[3] = {4, 2, 1};
+    int best = -1;
+    for (int v = 0; v < 3; ++v) {
+        const int slices = (nk2 + kbs[v] - 1) / kbs[v];
+        if (best < 0 || slices < pl.slices) { best = v; pl.slices = slices; }
+    }
+    pl.KB = kbs[best];
+    pl.CH = chs[best];
+    const int C = 8 * pl.CH;
+    pl.n_ctiles = (D + C - 1) / C;
+    const long long items = (long long)B * pl.n_ctiles * pl.slices;
+    if (items > 0x7fffffffll) return pl;
+    pl.n_items = (int)items;
+    pl.ok = 1;
+    return pl;
+}
+
+int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, void* yt_lo, int r_pad, int B, int N,
+                 int D, int sigma, int* status, cudaStream_t stream) {
+    const SpuFwd2Plan pl = spu_fwd2_plan(B, N, D, sigma);
+    if (!pl.ok) return LUVC_ERR_INTERNAL;
+    FwdArgs a;
+    a.x = reinterpret_cast<const __nv_bfloat16*>(hidden);
+    a.Y = Y; a.scale = scale; a.status = status;
+    a.B = B; a.N = N; a.D = D; a.P = pl.P; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
+    a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
+    cudaError_t err;
+    if (pl.KB == 4) err = launch_fwd2<4, 4>(a, pl, stream);
+    else if (pl.KB == 9) err = launch_fwd2<9, 2>(a, pl, stream);
+    else err = launch_fwd2<17, 1>(a, pl, stream);
+    count_launch();
+    if (err != cudaSuccess) return LUVC_ERR_CUDA;
+    if (yt_hi != nullptr) {
+        const int R = 2 * sigma + 1;
+        spu_y_transpose_kernel<<<dim3((r_pad + 31) / 32, (D + 31) / 32, B), 256, 0, stream>>>(
+            Y, reinterpret_cast<__nv_bfloat16*>(yt_hi), reinterpret_cast<__nv_bfloat16*>(yt_lo), R, r_pad, D);
+        count_launch();
+    }
+    return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
+}
+
+}  // namespace luvc

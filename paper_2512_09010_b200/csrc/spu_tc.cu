@@ -330,13 +330,15 @@ SpuTcPlan spu_tc_plan(int B, int N, int D, int sigma) {
 }
 
 int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float2* tw2, const float* scale,
-               int B, int N, int D, int sigma, int* status, cudaStream_t stream) {
+               int B, int N, int D, int sigma, int* status, cudaStream_t stream, bool have_yt) {
     const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
-    const long long phi_n = (long long)pl.phi_elems;
-    spu_phi_kernel<<<(unsigned)((phi_n + 255) / 256), 256, 0, stream>>>(
-        tw, reinterpret_cast<__nv_bfloat16*>(w.phi_hi), reinterpret_cast<__nv_bfloat16*>(w.phi_lo), N, sigma,
-        pl.r_pad, pl.n_pad);
-    count_launch();
+    if (!have_yt || !pl.coarse) {
+        const long long phi_n = (long long)pl.phi_elems;
+        spu_phi_kernel<<<(unsigned)((phi_n + 255) / 256), 256, 0, stream>>>(
+            tw, reinterpret_cast<__nv_bfloat16*>(w.phi_hi), reinterpret_cast<__nv_bfloat16*>(w.phi_lo), N, sigma,
+            pl.r_pad, pl.n_pad);
+        count_launch();
+    }
     if (pl.coarse) {   // the same rows sampled at t_j = j N / L: angle 2 pi k t_j / N = 2 pi k j / L
         const long long phi2_n = (long long)pl.phi2_elems;
         spu_phi_kernel<<<(unsigned)((phi2_n + 255) / 256), 256, 0, stream>>>(
@@ -346,7 +348,7 @@ int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, cons
     }
 
     // pass 1: YT[d][r] = c[r] * sum_n X[n][d] PhiT[r][n]
-    {
+    if (!have_yt) {
         TcArgs g = {};
         g.a[0] = reinterpret_cast<const __nv_bfloat16*>(hidden); g.a[1] = nullptr;
         g.b[0] = reinterpret_cast<const __nv_bfloat16*>(w.phi_hi);
