@@ -90,6 +90,7 @@ int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, cons
 struct SpuFwd2Plan {
     int ok;             // 0: N has no usable factor, use the dense contraction
     int P, Q;
+    int nblk;           // 128 / P channel blocks share one tile (block-diagonal stage-1 operand)
     int KB, CH;         // kernel variant: band bins per frequency class and channels per thread
     int slices;         // passes over the input, each covering KB values of k2
     int n_ctiles, n_items;

@@ -32,8 +32,9 @@ using namespace ptx;
 
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kThreads = kEpiThreads + 128;   // plus copy warps 16, 18, 19 and MMA warp 17
-constexpr int kCopyLanes = 96;
+constexpr int kThreads = kEpiThreads + 128;   // plus copy warps 16, 18, 19 and the MMA warp 17 (registers are
+                                              // granted per four warps, so a fifth group costs nothing extra)
+constexpr int kCopyWarps = 3;
 constexpr int kNmma = 256;                    // columns of a tile: QT tokens x C channels
 constexpr int kTmemCols = 512;                // two accumulator buffers
 constexpr int kSpin = 1 << 22;
@@ -44,6 +45,8 @@ struct FwdArgs {
     const float* scale;       // c[r], r < R
     int* status;
     int B, N, D, P, Q, sigma, R;
+    int nblk;                 // copies of the P x P matrix on the diagonal of the 128-row operand: each
+                              // serves its own block of channels of the same tokens (P <= 64)
     int n_ctiles, n_slices, n_items;
 };
 
@@ -67,7 +70,7 @@ __device__ __forceinline__ float2 cmul(float2 a, float2 b) {
     return make_float2(a.x * b.x - a.y * b.y, fmaf(a.x, b.y, a.y * b.x));
 }
 // e^{-2 pi i num / den}, 0 <= num < den
-__device__ __forceinline__ float2 root_neg(int num, int den) {
+__device__ __forceinline__ float2 root_neg(unsigned num, unsigned den) {
     float s, c;
     sincospif(2.0f * (float)num / (float)den, &s, &c);
     return make_float2(c, -s);
@@ -76,16 +79,65 @@ __device__ __forceinline__ float2 root_neg(int num, int den) {
 template <int NCOL> __device__ __forceinline__ void tmem_load(uint32_t addr, uint32_t (&v)[NCOL]) {
     if constexpr (NCOL == 2) tmem_ld2(addr, v);
     else if constexpr (NCOL == 4) tmem_ld4(addr, v);
-    else tmem_ld8(addr, v);
+    else if constexpr (NCOL == 8) tmem_ld8(addr, v);
+    else tmem_ld16(addr, v);
 }
 
-// KB: band bins per frequency class held by a thread; CH: channels per thread (C = 8 CH per item).
+// Stage 2 of one tile for one thread: NA / NB bins of the two frequency classes (compile time, so
+// that the loops carry no branches).  `tab` holds e^{-2 pi i q k2 / Q} for the tile's tokens.
+template <int KB, int CH, int NA, int NB>
+__device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float2* __restrict__ tab, float2& rotA,
+                                            float2& rotB, float2 stepA, float2 stepB, bool odd, bool special,
+                                            bool warp_active, uint32_t acc_empty_bar, int lane,
+                                            float (&yA)[KB][CH][2], float (&yB)[KB][CH][2]) {
+    constexpr int C = 8 * CH;
+    for (int ql = 0; ql < nq; ++ql) {
+        uint32_t v[2 * CH];
+        tmem_load<2 * CH>(taddr + (uint32_t)(ql * C), v);
+        tmem_ld_wait();
+        if (ql == nq - 1) {          // this warp has read all it needs of the buffer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar);
+        }
+        if (!warp_active) continue;
+        float2 g[KB];
+#pragma unroll
+        for (int t = 0; t < (NA > NB ? NA : NB); ++t) g[t] = tab[ql * KB + t];
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            // the even lane owns the row of real parts, the odd lane the imaginary parts
+            const float mine = __uint_as_float(odd ? v[CH + c] : v[c]);
+            const float send = __uint_as_float(odd ? v[c] : v[CH + c]);
+            const float got = __shfl_xor_sync(0xffffffffu, send, 1);
+            const float re = odd ? got : mine, im = odd ? mine : got;
+            // class A uses A[k1], class B its conjugate; the pair of rows 0 / 1 holds the two real
+            // values A[0] and A[P/2]
+            const float2 zA = make_float2(re, special ? 0.f : im);
+            const float2 zB = make_float2(special ? im : re, special ? 0.f : -im);
+            const float2 wA = cmul(rotA, zA), wB = cmul(rotB, zB);
+#pragma unroll
+            for (int t = 0; t < NA; ++t) {
+                yA[t][c][0] = fmaf(g[t].x, wA.x, fmaf(-g[t].y, wA.y, yA[t][c][0]));
+                yA[t][c][1] = fmaf(g[t].x, wA.y, fmaf(g[t].y, wA.x, yA[t][c][1]));
+            }
+#pragma unroll
+            for (int t = 0; t < NB; ++t) {
+                yB[t][c][0] = fmaf(g[t].x, wB.x, fmaf(-g[t].y, wB.y, yB[t][c][0]));
+                yB[t][c][1] = fmaf(g[t].x, wB.y, fmaf(g[t].y, wB.x, yB[t][c][1]));
+            }
+        }
+        rotA = cmul(rotA, stepA);
+        rotB = cmul(rotB, stepB);
+    }
+}
+
+// KB: band bins per frequency class held by a thread; CH: channels per thread (C = 8 CH per block).
 template <int KB, int CH>
 __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) {
     constexpr int C = 8 * CH;
     constexpr int QT = kNmma / C;
-    constexpr int LOG_CC = CH == 4 ? 2 : (CH == 2 ? 1 : 0);   // log2(C / 8)
-    constexpr int LOG_QT = 5 - LOG_CC;
+    constexpr int LOG_CC = CH == 8 ? 3 : (CH == 4 ? 2 : (CH == 2 ? 1 : 0));   // log2(C / 8)
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long s_bar[kBars];
     __shared__ uint32_t s_tmem;
@@ -93,8 +145,9 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int P = a.P, Q = a.Q, N = a.N, D = a.D, sigma = a.sigma;
-    const int f_bytes = P * 256;                 // one part of the stage-1 matrix: P/8 K chunks x 128 rows x 16 B
-    const int sbo_b = P * 16 + 16;               // distance between 8-column groups of a token tile (+16: bank spread)
+    const int KT = a.nblk * P;                   // K extent of a tile: nblk channel blocks x P tokens
+    const int f_bytes = KT * 256;                // one part of the stage-1 matrix: KT/8 K chunks x 128 rows x 16 B
+    const int sbo_b = KT * 16 + 16;              // distance between 8-column groups of a token tile (+16: bank spread)
     const int stage_bytes = 32 * sbo_b;
     unsigned char* s_fhi = smem;
     unsigned char* s_flo = smem + f_bytes;
@@ -105,7 +158,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
 
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(kBarFull + s), 3);
+            mbar_init(bar(kBarFull + s), kCopyWarps);
             mbar_init(bar(kBarEmpty + s), 1);
             mbar_init(bar(kBarAccFull + s), 1);
             mbar_init(bar(kBarAccEmpty + s), kEpiWarps);
@@ -116,21 +169,25 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
     }
     if (warp == 0) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
 
-    // stage-1 matrix, K-major: element (row j, token p) at (j/8)*128 + (p/8)*2048 + (j%8)*16 + (p%8)*2
-    for (int idx = tid; idx < 128 * P; idx += kThreads) {
-        const int j = idx / P, p = idx - j * P;
+    // stage-1 matrix, K-major: element (row j, column kk) at (j/8)*128 + (kk/8)*2048 + (j%8)*16 + (kk%8)*2;
+    // block-diagonal: row j = jb P + jr meets column kk = kb P + p only for jb == kb
+    for (int idx = tid; idx < 128 * KT; idx += kThreads) {
+        const int j = idx / KT, kk = idx - j * KT;
+        const int jb = j / P, jr = j - jb * P, kb = kk / P, p = kk - kb * P;
         float v = 0.f;
-        if (j == 0) v = 1.f;
-        else if (j == 1) v = (p & 1) ? -1.f : 1.f;
-        else if (j < P) {
-            const int m = ((j >> 1) * p) % P;
-            float s, c;
-            sincospif(2.0f * (float)m / (float)P, &s, &c);
-            v = (j & 1) ? -s : c;
+        if (j < KT && jb == kb) {
+            if (jr == 0) v = 1.f;
+            else if (jr == 1) v = (p & 1) ? -1.f : 1.f;
+            else {
+                const int m = ((jr >> 1) * p) % P;
+                float s, c;
+                sincospif(2.0f * (float)m / (float)P, &s, &c);
+                v = (jr & 1) ? -s : c;
+            }
         }
         const __nv_bfloat16 h = __float2bfloat16_rn(v);
         const __nv_bfloat16 l = __float2bfloat16_rn(v - __bfloat162float(h));
-        const int off = (j >> 3) * 128 + (p >> 3) * 2048 + (j & 7) * 16 + (p & 7) * 2;
+        const int off = (j >> 3) * 128 + (kk >> 3) * 2048 + (j & 7) * 16 + (kk & 7) * 2;
         *reinterpret_cast<__nv_bfloat16*>(s_fhi + off) = h;
         *reinterpret_cast<__nv_bfloat16*>(s_flo + off) = l;
     }
@@ -141,16 +198,19 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
     const uint32_t tmem = s_tmem;
     volatile int* fail = &s_fail;
     const int tiles_per_item = (Q + QT - 1) / QT;
+    const int item_channels = a.nblk * C;
 
     if (warp < kEpiWarps) {
         // ------------------------------------------------------------------ stage 2 (epilogue warps)
         const int quarter = warp & 3, grp = warp >> 2;
         const int j = quarter * 32 + lane;
-        const int i = j >> 1;
-        const bool odd = j & 1, special = i == 0;
-        const bool warp_active = quarter * 32 < P;
+        const int jb = j / P, jr = j - jb * P;
+        const bool active = j < KT;
+        const int i = jr >> 1;
+        const bool odd = jr & 1, special = i == 0;
+        const bool warp_active = quarter * 32 < KT;
         const int kA = special ? 0 : i, kB = special ? P / 2 : P - i;
-        const int my_c = grp * 2 * CH + (odd ? CH : 0);           // first of this thread's channels in the tile
+        const int my_c = jb * C + grp * 2 * CH + (odd ? CH : 0);   // first of this thread's channels in the item
         const float2 stepA = root_neg(kA % N, N), stepB = root_neg(kB % N, N);
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         int u = 0;
@@ -160,8 +220,8 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
             const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
             const int k2_lo = slice * KB;
             // bins of this thread in this slice: k = kA + P (k2_lo + t) <= sigma, likewise kB
-            int nA = (j < P && kA <= sigma) ? (sigma - kA) / P + 1 - k2_lo : 0;
-            int nB = (j < P && kB <= sigma) ? (sigma - kB) / P + 1 - k2_lo : 0;
+            int nA = (active && kA <= sigma) ? (sigma - kA) / P + 1 - k2_lo : 0;
+            int nB = (active && kB <= sigma) ? (sigma - kB) / P + 1 - k2_lo : 0;
             nA = max(0, min(KB, nA));
             nB = max(0, min(KB, nB));
             const int nA_w = __reduce_max_sync(0xffffffffu, nA), nB_w = __reduce_max_sync(0xffffffffu, nB);
@@ -177,7 +237,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
                 float2* tab = s_tab + buf * (QT * KB);
                 for (int e = tid; e < QT * KB; e += kEpiThreads) {
                     const int ql = e / KB, k2 = k2_lo + (e - ql * KB);
-                    tab[e] = root_neg((int)(((long long)(q0 + ql) * k2) % Q), Q);
+                    tab[e] = root_neg(((unsigned)(q0 + ql) * (unsigned)k2) % (unsigned)Q, Q);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarTab + buf));
@@ -186,55 +246,23 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                float2 rotA = root_neg((int)(((long long)q0 * kA) % N), N);
-                float2 rotB = root_neg((int)(((long long)q0 * kB) % N), N);
+                float2 rotA = root_neg(((unsigned)q0 * (unsigned)kA) % (unsigned)N, N);   // q0 kA < Q P = N
+                float2 rotB = root_neg(((unsigned)q0 * (unsigned)kB) % (unsigned)N, N);
                 const uint32_t taddr = lane_addr + (uint32_t)(buf * kNmma + grp * 2 * CH);
-                for (int ql = 0; ql < nq; ++ql) {
-                    uint32_t v[2 * CH];
-                    tmem_load<2 * CH>(taddr + (uint32_t)(ql * C), v);
-                    tmem_ld_wait();
-                    if (ql == nq - 1) {          // this warp has read all it needs of the buffer
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(kBarAccEmpty + buf));
-                    }
-                    if (warp_active) {
-                        const float2* trow = tab + ql * KB;
-#pragma unroll
-                        for (int c = 0; c < CH; ++c) {
-                            // the even lane owns the row of real parts, the odd lane the imaginary parts
-                            const float mine = __uint_as_float(odd ? v[CH + c] : v[c]);
-                            const float send = __uint_as_float(odd ? v[c] : v[CH + c]);
-                            const float got = __shfl_xor_sync(0xffffffffu, send, 1);
-                            const float re = odd ? got : mine, im = odd ? mine : got;
-                            // class A uses A[k1], class B its conjugate; the pair of row 0 / row 1 holds
-                            // the two real values A[0] and A[P/2]
-                            const float2 zA = special ? make_float2(re, 0.f) : make_float2(re, im);
-                            const float2 zB = special ? make_float2(im, 0.f) : make_float2(re, -im);
-                            const float2 wA = cmul(rotA, zA), wB = cmul(rotB, zB);
-#pragma unroll
-                            for (int t = 0; t < KB; ++t) {
-                                if (t < nA_w) {
-                                    const float2 g = trow[t];
-                                    yA[t][c][0] = fmaf(g.x, wA.x, fmaf(-g.y, wA.y, yA[t][c][0]));
-                                    yA[t][c][1] = fmaf(g.x, wA.y, fmaf(g.y, wA.x, yA[t][c][1]));
-                                }
-                                if (t < nB_w) {
-                                    const float2 g = trow[t];
-                                    yB[t][c][0] = fmaf(g.x, wB.x, fmaf(-g.y, wB.y, yB[t][c][0]));
-                                    yB[t][c][1] = fmaf(g.x, wB.y, fmaf(g.y, wB.x, yB[t][c][1]));
-                                }
-                            }
-                        }
-                        rotA = cmul(rotA, stepA);
-                        rotB = cmul(rotB, stepB);
-                    }
-                }
+                const uint32_t eb = bar(kBarAccEmpty + buf);
+                if (nA_w == KB && nB_w == KB)
+                    stage2_tile<KB, CH, KB, KB>(taddr, nq, tab, rotA, rotB, stepA, stepB, odd, special, warp_active, eb, lane, yA, yB);
+                else if (nA_w == KB && nB_w == KB - 1)
+                    stage2_tile<KB, CH, KB, KB - 1>(taddr, nq, tab, rotA, rotB, stepA, stepB, odd, special, warp_active, eb, lane, yA, yB);
+                else if (nA_w <= KB - 1 && nB_w <= KB - 1)
+                    stage2_tile<KB, CH, KB - 1, KB - 1>(taddr, nq, tab, rotA, rotB, stepA, stepB, odd, special, warp_active, eb, lane, yA, yB);
+                else
+                    stage2_tile<KB, CH, KB, KB>(taddr, nq, tab, rotA, rotB, stepA, stepB, odd, special, warp_active, eb, lane, yA, yB);
             }
             if (!ok) break;
             // band spectrum of this thread's channels: cos row k, sin row sigma + k
-            const int ch0 = ctile * C + my_c;
-            if (ch0 < D) {
+            const int ch0 = ctile * item_channels + my_c;
+            if (active && ch0 < D) {
                 float* Yb = a.Y + (size_t)b * a.R * D + ch0;
 #pragma unroll
                 for (int cls = 0; cls < 2; ++cls) {
@@ -272,7 +300,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t xb = xs + buf * stage_bytes, acc = tmem + (uint32_t)(buf * kNmma);
-                    for (int ks = 0; ks < P / 16; ++ks) {
+                    for (int ks = 0; ks < KT / 16; ++ks) {
                         const uint64_t bd = make_desc(xb + ks * 256, 128, sbo_b);
                         umma_bf16(acc, make_desc(fhi + ks * 4096, 2048, 128), bd, idesc, ks ? 1u : 0u);
                         umma_bf16(acc, make_desc(flo + ks * 4096, 2048, 128), bd, idesc, 1u);
@@ -284,29 +312,38 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
         }
     } else {
         // ------------------------------------------------------------------ copy warps
-        const int l = (warp == kEpiWarps ? 0 : warp - kEpiWarps - 1) * 32 + lane;   // 0 .. 95
+        const int cw = warp == kEpiWarps ? 0 : warp - kEpiWarps - 1;
         const uint32_t xs = smem_u32(s_x);
         int u = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
             const int rest = item / a.n_slices;
             const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
-            const int c0 = ctile * C;
-            const __nv_bfloat16* xb = a.x + (size_t)b * N * D + c0;
+            const int c0 = ctile * item_channels;
+            const __nv_bfloat16* xrow = a.x + (size_t)b * N * D;
             for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
                 const int q0 = tile * QT, buf = u & 1, par = (u >> 1) & 1;
                 ok = wait_bar(bar(kBarEmpty + buf), par ^ 1, fail, a.status);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 const uint32_t sbase = xs + buf * stage_bytes;
-                // chunk index bits: [channel chunk][token p mod 8][tile token ql][p / 8]
-                for (int idx = l; idx < 32 * P; idx += kCopyLanes) {
-                    const int cc = idx & ((1 << LOG_CC) - 1), pr = (idx >> LOG_CC) & 7;
-                    const int ql = (idx >> (LOG_CC + 3)) & (QT - 1), pg = idx >> (LOG_CC + 3 + LOG_QT);
-                    const bool valid = q0 + ql < Q && c0 + cc * 8 < D;
-                    const uint32_t dst = sbase + (uint32_t)((ql << LOG_CC) + cc) * sbo_b + pg * 128 + pr * 16;
-                    const __nv_bfloat16* src = xb + ((size_t)(pg * 8 + pr) * Q + q0 + ql) * D + cc * 8;
-                    cp_async16(dst, valid ? (const void*)src : (const void*)a.x, valid);
+                // a tile is KT/8 x 256 chunks of 16 bytes; the low 8 index bits are
+                // [channel chunk cc][K row kk mod 8][tile token ql], the rest is kk / 8
+#pragma unroll 1
+                for (int m = cw; m < 8; m += kCopyWarps) {
+                    const int low = lane + 32 * m;
+                    const int cc = low & ((1 << LOG_CC) - 1), kr = (low >> LOG_CC) & 7, ql = low >> (LOG_CC + 3);
+                    const bool q_ok = q0 + ql < Q;
+                    const uint32_t dst0 = sbase + (uint32_t)((ql << LOG_CC) + cc) * sbo_b + kr * 16;
+                    const __nv_bfloat16* src0 = xrow + (size_t)(q0 + ql) * D + cc * 8;
+                    int p = kr, chan = c0 + cc * 8;          // K row kk = kg 8 + kr is token p of channel block jb
+                    for (int kg = 0; kg < KT / 8; ++kg) {
+                        const bool valid = q_ok && chan < D;
+                        cp_async16(dst0 + kg * 128, valid ? (const void*)(src0 + (size_t)p * Q * D + chan - cc * 8)
+                                                          : (const void*)a.x, valid);
+                        p += 8;
+                        if (p >= P) { p -= P; chan += C; }
+                    }
                 }
                 cp_async_commit();
                 if (u > 0) {      // the previous tile has landed: publish it
@@ -354,7 +391,8 @@ __global__ void __launch_bounds__(256) spu_y_transpose_kernel(const float* __res
 template <int KB, int CH>
 cudaError_t launch_fwd2(const FwdArgs& a, const SpuFwd2Plan& pl, cudaStream_t stream) {
     constexpr int QT = kNmma / (8 * CH);
-    const size_t smem = (size_t)2 * a.P * 256 + (size_t)2 * 32 * (a.P * 16 + 16) + (size_t)2 * QT * KB * sizeof(float2);
+    const int KT = a.nblk * a.P;
+    const size_t smem = (size_t)2 * KT * 256 + (size_t)2 * 32 * (KT * 16 + 16) + (size_t)2 * QT * KB * sizeof(float2);
     static int sms = 0;
     if (!sms) {
         int dev = 0;
@@ -375,16 +413,18 @@ SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma) {
         if (N % p == 0) { pl.P = p; break; }
     if (!pl.P) return pl;
     pl.Q = N / pl.P;
+    if (pl.Q > 32768) return pl;                       // keeps q * k2 inside 32 bits
+    pl.nblk = 128 / pl.P;
     const int nk2 = sigma / pl.P + 1;                  // values of k2 that reach into the band
-    const int kbs[3] = {4, 9, 17}, chs[3] = {4, 2, 1};
+    const int kbs[4] = {2, 4, 9, 17}, chs[4] = {8, 4, 2, 1};
     int best = -1;
-    for (int v = 0; v < 3; ++v) {
+    for (int v = 0; v < 4; ++v) {
         const int slices = (nk2 + kbs[v] - 1) / kbs[v];
         if (best < 0 || slices < pl.slices) { best = v; pl.slices = slices; }
     }
     pl.KB = kbs[best];
     pl.CH = chs[best];
-    const int C = 8 * pl.CH;
+    const int C = 8 * pl.CH * pl.nblk;                 // channels of one work item
     pl.n_ctiles = (D + C - 1) / C;
     const long long items = (long long)B * pl.n_ctiles * pl.slices;
     if (items > 0x7fffffffll) return pl;
@@ -401,9 +441,11 @@ int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, 
     a.x = reinterpret_cast<const __nv_bfloat16*>(hidden);
     a.Y = Y; a.scale = scale; a.status = status;
     a.B = B; a.N = N; a.D = D; a.P = pl.P; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
+    a.nblk = pl.nblk;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
     cudaError_t err;
-    if (pl.KB == 4) err = launch_fwd2<4, 4>(a, pl, stream);
+    if (pl.KB == 2) err = launch_fwd2<2, 8>(a, pl, stream);
+    else if (pl.KB == 4) err = launch_fwd2<4, 4>(a, pl, stream);
     else if (pl.KB == 9) err = launch_fwd2<9, 2>(a, pl, stream);
     else err = launch_fwd2<17, 1>(a, pl, stream);
     count_launch();
