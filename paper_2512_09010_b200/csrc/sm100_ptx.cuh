@@ -19,6 +19,14 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint3
            ((uint64_t)((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46);
 }
 
+// The same descriptor for a swizzled layout (rows of 32, 64 or 128 bytes whose 16-byte chunks are
+// XOR-permuted by the row address, as a TMA tensor copy with the matching swizzle mode writes them).
+//   MN-major operand: lbo = distance between swizzle atoms along M/N, sbo = between 8-row K groups
+// `layout` is the 3-bit code: 0 none, 2 128-byte, 4 64-byte, 6 32-byte swizzle.
+__device__ __forceinline__ uint64_t make_desc_layout(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout) {
+    return make_desc(addr, lbo, sbo) | ((uint64_t)(layout & 7u) << 61);
+}
+
 // Instruction descriptor of tcgen05.mma kind::f16: bf16 x bf16 -> fp32, M x N tile.
 __device__ __forceinline__ uint32_t make_idesc_bf16(int m, int n, bool a_mn_major, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
@@ -41,6 +49,17 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
 __device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// One arrival that also announces `bytes` of asynchronous copies that will complete on the barrier.
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// TMA: one box of a 4-D tensor map into this CTA's shared memory (no multicast); completion is
+// counted in bytes on the mbarrier.  c0 (innermost) times the element size must be a multiple of 16.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, int parity) {
     uint32_t ok;

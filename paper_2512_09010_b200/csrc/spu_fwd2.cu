@@ -8,8 +8,9 @@
 // Stage 1 is a real P x P matrix (rows: A[0], A[P/2], then Re / Im of A[1 .. P/2-1]; the other half
 // follows from A[P-k1] = conj A[k1] because x is real) applied to a tile of Q-strided tokens: one
 // tcgen05 contraction per tile, the matrix held in shared memory as a bf16 pair (hi + lo) built
-// once per CTA, the token tile copied from global memory with 16-byte cp.async straight into the
-// no-swizzle operand layout, fp32 accumulators in TMEM (two buffers).  Stage 2 runs on the CUDA
+// once per CTA, the token tile brought in by TMA (one 4-D box {channels, P strided tokens, tile
+// tokens} per channel block, swizzled so that it is a legal MN-major operand as it lands), fp32
+// accumulators in TMEM (two buffers).  Stage 2 runs on the CUDA
 // cores straight out of TMEM: the thread that owns TMEM lane j owns the frequency pair
 // (k1, P - k1) of that row and keeps its band bins for a few channels in registers for the whole
 // sequence, so the input is read exactly once and nothing but the band spectrum is written:
@@ -17,9 +18,10 @@
 //   constants c[r] (mask of Eq. 5/6, 1/N and the weight of the conjugate half).
 //
 // Roles inside a CTA (persistent over work items = sequence x channel tile x bin slice):
-//   16 epilogue warps (stage 2), 3 copy warps, 1 thread issuing the MMAs; mbarrier rings between
+//   16 epilogue warps (stage 2), 1 thread issuing the TMA copies, 1 thread issuing the MMAs; mbarrier rings between
 //   them, every wait bounded (on expiry: status word, drain, free TMEM, return).
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "luvc_internal.h"
@@ -32,9 +34,7 @@ using namespace ptx;
 
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kThreads = kEpiThreads + 128;   // plus copy warps 16, 18, 19 and the MMA warp 17 (registers are
-                                              // granted per four warps, so a fifth group costs nothing extra)
-constexpr int kCopyWarps = 3;
+constexpr int kThreads = kEpiThreads + 64;    // plus the TMA warp (16) and the MMA warp (17)
 constexpr int kNmma = 256;                    // columns of a tile: QT tokens x C channels
 constexpr int kTmemCols = 512;                // two accumulator buffers
 constexpr int kSpin = 1 << 22;
@@ -134,11 +134,13 @@ __device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float2
 
 // KB: band bins per frequency class held by a thread; CH: channels per thread (C = 8 CH per block).
 template <int KB, int CH>
-__global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) {
+__global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_constant__ CUtensorMap tmap, const FwdArgs a) {
     constexpr int C = 8 * CH;
     constexpr int QT = kNmma / C;
     constexpr int LOG_CC = CH == 8 ? 3 : (CH == 4 ? 2 : (CH == 2 ? 1 : 0));   // log2(C / 8)
-    extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int ROWB = 2 * C;                  // bytes of one token row of a tile: 16 (no swizzle), 32, 64 or 128
+    constexpr uint32_t LAYOUT = CH == 8 ? 2u : (CH == 4 ? 4u : (CH == 2 ? 6u : 0u));
+    extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ __align__(8) unsigned long long s_bar[kBars];
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
@@ -147,8 +149,10 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
     const int P = a.P, Q = a.Q, N = a.N, D = a.D, sigma = a.sigma;
     const int KT = a.nblk * P;                   // K extent of a tile: nblk channel blocks x P tokens
     const int f_bytes = KT * 256;                // one part of the stage-1 matrix: KT/8 K chunks x 128 rows x 16 B
-    const int sbo_b = KT * 16 + 16;              // distance between 8-column groups of a token tile (+16: bank spread)
-    const int stage_bytes = 32 * sbo_b;
+    const int blk_bytes = QT * P * ROWB;         // one channel block of a tile: [tile token][P tokens][C channels]
+    const int stage_bytes = a.nblk * blk_bytes;  // = 256 columns x KT rows x 2 bytes
+    // swizzled tiles need their 1024-byte atoms on 1024-byte boundaries (1 KB of slack is requested for this)
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* s_fhi = smem;
     unsigned char* s_flo = smem + f_bytes;
     unsigned char* s_x = smem + 2 * f_bytes;
@@ -158,7 +162,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
 
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(kBarFull + s), kCopyWarps);
+            mbar_init(bar(kBarFull + s), 1);
             mbar_init(bar(kBarEmpty + s), 1);
             mbar_init(bar(kBarAccFull + s), 1);
             mbar_init(bar(kBarAccEmpty + s), kEpiWarps);
@@ -301,7 +305,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
                     tc_fence_after();
                     const uint32_t xb = xs + buf * stage_bytes, acc = tmem + (uint32_t)(buf * kNmma);
                     for (int ks = 0; ks < KT / 16; ++ks) {
-                        const uint64_t bd = make_desc(xb + ks * 256, 128, sbo_b);
+                        // K rows 16 ks .. 16 ks + 15 lie in channel block jb (16 divides P)
+                        const int jb = (ks * 16) / P, kl = ks * 16 - jb * P;
+                        const uint32_t baddr = xb + jb * blk_bytes + kl * ROWB;
+                        const uint64_t bd = LAYOUT ? make_desc_layout(baddr, P * ROWB, 8 * ROWB, LAYOUT)
+                                                   : make_desc(baddr, 128, P * 16);
                         umma_bf16(acc, make_desc(fhi + ks * 4096, 2048, 128), bd, idesc, ks ? 1u : 0u);
                         umma_bf16(acc, make_desc(flo + ks * 4096, 2048, 128), bd, idesc, 1u);
                     }
@@ -311,53 +319,26 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const FwdArgs a) 
             }
         }
     } else {
-        // ------------------------------------------------------------------ copy warps
-        const int cw = warp == kEpiWarps ? 0 : warp - kEpiWarps - 1;
-        const uint32_t xs = smem_u32(s_x);
-        int u = 0;
-        bool ok = true;
-        for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
-            const int rest = item / a.n_slices;
-            const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
-            const int c0 = ctile * item_channels;
-            const __nv_bfloat16* xrow = a.x + (size_t)b * N * D;
-            for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
-                const int q0 = tile * QT, buf = u & 1, par = (u >> 1) & 1;
-                ok = wait_bar(bar(kBarEmpty + buf), par ^ 1, fail, a.status);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const uint32_t sbase = xs + buf * stage_bytes;
-                // a tile is KT/8 x 256 chunks of 16 bytes; the low 8 index bits are
-                // [channel chunk cc][K row kk mod 8][tile token ql], the rest is kk / 8
-#pragma unroll 1
-                for (int m = cw; m < 8; m += kCopyWarps) {
-                    const int low = lane + 32 * m;
-                    const int cc = low & ((1 << LOG_CC) - 1), kr = (low >> LOG_CC) & 7, ql = low >> (LOG_CC + 3);
-                    const bool q_ok = q0 + ql < Q;
-                    const uint32_t dst0 = sbase + (uint32_t)((ql << LOG_CC) + cc) * sbo_b + kr * 16;
-                    const __nv_bfloat16* src0 = xrow + (size_t)(q0 + ql) * D + cc * 8;
-                    int p = kr, chan = c0 + cc * 8;          // K row kk = kg 8 + kr is token p of channel block jb
-                    for (int kg = 0; kg < KT / 8; ++kg) {
-                        const bool valid = q_ok && chan < D;
-                        cp_async16(dst0 + kg * 128, valid ? (const void*)(src0 + (size_t)p * Q * D + chan - cc * 8)
-                                                          : (const void*)a.x, valid);
-                        p += 8;
-                        if (p >= P) { p -= P; chan += C; }
-                    }
-                }
-                cp_async_commit();
-                if (u > 0) {      // the previous tile has landed: publish it
-                    cp_async_wait<1>();
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(kBarFull + (buf ^ 1)));
+        // ------------------------------------------------------------------ TMA issue (one thread)
+        if (lane == 0) {
+            const uint32_t xs = smem_u32(s_x);
+            int u = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
+                const int rest = item / a.n_slices;
+                const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
+                const int c0 = ctile * item_channels;
+                for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
+                    const int q0 = tile * QT, buf = u & 1, par = (u >> 1) & 1;
+                    ok = wait_bar(bar(kBarEmpty + buf), par ^ 1, fail, a.status);
+                    if (!ok) break;
+                    // boxes that reach past Q or D are filled with zeros there and still count in full
+                    mbar_arrive_expect_tx(bar(kBarFull + buf), (uint32_t)stage_bytes);
+                    for (int jb = 0; jb < a.nblk; ++jb)
+                        tma_load_4d(xs + buf * stage_bytes + jb * blk_bytes, &tmap, bar(kBarFull + buf), c0 + jb * C, 0, q0, b);
                 }
             }
         }
-        cp_async_wait<0>();
-        fence_proxy_async();
-        __syncwarp();
-        if (ok && u > 0 && lane == 0) mbar_arrive(bar(kBarFull + ((u - 1) & 1)));
     }
 
     tc_fence_before();
@@ -388,11 +369,42 @@ __global__ void __launch_bounds__(256) spu_y_transpose_kernel(const float* __res
     }
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
 template <int KB, int CH>
 cudaError_t launch_fwd2(const FwdArgs& a, const SpuFwd2Plan& pl, cudaStream_t stream) {
-    constexpr int QT = kNmma / (8 * CH);
+    constexpr int C = 8 * CH, QT = kNmma / C;
     const int KT = a.nblk * a.P;
-    const size_t smem = (size_t)2 * KT * 256 + (size_t)2 * 32 * (KT * 16 + 16) + (size_t)2 * QT * KB * sizeof(float2);
+    // the tokens of one sequence as [q][p][channel]: token p Q + q sits P-strided in memory
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return cudaErrorNotSupported;
+    CUtensorMap tmap;
+    const cuuint64_t dims[4] = {(cuuint64_t)a.D, (cuuint64_t)a.P, (cuuint64_t)a.Q, (cuuint64_t)a.B};
+    const cuuint64_t strides[3] = {(cuuint64_t)a.Q * a.D * 2, (cuuint64_t)a.D * 2, (cuuint64_t)a.N * a.D * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)a.P, (cuuint32_t)QT, 1u};
+    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    const CUtensorMapSwizzle swz = CH == 8 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                 : CH == 4 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                 : CH == 2 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
+    if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(a.x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    const size_t smem = 1024 + (size_t)2 * KT * 256 + (size_t)2 * kNmma * KT * 2 + (size_t)2 * QT * KB * sizeof(float2);
     static int sms = 0;
     if (!sms) {
         int dev = 0;
@@ -401,7 +413,7 @@ cudaError_t launch_fwd2(const FwdArgs& a, const SpuFwd2Plan& pl, cudaStream_t st
     }
     cudaFuncSetAttribute(spu_fwd2_kernel<KB, CH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int grid = pl.n_items < sms ? pl.n_items : sms;
-    spu_fwd2_kernel<KB, CH><<<grid, kThreads, smem, stream>>>(a);
+    spu_fwd2_kernel<KB, CH><<<grid, kThreads, smem, stream>>>(tmap, a);
     return cudaGetLastError();
 }
 
