@@ -17,9 +17,12 @@
 //   Y[b][r][d], r = k (cos rows, 0..sigma) and r = sigma + k (sin rows, k >= 1), times the row
 //   constants c[r] (mask of Eq. 5/6, 1/N and the weight of the conjugate half).
 //
-// Roles inside a CTA (persistent over work items = sequence x channel tile x bin slice):
-//   16 epilogue warps (stage 2), 1 thread issuing the TMA copies, 1 thread issuing the MMAs; mbarrier rings between
-//   them, every wait bounded (on expiry: status word, drain, free TMEM, return).
+// A CTA is persistent over work items (sequence x channel tile x bin slice) and runs 16 warps, all
+// of them doing stage 2.  Thread 0 is also the producer: when the accumulator of tile u has
+// arrived (so the MMAs of tile u are done and their shared-memory stage is free) it issues the TMA
+// copies of tile u + 2 into that stage and the MMAs of tile u + 1 into the other accumulator, which
+// then run underneath stage 2 of tile u.  Every mbarrier wait is bounded (on expiry: status word,
+// free TMEM, return).
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -34,7 +37,7 @@ using namespace ptx;
 
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kThreads = kEpiThreads + 64;    // plus the TMA warp (16) and the MMA warp (17)
+constexpr int kThreads = kEpiThreads;         // no producer warps: thread 0 also issues the TMA copies and the MMAs
 constexpr int kNmma = 256;                    // columns of a tile: QT tokens x C channels
 constexpr int kTmemCols = 512;                // two accumulator buffers
 constexpr int kSpin = 1 << 22;
@@ -50,8 +53,8 @@ struct FwdArgs {
     int n_ctiles, n_slices, n_items;
 };
 
-// barriers: 0,1 stage full | 2,3 stage empty | 4,5 accumulator full | 6,7 accumulator empty | 8,9 table ready
-enum { kBarFull = 0, kBarEmpty = 2, kBarAccFull = 4, kBarAccEmpty = 6, kBarTab = 8, kBars = 10 };
+// barriers: 0,1 stage full | 2,3 accumulator full | 4,5 accumulator empty | 6,7 table ready
+enum { kBarFull = 0, kBarAccFull = 2, kBarAccEmpty = 4, kBarTab = 6, kBars = 8 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, int parity, volatile int* s_fail, int* status) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -163,7 +166,6 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(kBarFull + s), 1);
-            mbar_init(bar(kBarEmpty + s), 1);
             mbar_init(bar(kBarAccFull + s), 1);
             mbar_init(bar(kBarAccEmpty + s), kEpiWarps);
             mbar_init(bar(kBarTab + s), kEpiWarps);
@@ -204,8 +206,49 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     const int tiles_per_item = (Q + QT - 1) / QT;
     const int item_channels = a.nblk * C;
 
-    if (warp < kEpiWarps) {
-        // ------------------------------------------------------------------ stage 2 (epilogue warps)
+    const uint32_t xs = smem_u32(s_x), fhi = smem_u32(s_fhi), flo = smem_u32(s_flo);
+    const uint32_t idesc = make_idesc_bf16(128, kNmma, false, true);
+    int n_my_items = 0;
+    for (int item = blockIdx.x; item < a.n_items; item += gridDim.x) ++n_my_items;
+    const int total_tiles = n_my_items * tiles_per_item;
+
+    // producer steps (thread 0 only)
+    auto issue_tma = [&](int v) {           // tile v of this CTA's sequence of tiles -> stage v & 1
+        const int item = blockIdx.x + (v / tiles_per_item) * gridDim.x, tile = v % tiles_per_item;
+        const int rest = item / a.n_slices;
+        const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
+        const int c0 = ctile * item_channels, buf = v & 1;
+        // boxes that reach past Q or D are filled with zeros there and still count in full
+        mbar_arrive_expect_tx(bar(kBarFull + buf), (uint32_t)stage_bytes);
+        for (int jb = 0; jb < a.nblk; ++jb)
+            tma_load_4d(xs + buf * stage_bytes + jb * blk_bytes, &tmap, bar(kBarFull + buf), c0 + jb * C, 0, tile * QT, b);
+    };
+    auto issue_mma = [&](int v) -> bool {   // needs tile v in its stage and accumulator v & 1 drained
+        const int buf = v & 1;
+        if (!wait_bar(bar(kBarFull + buf), (v >> 1) & 1, fail, a.status)) return false;
+        if (v >= 2 && !wait_bar(bar(kBarAccEmpty + buf), ((v - 2) >> 1) & 1, fail, a.status)) return false;
+        tc_fence_after();
+        const uint32_t xb = xs + buf * stage_bytes, acc = tmem + (uint32_t)(buf * kNmma);
+        for (int ks = 0; ks < KT / 16; ++ks) {
+            // K rows 16 ks .. 16 ks + 15 lie in channel block jb (16 divides P)
+            const int jb = (ks * 16) / P, kl = ks * 16 - jb * P;
+            const uint32_t baddr = xb + jb * blk_bytes + kl * ROWB;
+            const uint64_t bd = LAYOUT ? make_desc_layout(baddr, P * ROWB, 8 * ROWB, LAYOUT) : make_desc(baddr, 128, P * 16);
+            umma_bf16(acc, make_desc(fhi + ks * 4096, 2048, 128), bd, idesc, ks ? 1u : 0u);
+            umma_bf16(acc, make_desc(flo + ks * 4096, 2048, 128), bd, idesc, 1u);
+        }
+        umma_commit(bar(kBarAccFull + buf));
+        return true;
+    };
+    if (tid == 0) {
+        issue_tma(0);
+        if (total_tiles > 1) issue_tma(1);
+        issue_mma(0);
+    }
+    __syncwarp();
+
+    {
+        // ------------------------------------------------------------------ stage 2 (all warps)
         const int quarter = warp & 3, grp = warp >> 2;
         const int j = quarter * 32 + lane;
         const int jb = j / P, jr = j - jb * P;
@@ -247,6 +290,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                 if (lane == 0) mbar_arrive(bar(kBarTab + buf));
                 ok = wait_bar(bar(kBarTab + buf), par, fail, a.status);
                 ok = wait_bar(bar(kBarAccFull + buf), par, fail, a.status) && ok;
+                if (tid == 0 && ok) {
+                    // the MMAs of tile u are done: refill their stage, and start tile u + 1
+                    if (u + 2 < total_tiles) issue_tma(u + 2);
+                    if (u + 1 < total_tiles) ok = issue_mma(u + 1);
+                }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -286,56 +334,6 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                             for (int c = 0; c < CH; ++c) yi[c] = ci * (cls == 0 ? yA[t][c][1] : yB[t][c][1]);
                         }
                     }
-                }
-            }
-        }
-    } else if (warp == kEpiWarps + 1) {
-        // ------------------------------------------------------------------ MMA issue (one thread)
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(128, kNmma, false, true);
-            const uint32_t fhi = smem_u32(s_fhi), flo = smem_u32(s_flo), xs = smem_u32(s_x);
-            int u = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
-                for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
-                    const int buf = u & 1, par = (u >> 1) & 1;
-                    ok = wait_bar(bar(kBarFull + buf), par, fail, a.status) &&
-                         wait_bar(bar(kBarAccEmpty + buf), par ^ 1, fail, a.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t xb = xs + buf * stage_bytes, acc = tmem + (uint32_t)(buf * kNmma);
-                    for (int ks = 0; ks < KT / 16; ++ks) {
-                        // K rows 16 ks .. 16 ks + 15 lie in channel block jb (16 divides P)
-                        const int jb = (ks * 16) / P, kl = ks * 16 - jb * P;
-                        const uint32_t baddr = xb + jb * blk_bytes + kl * ROWB;
-                        const uint64_t bd = LAYOUT ? make_desc_layout(baddr, P * ROWB, 8 * ROWB, LAYOUT)
-                                                   : make_desc(baddr, 128, P * 16);
-                        umma_bf16(acc, make_desc(fhi + ks * 4096, 2048, 128), bd, idesc, ks ? 1u : 0u);
-                        umma_bf16(acc, make_desc(flo + ks * 4096, 2048, 128), bd, idesc, 1u);
-                    }
-                    umma_commit(bar(kBarEmpty + buf));
-                    umma_commit(bar(kBarAccFull + buf));
-                }
-            }
-        }
-    } else {
-        // ------------------------------------------------------------------ TMA issue (one thread)
-        if (lane == 0) {
-            const uint32_t xs = smem_u32(s_x);
-            int u = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
-                const int rest = item / a.n_slices;
-                const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
-                const int c0 = ctile * item_channels;
-                for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
-                    const int q0 = tile * QT, buf = u & 1, par = (u >> 1) & 1;
-                    ok = wait_bar(bar(kBarEmpty + buf), par ^ 1, fail, a.status);
-                    if (!ok) break;
-                    // boxes that reach past Q or D are filled with zeros there and still count in full
-                    mbar_arrive_expect_tx(bar(kBarFull + buf), (uint32_t)stage_bytes);
-                    for (int jb = 0; jb < a.nblk; ++jb)
-                        tma_load_4d(xs + buf * stage_bytes + jb * blk_bytes, &tmap, bar(kBarFull + buf), c0 + jb * C, 0, q0, b);
                 }
             }
         }
