@@ -100,4 +100,16 @@ SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma);
 int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, void* yt_lo, int r_pad, int B, int N,
                  int D, int sigma, int* status, cudaStream_t stream);
 
+// Two-stage inverse transform and energies of the bf16 path (spu_inv2.cu); needs the forward plan.
+struct SpuInv2Plan {
+    int ok;             // 0: use the dense inverse contraction
+    int P, Q, nblk;
+    int coarse, J, L;   // L = P J points of the period (J = Q, L = N when not coarse)
+    int KB, CHT;        // kernel variant
+    int n_ctiles, n_items;
+    int n_parts;        // partial sums per point and sequence: part[b][n_parts][L]
+};
+SpuInv2Plan spu_inv2_plan(int B, int N, int D, int sigma);
+int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream);
+
 }  // namespace luvc

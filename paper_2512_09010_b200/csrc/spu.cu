@@ -339,7 +339,7 @@ __global__ void __launch_bounds__(128) spu_gather_kernel(const uint4* __restrict
 
 struct Workspace {
     float2* tw;
-    float2* tw2;     // table for the coarse period (tensor path)
+    float2* tw2;     // table for the coarse period (dense inverse)
     float* S;        // squared energies at the coarse points [B][L]
     float2* gpart;   // their spectrum, partial sums [B][chunks][2 sigma * 2 + 1]
     float* scale;
@@ -352,8 +352,22 @@ struct Workspace {
     float* Y2;       // band spectrum of the two-stage forward transform [B][2 sigma + 1][D]
 };
 
-size_t fwd2_y_bytes(int B, int N, int D, int sigma) {
-    return spu_fwd2_plan(B, N, D, sigma).ok ? (size_t)B * (2 * (size_t)sigma + 1) * D * sizeof(float) : 0;
+// How the bf16 path runs a problem, and the points its inverse is evaluated on.
+struct Bf16Mode {
+    bool fwd2, inv2;    // two-stage forward / inverse kernels (else the dense contractions of spu_tc.cu)
+    int coarse, L;      // the inverse is evaluated on L uniform points of the period (L = N: the tokens)
+    int n_parts;        // partial energy sums per point
+};
+Bf16Mode bf16_mode(int B, int N, int D, int sigma) {
+    const SpuTcPlan tc = spu_tc_plan(B, N, D, sigma);
+    const SpuInv2Plan iv = spu_inv2_plan(B, N, D, sigma);
+    Bf16Mode m;
+    m.fwd2 = spu_fwd2_plan(B, N, D, sigma).ok != 0;
+    m.inv2 = m.fwd2 && iv.ok != 0;
+    m.coarse = m.inv2 ? iv.coarse : tc.coarse;
+    m.L = m.inv2 ? iv.L : tc.L;
+    m.n_parts = m.inv2 ? iv.n_parts : 2 * tc.tiles2;
+    return m;
 }
 
 size_t coarse_gpart_elems(int B, int L, int sigma) {
@@ -361,48 +375,52 @@ size_t coarse_gpart_elems(int B, int L, int sigma) {
 }
 
 // Both paths share the twiddle table, the row constants and the scores; the rest differs.
-Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path) {
+// With ws == nullptr only the size is computed.
+Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path, size_t* total) {
     unsigned char* p = static_cast<unsigned char*>(ws);
+    unsigned char* const p0 = p;
     const int R = 2 * sigma + 1, tiles = (D + BN - 1) / BN;
     const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
     Workspace w = {};
-    w.tw = reinterpret_cast<float2*>(p); p += align_up((size_t)N * sizeof(float2));
-    w.scale = reinterpret_cast<float*>(p); p += align_up((size_t)pl.r_pad * 4);
-    w.E = reinterpret_cast<float*>(p); p += align_up((size_t)B * N * 4);
+    auto take = [&](size_t bytes) { unsigned char* q = p; p += align_up(bytes); return q; };
+    w.tw = reinterpret_cast<float2*>(take((size_t)N * sizeof(float2)));
+    w.scale = reinterpret_cast<float*>(take((size_t)pl.r_pad * 4));
+    w.E = reinterpret_cast<float*>(take((size_t)B * N * 4));
     if (!tensor_path) {
-        w.Y = reinterpret_cast<float*>(p); p += align_up((size_t)B * R * D * 4);
-        w.part = reinterpret_cast<float*>(p);
+        w.Y = reinterpret_cast<float*>(take((size_t)B * R * D * 4));
+        w.part = reinterpret_cast<float*>(take((size_t)B * tiles * N * 4));
     } else {
-        w.tc.phi_hi = p; p += align_up(pl.phi_elems * 2);
-        w.tc.phi_lo = p; p += align_up(pl.phi_elems * 2);
-        w.tc.phi2_hi = p; p += align_up(pl.phi2_elems * 2);
-        w.tc.phi2_lo = p; p += align_up(pl.phi2_elems * 2);
-        w.tw2 = reinterpret_cast<float2*>(p); p += align_up((size_t)pl.L * sizeof(float2));
-        w.S = reinterpret_cast<float*>(p); p += align_up((size_t)B * pl.L * 4);
-        w.gpart = reinterpret_cast<float2*>(p); p += align_up(coarse_gpart_elems(B, pl.L, sigma) * sizeof(float2));
-        w.Y2 = reinterpret_cast<float*>(p); p += align_up(fwd2_y_bytes(B, N, D, sigma));
-        w.tc.yt_hi = p; p += align_up(pl.yt_elems * 2);
-        w.tc.yt_lo = p; p += align_up(pl.yt_elems * 2);
-        w.tc.part = reinterpret_cast<float*>(p);
+        const Bf16Mode m = bf16_mode(B, N, D, sigma);
+        if (m.coarse) {
+            w.S = reinterpret_cast<float*>(take((size_t)B * m.L * 4));
+            w.gpart = reinterpret_cast<float2*>(take(coarse_gpart_elems(B, m.L, sigma) * sizeof(float2)));
+        }
+        if (m.fwd2) w.Y2 = reinterpret_cast<float*>(take((size_t)B * R * D * sizeof(float)));
+        w.tc.part = reinterpret_cast<float*>(take((size_t)B * m.n_parts * m.L * 4));
+        if (!m.inv2) {      // the dense inverse (and, without the two-stage forward, the dense forward)
+            if (!m.fwd2 || !pl.coarse) {
+                w.tc.phi_hi = take(pl.phi_elems * 2);
+                w.tc.phi_lo = take(pl.phi_elems * 2);
+            }
+            if (pl.coarse) {
+                w.tc.phi2_hi = take(pl.phi2_elems * 2);
+                w.tc.phi2_lo = take(pl.phi2_elems * 2);
+                w.tw2 = reinterpret_cast<float2*>(take((size_t)pl.L * sizeof(float2)));
+            }
+            w.tc.yt_hi = take(pl.yt_elems * 2);
+            w.tc.yt_lo = take(pl.yt_elems * 2);
+        }
     }
+    if (total) *total = (size_t)(p - p0);
     return w;
 }
 
 }  // namespace
 
 size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype) {
-    const int R = 2 * sigma + 1, tiles = (D + BN - 1) / BN;
-    const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
-    size_t bytes = align_up((size_t)N * sizeof(float2)) + align_up((size_t)pl.r_pad * 4) + align_up((size_t)B * N * 4);
-    if (dtype == LUVC_F32)
-        bytes += align_up((size_t)B * R * D * 4) + align_up((size_t)B * tiles * N * 4);
-    else
-        bytes += 2 * align_up(pl.phi_elems * 2) + 2 * align_up(pl.phi2_elems * 2) +
-                 align_up((size_t)pl.L * sizeof(float2)) + align_up((size_t)B * pl.L * 4) +
-                 align_up(coarse_gpart_elems(B, pl.L, sigma) * sizeof(float2)) +
-                 align_up(fwd2_y_bytes(B, N, D, sigma)) + 2 * align_up(pl.yt_elems * 2) +
-                 align_up(pl.part_elems * 4);
-    return bytes;
+    size_t total = 0;
+    carve(nullptr, B, N, D, sigma, dtype != LUVC_F32, &total);
+    return total;
 }
 
 template <typename T>
@@ -410,31 +428,32 @@ static int spu_run_typed(const SpuProblem& p) {
     constexpr bool kTensor = sizeof(T) == 2;     // bf16 tokens go through the tensor cores
     const int N = p.N, D = p.D, B = p.B, sigma = p.sigma, R = 2 * sigma + 1;
     const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
-    Workspace ws = carve(p.workspace, B, N, D, sigma, kTensor);
+    Workspace ws = carve(p.workspace, B, N, D, sigma, kTensor, nullptr);
     float* E = p.out_scores ? p.out_scores : ws.E;
+    const Bf16Mode mode = kTensor ? bf16_mode(B, N, D, sigma) : Bf16Mode{};
     const int tab = max(max(N, pl.r_pad), pl.L);
     const long long bn = (long long)B * N;
     phase_begin(LUVC_PHASE_SPU_TRANSFORM, p.stream);
-    const bool coarse = kTensor && pl.coarse;
-    spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, coarse ? ws.tw2 : nullptr, ws.scale, N, pl.L, sigma,
-                                                               pl.r_pad, p.no_window);
+    spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, ws.tw2, ws.scale, N, pl.L, sigma, pl.r_pad,
+                                                               p.no_window);
     count_launch();
     if constexpr (kTensor) {
-        const bool two_stage = spu_fwd2_plan(B, N, D, sigma).ok;
-        if (two_stage) {
-            const int rc1 = spu_fwd2_run(p.hidden, ws.Y2, ws.scale, ws.tc.yt_hi, ws.tc.yt_lo, pl.r_pad, B, N, D, sigma,
-                                         p.status, p.stream);
+        if (mode.fwd2) {
+            const int rc1 = spu_fwd2_run(p.hidden, ws.Y2, ws.scale, mode.inv2 ? nullptr : ws.tc.yt_hi,
+                                         mode.inv2 ? nullptr : ws.tc.yt_lo, pl.r_pad, B, N, D, sigma, p.status, p.stream);
             if (rc1 != LUVC_OK) return rc1;
         }
-        const int rc = spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status, p.stream, two_stage);
+        const int rc = mode.inv2 ? spu_inv2_run(ws.Y2, ws.tc.part, B, N, D, sigma, p.status, p.stream)
+                                 : spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status,
+                                              p.stream, mode.fwd2);
         if (rc != LUVC_OK) return rc;
-        if (!coarse) {
-            spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, E, N, 2 * pl.tiles2, bn, 0);
+        if (!mode.coarse) {
+            spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, E, N, mode.n_parts, bn, 0);
             count_launch();
         } else {
-            const int L = pl.L, F = 2 * sigma, chunks = (L + kSpecChunk - 1) / kSpecChunk;
+            const int L = mode.L, F = 2 * sigma, chunks = (L + kSpecChunk - 1) / kSpecChunk;
             const long long bl = (long long)B * L;
-            spu_energy_kernel<<<(unsigned)((bl + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, ws.S, L, 2 * pl.tiles2, bl, 1);
+            spu_energy_kernel<<<(unsigned)((bl + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, ws.S, L, mode.n_parts, bl, 1);
             spu_coarse_spectrum_kernel<<<dim3((F + 128) / 128, chunks, B), 128, 0, p.stream>>>(ws.S, ws.gpart, L, F);
             spu_coarse_synthesis_kernel<<<dim3((N + 255) / 256, B), 256, 0, p.stream>>>(ws.gpart, E, N, L, F, chunks);
             count_launch(3);

@@ -94,11 +94,15 @@ __device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float2
                                             bool warp_active, uint32_t acc_empty_bar, int lane,
                                             float (&yA)[KB][CH][2], float (&yB)[KB][CH][2]) {
     constexpr int C = 8 * CH;
+    uint32_t v[2 * CH], vn[2 * CH];
+    tmem_load<2 * CH>(taddr, vn);
     for (int ql = 0; ql < nq; ++ql) {
-        uint32_t v[2 * CH];
-        tmem_load<2 * CH>(taddr + (uint32_t)(ql * C), v);
-        tmem_ld_wait();
-        if (ql == nq - 1) {          // this warp has read all it needs of the buffer
+        tmem_ld_wait_for(vn);
+#pragma unroll
+        for (int c = 0; c < 2 * CH; ++c) v[c] = vn[c];
+        if (ql + 1 < nq) {
+            tmem_load<2 * CH>(taddr + (uint32_t)((ql + 1) * C), vn);   // in flight under this token's arithmetic
+        } else {                     // this warp has read all it needs of the buffer
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty_bar);
