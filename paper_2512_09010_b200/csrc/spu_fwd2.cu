@@ -41,6 +41,8 @@ constexpr int kThreads = kEpiThreads;         // no producer warps: thread 0 als
 constexpr int kNmma = 256;                    // columns of a tile: QT tokens x C channels
 constexpr int kTmemCols = 512;                // two accumulator buffers
 constexpr int kSpin = 1 << 22;
+constexpr int kProducer = 96;                 // thread that issues TMA and MMA: lane 0 of a warp with the fewest bins
+constexpr int kStaticTabBytes = 24 * 1024;
 
 struct FwdArgs {
     const __nv_bfloat16* x;   // [B][N][D]
@@ -51,6 +53,7 @@ struct FwdArgs {
     int nblk;                 // copies of the P x P matrix on the diagonal of the 128-row operand: each
                               // serves its own block of channels of the same tokens (P <= 64)
     int n_ctiles, n_slices, n_items;
+    int static_tab;           // 1: the table of e^{-2 pi i q k2 / Q} for all q is built once per CTA (one slice only)
 };
 
 // barriers: 0,1 stage full | 2,3 accumulator full | 4,5 accumulator empty | 6,7 table ready
@@ -201,6 +204,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
         *reinterpret_cast<__nv_bfloat16*>(s_fhi + off) = h;
         *reinterpret_cast<__nv_bfloat16*>(s_flo + off) = l;
     }
+    if (a.static_tab)
+        for (int e = tid; e < Q * KB; e += kThreads) {
+            const int q = e / KB, k2 = e - q * KB;
+            s_tab[e] = root_neg(((unsigned)q * (unsigned)k2) % (unsigned)Q, Q);
+        }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -216,7 +224,10 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     for (int item = blockIdx.x; item < a.n_items; item += gridDim.x) ++n_my_items;
     const int total_tiles = n_my_items * tiles_per_item;
 
-    // producer steps (thread 0 only)
+    const uint64_t a_hi0 = make_desc(fhi, 2048, 128), a_lo0 = make_desc(flo, 2048, 128);
+    const uint64_t b0 = LAYOUT ? make_desc_layout(xs, P * ROWB, 8 * ROWB, LAYOUT) : make_desc(xs, 128, P * 16);
+
+    // producer steps (one thread only)
     auto issue_tma = [&](int v) {           // tile v of this CTA's sequence of tiles -> stage v & 1
         const int item = blockIdx.x + (v / tiles_per_item) * gridDim.x, tile = v % tiles_per_item;
         const int rest = item / a.n_slices;
@@ -232,19 +243,20 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
         if (!wait_bar(bar(kBarFull + buf), (v >> 1) & 1, fail, a.status)) return false;
         if (v >= 2 && !wait_bar(bar(kBarAccEmpty + buf), ((v - 2) >> 1) & 1, fail, a.status)) return false;
         tc_fence_after();
-        const uint32_t xb = xs + buf * stage_bytes, acc = tmem + (uint32_t)(buf * kNmma);
-        for (int ks = 0; ks < KT / 16; ++ks) {
-            // K rows 16 ks .. 16 ks + 15 lie in channel block jb (16 divides P)
-            const int jb = (ks * 16) / P, kl = ks * 16 - jb * P;
-            const uint32_t baddr = xb + jb * blk_bytes + kl * ROWB;
-            const uint64_t bd = LAYOUT ? make_desc_layout(baddr, P * ROWB, 8 * ROWB, LAYOUT) : make_desc(baddr, 128, P * 16);
-            umma_bf16(acc, make_desc(fhi + ks * 4096, 2048, 128), bd, idesc, ks ? 1u : 0u);
-            umma_bf16(acc, make_desc(flo + ks * 4096, 2048, 128), bd, idesc, 1u);
+        const uint32_t acc = tmem + (uint32_t)(buf * kNmma);
+        uint64_t ah = a_hi0, al = a_lo0;             // descriptors advance by adding to the address field
+        for (int jb = 0; jb < a.nblk; ++jb) {        // K rows of channel block jb
+            uint64_t bd = b0 + (uint64_t)((buf * stage_bytes + jb * blk_bytes) >> 4);
+            for (int kl = 0; kl < P / 16; ++kl) {
+                umma_bf16(acc, ah, bd, idesc, (jb | kl) ? 1u : 0u);
+                umma_bf16(acc, al, bd, idesc, 1u);
+                ah += 4096 >> 4; al += 4096 >> 4; bd += (16 * ROWB) >> 4;
+            }
         }
         umma_commit(bar(kBarAccFull + buf));
         return true;
     };
-    if (tid == 0) {
+    if (tid == kProducer) {
         issue_tma(0);
         if (total_tiles > 1) issue_tma(1);
         issue_mma(0);
@@ -285,16 +297,20 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
             for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
                 const int q0 = tile * QT, nq = min(QT, Q - q0), buf = u & 1, par = (u >> 1) & 1;
                 // table of e^{-2 pi i q k2 / Q} for the tile's tokens and the slice's k2
-                float2* tab = s_tab + buf * (QT * KB);
-                for (int e = tid; e < QT * KB; e += kEpiThreads) {
-                    const int ql = e / KB, k2 = k2_lo + (e - ql * KB);
-                    tab[e] = root_neg(((unsigned)(q0 + ql) * (unsigned)k2) % (unsigned)Q, Q);
+                const float2* tab = s_tab + q0 * KB;
+                if (!a.static_tab) {
+                    float2* tw = s_tab + buf * (QT * KB);
+                    for (int e = tid; e < QT * KB; e += kEpiThreads) {
+                        const int ql = e / KB, k2 = k2_lo + (e - ql * KB);
+                        tw[e] = root_neg(((unsigned)(q0 + ql) * (unsigned)k2) % (unsigned)Q, Q);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarTab + buf));
+                    ok = wait_bar(bar(kBarTab + buf), par, fail, a.status);
+                    tab = tw;
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarTab + buf));
-                ok = wait_bar(bar(kBarTab + buf), par, fail, a.status);
                 ok = wait_bar(bar(kBarAccFull + buf), par, fail, a.status) && ok;
-                if (tid == 0 && ok) {
+                if (tid == kProducer && ok) {
                     // the MMAs of tile u are done: refill their stage, and start tile u + 1
                     if (u + 2 < total_tiles) issue_tma(u + 2);
                     if (u + 1 < total_tiles) ok = issue_mma(u + 1);
@@ -406,7 +422,8 @@ cudaError_t launch_fwd2(const FwdArgs& a, const SpuFwd2Plan& pl, cudaStream_t st
                CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
-    const size_t smem = 1024 + (size_t)2 * KT * 256 + (size_t)2 * kNmma * KT * 2 + (size_t)2 * QT * KB * sizeof(float2);
+    const size_t tab_bytes = a.static_tab ? (size_t)a.Q * KB * sizeof(float2) : (size_t)2 * QT * KB * sizeof(float2);
+    const size_t smem = 1024 + (size_t)2 * KT * 256 + (size_t)2 * kNmma * KT * 2 + tab_bytes;
     static int sms = 0;
     if (!sms) {
         int dev = 0;
@@ -457,6 +474,7 @@ int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, 
     a.B = B; a.N = N; a.D = D; a.P = pl.P; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
     a.nblk = pl.nblk;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
+    a.static_tab = (pl.slices == 1 && (size_t)pl.Q * pl.KB * sizeof(float2) <= (size_t)kStaticTabBytes) ? 1 : 0;
     cudaError_t err;
     if (pl.KB == 2) err = launch_fwd2<2, 8>(a, pl, stream);
     else if (pl.KB == 4) err = launch_fwd2<4, 4>(a, pl, stream);

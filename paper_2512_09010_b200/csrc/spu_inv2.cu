@@ -206,7 +206,8 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     const int item_channels = a.nblk * C;
     const float2 step = root_pos((unsigned)k1 % (unsigned)L, L);
     const uint32_t idesc = make_idesc_bf16(128, kNcol, false, true);
-    const uint32_t fhi = smem_u32(s_fhi), flo = smem_u32(s_flo), bhi = smem_u32(s_bhi), blo = smem_u32(s_blo);
+    const uint64_t a_hi0 = make_desc(smem_u32(s_fhi), 2048, 128), a_lo0 = make_desc(smem_u32(s_flo), 2048, 128);
+    const uint64_t b_hi0 = make_desc(smem_u32(s_bhi), 128, kBSbo), b_lo0 = make_desc(smem_u32(s_blo), 128, kBSbo);
 
     // energies of tile `t` (accumulator t & 1) of the item (b, ctile), points jj0 ..: warps 0-3 only
     auto read_tile = [&](int t, int b, int ctile, int jj0) {
@@ -289,12 +290,12 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
                     tc_fence_after();
                     const uint32_t acc = tmem + (uint32_t)((t & 1) * kNcol);
                     const int ksteps = 2 * KT / 16;
+                    uint64_t ah = a_hi0, al = a_lo0, bh_d = b_hi0, bl_d = b_lo0;   // advance by adding to the address field
                     for (int ks = 0; ks < ksteps; ++ks) {
-                        const uint64_t ah = make_desc(fhi + ks * 4096, 2048, 128), al = make_desc(flo + ks * 4096, 2048, 128);
-                        const uint64_t bh_d = make_desc(bhi + ks * 256, 128, kBSbo), bl_d = make_desc(blo + ks * 256, 128, kBSbo);
                         umma_bf16(acc, ah, bh_d, idesc, ks ? 1u : 0u);
                         umma_bf16(acc, ah, bl_d, idesc, 1u);
                         umma_bf16(acc, al, bh_d, idesc, 1u);
+                        ah += 4096 >> 4; al += 4096 >> 4; bh_d += 256 >> 4; bl_d += 256 >> 4;
                     }
                     umma_commit(bar(kBarAccFull + (t & 1)));
                 }
