@@ -89,6 +89,17 @@ template <int NCOL> __device__ __forceinline__ void tmem_load(uint32_t addr, uin
     else tmem_ld16(addr, v);
 }
 
+template <int CH> __device__ __forceinline__ void store_row(float* dst, const float (&v)[CH]) {
+    if constexpr (CH >= 4) {
+#pragma unroll
+        for (int c = 0; c < CH; c += 4) *reinterpret_cast<float4*>(dst + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+    } else if constexpr (CH == 2) {
+        *reinterpret_cast<float2*>(dst) = make_float2(v[0], v[1]);
+    } else {
+        dst[0] = v[0];
+    }
+}
+
 // Stage 2 of one tile for one thread: NA / NB bins of the two frequency classes (compile time, so
 // that the loops carry no branches).  `tab` holds e^{-2 pi i q k2 / Q} for the tile's tokens.
 template <int KB, int CH, int NA, int NB>
@@ -345,13 +356,18 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                         const int k = kbase + P * (k2_lo + t);
                         const float cr = __ldg(a.scale + k);
                         float* yr = Yb + (size_t)k * D;
+                        float vr[CH], vi[CH];
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) yr[c] = cr * (cls == 0 ? yA[t][c][0] : yB[t][c][0]);
+                        for (int c = 0; c < CH; ++c) {
+                            vr[c] = cr * (cls == 0 ? yA[t][c][0] : yB[t][c][0]);
+                            vi[c] = cls == 0 ? yA[t][c][1] : yB[t][c][1];
+                        }
+                        store_row<CH>(yr, vr);           // ch0 is a multiple of CH: aligned vector stores
                         if (k >= 1) {
                             const float ci = __ldg(a.scale + sigma + k);
-                            float* yi = Yb + (size_t)(sigma + k) * D;
 #pragma unroll
-                            for (int c = 0; c < CH; ++c) yi[c] = ci * (cls == 0 ? yA[t][c][1] : yB[t][c][1]);
+                            for (int c = 0; c < CH; ++c) vi[c] *= ci;
+                            store_row<CH>(Yb + (size_t)(sigma + k) * D, vi);
                         }
                     }
                 }

@@ -243,11 +243,32 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
 #pragma unroll
         for (int q = 0; q < KB; ++q) {
             const int k = k1 + P * q;
-            const bool have = q < nA && ch0 < D;
+            const bool have = q < nA && ch0 < D;          // ch0 is a multiple of CHT and D of 8: all CHT channels exist
+            const float* yc = Yb + (size_t)k * D;
+            const float* ys = Yb + (size_t)(sigma + k) * D;
+            constexpr int VEC = CHT >= 4 ? 4 : 2;
 #pragma unroll
-            for (int c = 0; c < CHT; ++c) {
-                yv[q][c][0] = have ? __ldg(Yb + (size_t)k * D + c) : 0.f;
-                yv[q][c][1] = (have && k >= 1) ? __ldg(Yb + (size_t)(sigma + k) * D + c) : 0.f;
+            for (int c = 0; c < CHT; c += VEC) {
+                float vc[4] = {0.f, 0.f, 0.f, 0.f}, vs[4] = {0.f, 0.f, 0.f, 0.f};
+                if (have) {
+                    if constexpr (VEC == 4) {
+                        const float4 t4 = __ldg(reinterpret_cast<const float4*>(yc + c));
+                        vc[0] = t4.x; vc[1] = t4.y; vc[2] = t4.z; vc[3] = t4.w;
+                        if (k >= 1) {
+                            const float4 u4 = __ldg(reinterpret_cast<const float4*>(ys + c));
+                            vs[0] = u4.x; vs[1] = u4.y; vs[2] = u4.z; vs[3] = u4.w;
+                        }
+                    } else {
+                        const float2 t2 = __ldg(reinterpret_cast<const float2*>(yc + c));
+                        vc[0] = t2.x; vc[1] = t2.y;
+                        if (k >= 1) {
+                            const float2 u2 = __ldg(reinterpret_cast<const float2*>(ys + c));
+                            vs[0] = u2.x; vs[1] = u2.y;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) { yv[q][c + e][0] = vc[e]; yv[q][c + e][1] = vs[e]; }
             }
         }
         const int nA_w = __reduce_max_sync(0xffffffffu, nA);
