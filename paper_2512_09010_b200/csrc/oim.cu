@@ -199,8 +199,9 @@ __device__ bool wait_for_count(const int* ctr, int target, int* status) {
     return false;
 }
 
-template <typename T, int NCHUNK>
-__global__ void __launch_bounds__(kThreads, 3) oim_chain_kernel(const ChainArgs a) {
+// MINB: CTAs per SM the register budget is cut for (3: 80 registers, 4: 64 registers).
+template <typename T, int NCHUNK, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) oim_chain_kernel(const ChainArgs a) {
     constexpr int V = Elem<T>::kVec;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_item;
@@ -524,23 +525,33 @@ size_t oim_workspace_bytes(int B, int H, int W, int D, int /*dtype*/) {
            align_up(max_steps(H, W) * B * sizeof(int)) + 256;
 }
 
-template <typename T, int NCHUNK>
-static cudaError_t launch_chain(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
-    static int blocks_per_sm = 0, sms = 0;      // per kernel instantiation
+template <typename T, int NCHUNK, int MINB>
+static cudaError_t launch_chain_b(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
+    static int sms = 0;      // per kernel instantiation
+    int blocks_per_sm = 0;
     const size_t smem = (size_t)(3 * max_len + 2 * ((max_len + 1) / 2) + r + 8) * 4;
     if (smem > 48 * 1024)
-        cudaFuncSetAttribute(oim_chain_kernel<T, NCHUNK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaFuncSetAttribute(oim_chain_kernel<T, NCHUNK, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (!sms) {
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, oim_chain_kernel<T, NCHUNK>, kThreads, smem);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, oim_chain_kernel<T, NCHUNK, MINB>, kThreads, smem);
     if (blocks_per_sm < 1) blocks_per_sm = 1;
     int grid = blocks_per_sm * sms;
     if (grid > a.total_items) grid = a.total_items;
-    oim_chain_kernel<T, NCHUNK><<<grid, kThreads, smem, stream>>>(a);
+    oim_chain_kernel<T, NCHUNK, MINB><<<grid, kThreads, smem, stream>>>(a);
     return cudaGetLastError();
+}
+
+// Short lines leave a CTA mostly in its serial phases (ranking, merging, waiting for the image's
+// previous step): more resident CTAs overlap them.  Long lines are dominated by the streaming pass,
+// where the larger register budget wins.  The switch point is measured (36- vs 72-cell lines).
+template <typename T, int NCHUNK>
+static cudaError_t launch_chain(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
+    return max_len <= 48 ? launch_chain_b<T, NCHUNK, 4>(a, max_len, r, stream)
+                         : launch_chain_b<T, NCHUNK, 3>(a, max_len, r, stream);
 }
 
 template <typename T>
