@@ -339,45 +339,50 @@ __global__ void __launch_bounds__(kThreads, MINB) oim_chain_kernel(const ChainAr
             }
         }
 
-        // ---- merges: one warp per destination cell; its new sum is written as fp32
-        for (int k = warp; k < st.m; k += kWarps) {
-            const int pos = s_sel[k] >> 1, dst = pos + ((s_sel[k] & 1) ? 1 : -1);
-            bool first = true;          // the lowest rank that targets this destination does the work
-            int other = -1;             // a second source of the same destination, if any
-            for (int q = 0; q < st.m; ++q) {
-                if (q == k) continue;
-                const int qpos = s_sel[q] >> 1, qdst = qpos + ((s_sel[q] & 1) ? 1 : -1);
-                if (qdst == dst) { if (q < k) first = false; else other = qpos; }
-            }
-            if (!first) continue;
-            const unsigned rd = s_root[dst], ra = s_root[pos], rb = other >= 0 ? s_root[other] : 0u;
-            const size_t od = (size_t)(rd & ~kMergedBit) * D, oa = (size_t)(ra & ~kMergedBit) * D,
-                         ob = (size_t)(rb & ~kMergedBit) * D;
-            for (int e = lane * V; e < D; e += 32 * V) {
-                float x[V], y[V];
-                load_vec<T>(tokens + od, acc + od, rd & kMergedBit, e, x);
-                load_vec<T>(tokens + oa, acc + oa, ra & kMergedBit, e, y);
-#pragma unroll
-                for (int q = 0; q < V; ++q) x[q] += y[q];
-                if (other >= 0) {
-                    load_vec<T>(tokens + ob, acc + ob, rb & kMergedBit, e, y);
+        // ---- merges: the warps are dealt out over (destination cell, slice of D); new sums are written as fp32
+        {
+            const int m = st.m;
+            const int nsl = m < kWarps ? kWarps / m : 1;        // slices of D per merge
+            for (int idx = warp; idx < m * nsl; idx += kWarps) {
+                const int k = idx % m, sl = idx / m;
+                const int pos = s_sel[k] >> 1, dst = pos + ((s_sel[k] & 1) ? 1 : -1);
+                bool first = true;          // the lowest rank that targets this destination does the work
+                int other = -1;             // a second source of the same destination, if any
+                for (int q = 0; q < m; ++q) {
+                    if (q == k) continue;
+                    const int qpos = s_sel[q] >> 1, qdst = qpos + ((s_sel[q] & 1) ? 1 : -1);
+                    if (qdst == dst) { if (q < k) first = false; else other = qpos; }
+                }
+                if (!first) continue;
+                const unsigned rd = s_root[dst], ra = s_root[pos], rb = other >= 0 ? s_root[other] : 0u;
+                const size_t od = (size_t)(rd & ~kMergedBit) * D, oa = (size_t)(ra & ~kMergedBit) * D,
+                             ob = (size_t)(rb & ~kMergedBit) * D;
+                for (int e = (sl * 32 + lane) * V; e < D; e += nsl * 32 * V) {
+                    float x[V], y[V];
+                    load_vec<T>(tokens + od, acc + od, rd & kMergedBit, e, x);
+                    load_vec<T>(tokens + oa, acc + oa, ra & kMergedBit, e, y);
 #pragma unroll
                     for (int q = 0; q < V; ++q) x[q] += y[q];
-                }
+                    if (other >= 0) {
+                        load_vec<T>(tokens + ob, acc + ob, rb & kMergedBit, e, y);
 #pragma unroll
-                for (int q = 0; q < V; q += 4)
-                    *reinterpret_cast<float4*>(acc + od + e + q) = make_float4(x[q], x[q + 1], x[q + 2], x[q + 3]);
-            }
-            if (lane == 0) {
-                const int id = rd & ~kMergedBit, ia = ra & ~kMergedBit;
-                int s = __ldcg(size + id) + __ldcg(size + ia);
-                a.parent[img + ia] = id;
-                if (other >= 0) {
-                    const int ib = rb & ~kMergedBit;
-                    s += __ldcg(size + ib);
-                    a.parent[img + ib] = id;
+                        for (int q = 0; q < V; ++q) x[q] += y[q];
+                    }
+#pragma unroll
+                    for (int q = 0; q < V; q += 4)
+                        *reinterpret_cast<float4*>(acc + od + e + q) = make_float4(x[q], x[q + 1], x[q + 2], x[q + 3]);
                 }
-                size[id] = s;
+                if (sl == 0 && lane == 0) {
+                    const int id = rd & ~kMergedBit, ia = ra & ~kMergedBit;
+                    int sz = __ldcg(size + id) + __ldcg(size + ia);
+                    a.parent[img + ia] = id;
+                    if (other >= 0) {
+                        const int ib = rb & ~kMergedBit;
+                        sz += __ldcg(size + ib);
+                        a.parent[img + ib] = id;
+                    }
+                    size[id] = sz;
+                }
             }
         }
 
