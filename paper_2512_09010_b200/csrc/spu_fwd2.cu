@@ -305,6 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
 #pragma unroll
                 for (int c = 0; c < CH; ++c) { yA[t][c][0] = yA[t][c][1] = yB[t][c][0] = yB[t][c][1] = 0.f; }
 
+            float2 rotA = make_float2(1.f, 0.f), rotB = make_float2(1.f, 0.f);
             for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
                 const int q0 = tile * QT, nq = min(QT, Q - q0), buf = u & 1, par = (u >> 1) & 1;
                 // table of e^{-2 pi i q k2 / Q} for the tile's tokens and the slice's k2
@@ -329,8 +330,10 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                float2 rotA = root_neg(((unsigned)q0 * (unsigned)kA) % (unsigned)N, N);   // q0 kA < Q P = N
-                float2 rotB = root_neg(((unsigned)q0 * (unsigned)kB) % (unsigned)N, N);
+                if ((tile & 15) == 0) {     // exact restart of e^{-2 pi i q k / N}; in between it is carried along
+                    rotA = root_neg(((unsigned)q0 * (unsigned)kA) % (unsigned)N, N);   // q0 kA < Q P = N
+                    rotB = root_neg(((unsigned)q0 * (unsigned)kB) % (unsigned)N, N);
+                }
                 const uint32_t taddr = lane_addr + (uint32_t)(buf * kNmma + grp * 2 * CH);
                 const uint32_t eb = bar(kBarAccEmpty + buf);
                 if (nA_w == KB && nB_w == KB)
