@@ -35,7 +35,7 @@ constexpr int kSpin = 1 << 22;
 
 struct InvArgs {
     const float* Y;      // [B][R][D]
-    float* part;         // [B][n_ctiles * nblk][L]
+    float* part;         // [B][n_ctiles * nblk * (2 if C = 32)][L]
     int* status;
     int B, N, D, P, Q, sigma, R, nblk, J, L;
     int n_ctiles, n_items;
@@ -209,25 +209,32 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     const uint64_t a_hi0 = make_desc(smem_u32(s_fhi), 2048, 128), a_lo0 = make_desc(smem_u32(s_flo), 2048, 128);
     const uint64_t b_hi0 = make_desc(smem_u32(s_bhi), 128, kBSbo), b_lo0 = make_desc(smem_u32(s_blo), 128, kBSbo);
 
-    // energies of tile `t` (accumulator t & 1) of the item (b, ctile), points jj0 ..: warps 0-3 only
+    // energies of tile `t` (accumulator t & 1) of the item (b, ctile), points jj0 ..: the warp of channel
+    // group grp reads the 16 columns [16 grp, 16 grp + 16) of its rows with ONE TMEM load (a load's round
+    // trip is long, so the 64 columns are spread over the four warps that share the lanes):
+    //   C = 32: point jl = grp / 2, channel half grp % 2 (two partial sums per point)
+    //   C = 16: point jl = grp;   C = 8: points 2 grp and 2 grp + 1
+    constexpr int SPLIT = C == 32 ? 2 : 1;           // partial sums per (channel block, point)
     auto read_tile = [&](int t, int b, int ctile, int jj0) {
-        if (warp >= 4) return;
-        const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)((t & 1) * kNcol);
-        float* out = a.part + ((size_t)b * (a.n_ctiles * a.nblk) + ctile * a.nblk + jb) * L + (size_t)k1 * J;
-#pragma unroll 1
-        for (int jl = 0; jl < TJ; ++jl) {
-            float s = 0.f;
-#pragma unroll
-            for (int c0 = 0; c0 < C; c0 += 8) {
-                uint32_t v[8];
-                tmem_ld8(taddr + (uint32_t)(jl * C + c0), v);
-                tmem_ld_wait_for(v);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) { const float x = __uint_as_float(v[q]); s = fmaf(x, x, s); }
-            }
-            if (active && jj0 + jl < J) out[jj0 + jl] = s;
-        }
+        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((t & 1) * kNcol + grp * 16);
+        uint32_t v[16];
+        tmem_ld16(taddr, v);
+        tmem_ld_wait_for(v);
         tc_fence_before();
+        if (!active) return;
+        const int half = C == 32 ? (grp & 1) : 0;
+        float* out = a.part + ((size_t)b * (a.n_ctiles * a.nblk * SPLIT) + (ctile * a.nblk + jb) * SPLIT + half) * L +
+                     (size_t)k1 * J;
+        constexpr int PTS = C >= 16 ? 1 : 2;          // points among the 16 columns
+        constexpr int W = 16 / PTS;                   // columns per point
+#pragma unroll
+        for (int pt = 0; pt < PTS; ++pt) {
+            float sum = 0.f;
+#pragma unroll
+            for (int q = 0; q < W; ++q) { const float x = __uint_as_float(v[pt * W + q]); sum = fmaf(x, x, sum); }
+            const int jl = C == 32 ? (grp >> 1) : (C == 16 ? grp : 2 * grp + pt);
+            if (jj0 + jl < J) out[jj0 + jl] = sum;
+        }
     };
 
     int t = 0;                                       // tiles issued so far by this CTA
@@ -382,7 +389,7 @@ SpuInv2Plan spu_inv2_plan(int B, int N, int D, int sigma) {
     const long long items = (long long)B * pl.n_ctiles;
     if (items > 0x7fffffffll) return pl;
     pl.n_items = (int)items;
-    pl.n_parts = pl.n_ctiles * pl.nblk;
+    pl.n_parts = pl.n_ctiles * pl.nblk * (pl.CHT == 8 ? 2 : 1);
     pl.ok = 1;
     return pl;
 }
