@@ -100,56 +100,47 @@ template <int CH> __device__ __forceinline__ void store_row(float* dst, const fl
     }
 }
 
-// Stage 2 of one tile for one thread: NA / NB bins of the two frequency classes (compile time, so
-// that the loops carry no branches).  `tab` holds e^{-2 pi i q k2 / Q} for the tile's tokens.
-template <int KB, int CH, int NA, int NB>
-__device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float2* __restrict__ tab, float2& rotA,
-                                            float2& rotB, float2 stepA, float2 stepB, bool odd, bool special,
-                                            bool warp_active, uint32_t acc_empty_bar, int lane,
-                                            float (&yA)[KB][CH][2], float (&yB)[KB][CH][2]) {
-    constexpr int C = 8 * CH;
-    uint32_t v[2 * CH], vn[2 * CH];
-    tmem_load<2 * CH>(taddr, vn);
+// Stage 2 of one tile for one thread: NB bins (compile time, so that the loops carry no branches) of
+// the thread's frequency for the 2 CH channels of its warp.  The even lane of a pair owns the row
+// of real parts and the frequency k1, the odd lane the imaginary parts and the frequency P - k1,
+// whose stage-1 value is the conjugate: each sends its row to the other, and with e = own + i c other
+// the even lane holds A[k1] (c = 1) while the odd lane holds i conj(A[k1]) (c = 1), so the factor
+// -i is folded into its rotation; the pair of rows 0 / 1 holds the two real values A[0], A[P/2] (c = 0).
+// `tab` holds e^{-2 pi i q k2 / Q} for the tile's tokens.
+template <int KB, int CH, int NB>
+__device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float2* __restrict__ tab, float2& rot,
+                                            float2 step, float cg, bool warp_active, uint32_t acc_empty_bar,
+                                            int lane, float (&y)[KB][2 * CH][2]) {
+    constexpr int C = 8 * CH, W = 2 * CH;
+    uint32_t v[W], vn[W];
+    tmem_load<W>(taddr, vn);
     for (int ql = 0; ql < nq; ++ql) {
         tmem_ld_wait_for(vn);
 #pragma unroll
-        for (int c = 0; c < 2 * CH; ++c) v[c] = vn[c];
+        for (int c = 0; c < W; ++c) v[c] = vn[c];
         if (ql + 1 < nq) {
-            tmem_load<2 * CH>(taddr + (uint32_t)((ql + 1) * C), vn);   // in flight under this token's arithmetic
+            tmem_load<W>(taddr + (uint32_t)((ql + 1) * C), vn);   // in flight under this token's arithmetic
         } else {                     // this warp has read all it needs of the buffer
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty_bar);
         }
         if (!warp_active) continue;
-        float2 g[KB];
+        float2 g[NB];
 #pragma unroll
-        for (int t = 0; t < (NA > NB ? NA : NB); ++t) g[t] = tab[ql * KB + t];
+        for (int t = 0; t < NB; ++t) g[t] = tab[ql * KB + t];
 #pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            // the even lane owns the row of real parts, the odd lane the imaginary parts
-            const float mine = __uint_as_float(odd ? v[CH + c] : v[c]);
-            const float send = __uint_as_float(odd ? v[c] : v[CH + c]);
-            const float got = __shfl_xor_sync(0xffffffffu, send, 1);
-            const float re = odd ? got : mine, im = odd ? mine : got;
-            // class A uses A[k1], class B its conjugate; the pair of rows 0 / 1 holds the two real
-            // values A[0] and A[P/2]
-            const float2 zA = make_float2(re, special ? 0.f : im);
-            const float2 zB = make_float2(special ? im : re, special ? 0.f : -im);
-            const float2 wA = cmul(rotA, zA), wB = cmul(rotB, zB);
-#pragma unroll
-            for (int t = 0; t < NA; ++t) {
-                yA[t][c][0] = fmaf(g[t].x, wA.x, fmaf(-g[t].y, wA.y, yA[t][c][0]));
-                yA[t][c][1] = fmaf(g[t].x, wA.y, fmaf(g[t].y, wA.x, yA[t][c][1]));
-            }
+        for (int c = 0; c < W; ++c) {
+            const float own = __uint_as_float(v[c]);
+            const float other = cg * __shfl_xor_sync(0xffffffffu, own, 1);
+            const float2 w = cmul(rot, make_float2(own, other));
 #pragma unroll
             for (int t = 0; t < NB; ++t) {
-                yB[t][c][0] = fmaf(g[t].x, wB.x, fmaf(-g[t].y, wB.y, yB[t][c][0]));
-                yB[t][c][1] = fmaf(g[t].x, wB.y, fmaf(g[t].y, wB.x, yB[t][c][1]));
+                y[t][c][0] = fmaf(g[t].x, w.x, fmaf(-g[t].y, w.y, y[t][c][0]));
+                y[t][c][1] = fmaf(g[t].x, w.y, fmaf(g[t].y, w.x, y[t][c][1]));
             }
         }
-        rotA = cmul(rotA, stepA);
-        rotB = cmul(rotB, stepB);
+        rot = cmul(rot, step);
     }
 }
 
@@ -283,9 +274,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
         const int i = jr >> 1;
         const bool odd = jr & 1, special = i == 0;
         const bool warp_active = quarter * 32 < KT;
-        const int kA = special ? 0 : i, kB = special ? P / 2 : P - i;
-        const int my_c = jb * C + grp * 2 * CH + (odd ? CH : 0);   // first of this thread's channels in the item
-        const float2 stepA = root_neg(kA % N, N), stepB = root_neg(kB % N, N);
+        // this lane's frequency: k1 = i on the even lane, P - i on the odd lane (0 and P/2 for the first pair)
+        const int kf = special ? (odd ? P / 2 : 0) : (odd ? P - i : i);
+        const float cg = special ? 0.f : 1.f;
+        const int my_c = jb * C + grp * 2 * CH;                    // first of this thread's channels in the item
+        const float2 step = root_neg(kf % N, N);
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         int u = 0;
         bool ok = true;
@@ -293,19 +286,17 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
             const int slice = item % a.n_slices, rest = item / a.n_slices;
             const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
             const int k2_lo = slice * KB;
-            // bins of this thread in this slice: k = kA + P (k2_lo + t) <= sigma, likewise kB
-            int nA = (active && kA <= sigma) ? (sigma - kA) / P + 1 - k2_lo : 0;
-            int nB = (active && kB <= sigma) ? (sigma - kB) / P + 1 - k2_lo : 0;
-            nA = max(0, min(KB, nA));
-            nB = max(0, min(KB, nB));
-            const int nA_w = __reduce_max_sync(0xffffffffu, nA), nB_w = __reduce_max_sync(0xffffffffu, nB);
-            float yA[KB][CH][2], yB[KB][CH][2];
+            // bins of this thread in this slice: k = kf + P (k2_lo + t) <= sigma
+            int nb = (active && kf <= sigma) ? (sigma - kf) / P + 1 - k2_lo : 0;
+            nb = max(0, min(KB, nb));
+            const int nb_w = __reduce_max_sync(0xffffffffu, nb);
+            float y[KB][2 * CH][2];
 #pragma unroll
             for (int t = 0; t < KB; ++t)
 #pragma unroll
-                for (int c = 0; c < CH; ++c) { yA[t][c][0] = yA[t][c][1] = yB[t][c][0] = yB[t][c][1] = 0.f; }
+                for (int c = 0; c < 2 * CH; ++c) y[t][c][0] = y[t][c][1] = 0.f;
 
-            float2 rotA = make_float2(1.f, 0.f), rotB = make_float2(1.f, 0.f);
+            float2 rot = make_float2(1.f, 0.f);
             for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
                 const int q0 = tile * QT, nq = min(QT, Q - q0), buf = u & 1, par = (u >> 1) & 1;
                 // table of e^{-2 pi i q k2 / Q} for the tile's tokens and the slice's k2
@@ -331,47 +322,40 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                 if (!ok) break;
                 tc_fence_after();
                 if ((tile & 15) == 0) {     // exact restart of e^{-2 pi i q k / N}; in between it is carried along
-                    rotA = root_neg(((unsigned)q0 * (unsigned)kA) % (unsigned)N, N);   // q0 kA < Q P = N
-                    rotB = root_neg(((unsigned)q0 * (unsigned)kB) % (unsigned)N, N);
+                    rot = root_neg(((unsigned)q0 * (unsigned)kf) % (unsigned)N, N);   // q0 kf < Q P = N
+                    if (odd && !special) rot = make_float2(rot.y, -rot.x);           // times -i (see stage2_tile)
                 }
                 const uint32_t taddr = lane_addr + (uint32_t)(buf * kNmma + grp * 2 * CH);
                 const uint32_t eb = bar(kBarAccEmpty + buf);
-                if (nA_w == KB && nB_w == KB)
-                    stage2_tile<KB, CH, KB, KB>(taddr, nq, tab, rotA, rotB, stepA, stepB, odd, special, warp_active, eb, lane, yA, yB);
-                else if (nA_w == KB && nB_w == KB - 1)
-                    stage2_tile<KB, CH, KB, KB - 1>(taddr, nq, tab, rotA, rotB, stepA, stepB, odd, special, warp_active, eb, lane, yA, yB);
-                else if (nA_w <= KB - 1 && nB_w <= KB - 1)
-                    stage2_tile<KB, CH, KB - 1, KB - 1>(taddr, nq, tab, rotA, rotB, stepA, stepB, odd, special, warp_active, eb, lane, yA, yB);
+                if (nb_w == KB)
+                    stage2_tile<KB, CH, KB>(taddr, nq, tab, rot, step, cg, warp_active, eb, lane, y);
+                else if (nb_w == KB - 1 || KB == 2)
+                    stage2_tile<KB, CH, (KB > 1 ? KB - 1 : 1)>(taddr, nq, tab, rot, step, cg, warp_active, eb, lane, y);
+                else if (KB >= 4 && nb_w <= KB / 2)
+                    stage2_tile<KB, CH, (KB >= 4 ? KB / 2 : KB)>(taddr, nq, tab, rot, step, cg, warp_active, eb, lane, y);
                 else
-                    stage2_tile<KB, CH, KB, KB>(taddr, nq, tab, rotA, rotB, stepA, stepB, odd, special, warp_active, eb, lane, yA, yB);
+                    stage2_tile<KB, CH, KB>(taddr, nq, tab, rot, step, cg, warp_active, eb, lane, y);
             }
             if (!ok) break;
             // band spectrum of this thread's channels: cos row k, sin row sigma + k
             const int ch0 = ctile * item_channels + my_c;
             if (active && ch0 < D) {
                 float* Yb = a.Y + (size_t)b * a.R * D + ch0;
+                const bool second = ch0 + CH < D;      // D is a multiple of 8 and ch0 of CH: each half is whole or absent
 #pragma unroll
-                for (int cls = 0; cls < 2; ++cls) {
-                    const int kbase = cls == 0 ? kA : kB, cnt = cls == 0 ? nA : nB;
+                for (int t = 0; t < KB; ++t) {
+                    if (t >= nb) continue;
+                    const int k = kf + P * (k2_lo + t);
+                    const float cr = __ldg(a.scale + k);
+                    const float ci = k >= 1 ? __ldg(a.scale + sigma + k) : 0.f;
 #pragma unroll
-                    for (int t = 0; t < KB; ++t) {
-                        if (t >= cnt) continue;
-                        const int k = kbase + P * (k2_lo + t);
-                        const float cr = __ldg(a.scale + k);
-                        float* yr = Yb + (size_t)k * D;
+                    for (int h = 0; h < 2; ++h) {
+                        if (h == 1 && !second) continue;
                         float vr[CH], vi[CH];
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) {
-                            vr[c] = cr * (cls == 0 ? yA[t][c][0] : yB[t][c][0]);
-                            vi[c] = cls == 0 ? yA[t][c][1] : yB[t][c][1];
-                        }
-                        store_row<CH>(yr, vr);           // ch0 is a multiple of CH: aligned vector stores
-                        if (k >= 1) {
-                            const float ci = __ldg(a.scale + sigma + k);
-#pragma unroll
-                            for (int c = 0; c < CH; ++c) vi[c] *= ci;
-                            store_row<CH>(Yb + (size_t)(sigma + k) * D, vi);
-                        }
+                        for (int c = 0; c < CH; ++c) { vr[c] = cr * y[t][h * CH + c][0]; vi[c] = ci * y[t][h * CH + c][1]; }
+                        store_row<CH>(Yb + (size_t)k * D + h * CH, vr);          // aligned vector stores
+                        if (k >= 1) store_row<CH>(Yb + (size_t)(sigma + k) * D + h * CH, vi);
                     }
                 }
             }
