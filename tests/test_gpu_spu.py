@@ -52,6 +52,26 @@ def test_small_sequences_match_the_oracle(luvc, oracle_mod, dtype, B, N, D, keep
     _check(luvc, oracle_mod, x, keep, cutoff, method="naive" if N <= 130 else "fft")
 
 
+@pytest.mark.parametrize("B,N,D,keep,cutoff", [
+    (2, 112, 40, 30, 0.5),      # N = 16 x 7: eight channel blocks on the diagonal of the stage-1 operand
+    (1, 592, 24, 100, 1.0),     # N = 16 x 37, full band: two bin slices forward, dense inverse
+    (2, 592, 16, 50, 0.3),      # same N, narrower band: two-stage inverse with 9 bins per row
+    (1, 2048, 72, 500, 1.0),    # P = 128, sigma = N/2: 9 bins per class, inverse on the tokens themselves
+    (2, 2048, 40, 300, 0.5),    # inverse not coarse (4 sigma + 2 > 3N/4)
+    (1, 4096, 16, 1000, 0.9),   # 17 bins per class, one channel per thread
+    (2, 1296, 136, 324, 0.125), # P = 48, Q = 27: ragged last tile, partial channel block
+    (1, 2592, 264, 648, 0.05),  # P = 96
+    (3, 768, 8, 77, 0.02),      # sigma smaller than P: most rows hold no bin
+])
+def test_two_stage_paths_match_the_oracle(luvc, oracle_mod, B, N, D, keep, cutoff):
+    g = torch.Generator().manual_seed(N * 7 + D)
+    x = torch.randn((B, N, D), generator=g).to(torch.bfloat16)
+    # add a smooth component so that the band is not pure noise
+    n = torch.arange(N, dtype=torch.float32)[None, :, None]
+    x = (x.float() + 2.0 * torch.cos(2 * np.pi * 3 * n / N + torch.arange(D)[None, None, :])).to(torch.bfloat16)
+    _check(luvc, oracle_mod, x, keep, cutoff)
+
+
 def test_flat_pass_band_option(luvc, oracle_mod):
     g = torch.Generator().manual_seed(3)
     x = torch.randn((2, 48, 16), generator=g)
