@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(kThreads, MINB) oim_chain_kernel(const ChainAr
 
         const int ncand = (len + 1) >> 1;
         float* s_dot = reinterpret_cast<float*>(smem_raw);          // <v_j, v_{j+1}>
-        float* s_nrm = s_dot + len;                                  // |v_j|^2
+        float* s_nrm = s_dot + len;                                  // 1 / |v_j| (0 for a zero vector)
         float* s_score = s_nrm + len;                                // best cosine of even cell 2c
         unsigned* s_root = reinterpret_cast<unsigned*>(s_score + ncand);   // root | merged bit
         int* s_dir = reinterpret_cast<int*>(s_root + len);           // best direction of even cell 2c
@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, MINB) oim_chain_kernel(const ChainAr
                                   has_next, lane, D, nn, dd);
             nn = warp_sum(nn);
             dd = warp_sum(dd);
-            if (lane == 0) { s_nrm[j] = nn; s_dot[j] = dd; }
+            if (lane == 0) { s_nrm[j] = nn > 0.f ? 1.0f / sqrtf(nn) : 0.f; s_dot[j] = dd; }
         }
         __syncthreads();
 
@@ -277,16 +277,14 @@ __global__ void __launch_bounds__(kThreads, MINB) oim_chain_kernel(const ChainAr
         if (warp == 0) {
             for (int c = lane; c < ncand; c += 32) {
                 const int j = 2 * c;
-                const float nj = sqrtf(s_nrm[j]);
+                const float ij = s_nrm[j];                       // a zero vector has similarity 0 with everything
                 float cl = -FLT_MAX, cr = -FLT_MAX;
                 if (j >= 1) {
-                    const float nb = sqrtf(s_nrm[j - 1]);
-                    cl = (nj == 0.f || nb == 0.f) ? 0.f : s_dot[j - 1] / (nj * nb);
+                    cl = s_dot[j - 1] * (ij * s_nrm[j - 1]);
                     if (!(cl == cl)) cl = -FLT_MAX;
                 }
                 if (j + 1 < len) {
-                    const float nb = sqrtf(s_nrm[j + 1]);
-                    cr = (nj == 0.f || nb == 0.f) ? 0.f : s_dot[j] / (nj * nb);
+                    cr = s_dot[j] * (ij * s_nrm[j + 1]);
                     if (!(cr == cr)) cr = -FLT_MAX;
                 }
                 const bool right = (j < 1) || (j + 1 < len && cr > cl);   // ties stay with the previous cell
