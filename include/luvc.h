@@ -128,6 +128,8 @@ typedef struct {
                                 (position of the merged cell in its line) * 2 + direction
                                 (0 = into the previous cell of the line, 1 = into the next),
                                 ordered by step, line, rank of the candidate */
+    float* out_log_sizes;    /* optional device [B, target_count] fp32: log(s), the bias that the
+                                value enhancement of Eq. 2 adds to the values (V + log s) */
 } luvc_oim_opts;
 
 /*
@@ -164,6 +166,16 @@ int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target
  * before returning.  dtype is a luvc_dtype. */
 int luvc_oim_merge_host(const void* tokens, int B, int H, int W, int D, int target_count, int dtype,
                         void* out_tokens, int32_t* out_sizes, int32_t* out_map);
+
+/*
+ * Value enhancement of Eq. 2, O = A (V + log s): out[b, t, :] = values[b, t, :] + log(sizes[b, t]),
+ * the row-wise bias that lets attention weigh a merged token by the number of tokens it stands for
+ * (the attention itself is the caller's).  values / out [B, T, D] of element type `dtype` (DEVICE,
+ * out may be the same buffer as values), sizes [B, T] int32 (the out_sizes of luvc_oim_merge*).
+ * The sum is formed in fp32 and rounded once.  cuda_stream: a cudaStream_t, NULL = legacy default.
+ */
+int luvc_oim_value_enhance(const void* values, const int32_t* sizes, int B, int T, int D, int dtype,
+                           void* out, void* cuda_stream);
 
 /* ---- SPU ---------------------------------------------------------------- */
 

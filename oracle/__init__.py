@@ -127,6 +127,13 @@ def oim(tokens, target=None, out_hw=None, r=2, height_first=False, trace=None, t
                 grid=(Hf, Wf), threads=min(nt, B))
 
 
+def oim_value_enhance(values, sizes):
+    """Eq. 2's enhanced values V + log s, in double: values [B,T,D], sizes [B,T]."""
+    v = np.asarray(values, dtype=np.float64)
+    s = np.asarray(sizes, dtype=np.float64)
+    return v + np.log(s)[..., None]
+
+
 # --------------------------------------------------------------------------- SPU
 
 

@@ -28,7 +28,7 @@ EXPORTS = (
     "luvc_version", "luvc_status_string", "luvc_set_stream", "luvc_shutdown", "luvc_kernel_launches",
     "luvc_profile_enable", "luvc_profile_read", "luvc_check_status",
     "luvc_oim_plan", "luvc_oim_workspace_bytes", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
-    "luvc_oim_merge_host", "luvc_spu_sigma", "luvc_spu_workspace_bytes", "luvc_spu_prune",
+    "luvc_oim_merge_host", "luvc_oim_value_enhance", "luvc_spu_sigma", "luvc_spu_workspace_bytes", "luvc_spu_prune",
     "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host", "luvc_spu_prune_static",
 )
 
@@ -45,6 +45,7 @@ class OimOpts(ctypes.Structure):
         ("dtype", ctypes.c_int), ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("out_h", ctypes.c_int), ("out_w", ctypes.c_int),
         ("merge_per_step", ctypes.c_int), ("height_first", ctypes.c_int), ("trace", ctypes.c_void_p),
+        ("out_log_sizes", ctypes.c_void_p),
     ]
 
 
@@ -80,6 +81,7 @@ def _load() -> ctypes.CDLL:
     L.luvc_oim_merge_f32.argtypes = [p, i, i, i, i, i, p, p, p]
     L.luvc_oim_merge_ex.argtypes = [p, i, i, i, i, i, p, p, p, ctypes.POINTER(OimOpts)]
     L.luvc_oim_merge_host.argtypes = [p, i, i, i, i, i, i, p, p, p]
+    L.luvc_oim_value_enhance.argtypes = [p, p, i, i, i, i, p, p]
     L.luvc_spu_sigma.argtypes = [i, f]
     L.luvc_spu_workspace_bytes.restype = sz
     L.luvc_spu_workspace_bytes.argtypes = [i, i, i, f, i]
@@ -155,7 +157,8 @@ def spu_sigma(N: int, cutoff: float = 0.0) -> int:
 
 
 def oim_merge(tokens: torch.Tensor, target_count: int, *, out_hw=None, merge_per_step: int = 0,
-              height_first: bool = False, want_trace: bool = False, workspace: torch.Tensor | None = None):
+              height_first: bool = False, want_trace: bool = False, workspace: torch.Tensor | None = None,
+              want_log_sizes: bool = False):
     """luvc_oim_merge_ex on a CUDA tensor [B,H,W,D]; returns (out_tokens [B,T,D], out_sizes [B,T] int32,
     out_map [B,H*W] int32) and, with want_trace, the per-merge decision log [B,H*W-T] int32."""
     if not tokens.is_cuda:
@@ -179,11 +182,30 @@ def oim_merge(tokens: torch.Tensor, target_count: int, *, out_hw=None, merge_per
         o.merge_per_step = int(merge_per_step)
         o.height_first = int(bool(height_first))
         o.trace = trace.data_ptr() if (trace is not None and trace.numel()) else None
+        log_sizes = torch.empty((B, max(T, 0)), dtype=torch.float32, device=dev) if want_log_sizes else None
+        o.out_log_sizes = log_sizes.data_ptr() if log_sizes is not None else None
         _check(lib.luvc_oim_merge_ex(tokens.data_ptr(), B, H, W, D, T, out_tokens.data_ptr(), out_sizes.data_ptr(),
                                      out_map.data_ptr(), ctypes.byref(o)), "luvc_oim_merge_ex")
+    res = (out_tokens, out_sizes, out_map)
     if want_trace:
-        return out_tokens, out_sizes, out_map, trace
-    return out_tokens, out_sizes, out_map
+        res = res + (trace,)
+    if want_log_sizes:
+        res = res + (log_sizes,)
+    return res
+
+
+def oim_value_enhance(values: torch.Tensor, sizes: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """luvc_oim_value_enhance: values [B,T,D] + log(sizes [B,T]) per row (Eq. 2); `out` may be `values`."""
+    values = values.contiguous()
+    sizes = sizes.contiguous()
+    B, T, D = values.shape
+    dev = values.device
+    if out is None:
+        out = torch.empty_like(values)
+    with torch.cuda.device(dev):
+        _check(lib.luvc_oim_value_enhance(values.data_ptr(), sizes.data_ptr(), B, T, D, _dtype_code(values),
+                                          out.data_ptr(), _stream_ptr(dev)), "luvc_oim_value_enhance")
+    return out
 
 
 def oim_merge_plain(tokens: torch.Tensor, target_count: int):

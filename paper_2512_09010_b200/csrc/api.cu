@@ -219,6 +219,7 @@ int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target
     p.height_first = opts->height_first ? 1 : 0;
     p.dtype = opts->dtype;
     p.out_tokens = out_tokens; p.out_sizes = out_sizes; p.out_map = out_map; p.trace = opts->trace;
+    p.out_log_sizes = opts->out_log_sizes;
     p.workspace = ws; p.stream = static_cast<cudaStream_t>(opts->stream);
     p.status = status_word();
     if (!p.status) return LUVC_ERR_CUDA;
@@ -263,6 +264,17 @@ int luvc_oim_merge_host(const void* tokens, int B, int H, int W, int D, int targ
     cudaMemcpyAsync(out_sizes, dsz, (size_t)B * target_count * 4, cudaMemcpyDeviceToHost, st);
     cudaMemcpyAsync(out_map, dmap, (size_t)B * hw * 4, cudaMemcpyDeviceToHost, st);
     return cudaStreamSynchronize(st) == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
+}
+
+int luvc_oim_value_enhance(const void* values, const int32_t* sizes, int B, int T, int D, int dtype, void* out,
+                           void* cuda_stream) {
+    if (!values || !sizes || !out) return LUVC_ERR_NULL;
+    if (dtype != LUVC_BF16 && dtype != LUVC_F32) return LUVC_ERR_DTYPE;
+    if (B < 1 || T < 1 || D < 1 || (long long)B * T > (1ll << 31) - 1) return LUVC_ERR_SHAPE;
+    if (((size_t)D * elem_size(dtype)) % 16 != 0 || !aligned16(values) || !aligned16(out) ||
+        (reinterpret_cast<uintptr_t>(sizes) & 3u))
+        return LUVC_ERR_ALIGN;
+    return oim_value_enhance(values, sizes, (long long)B * T, D, dtype, out, static_cast<cudaStream_t>(cuda_stream));
 }
 
 // ---- SPU ---------------------------------------------------------------------

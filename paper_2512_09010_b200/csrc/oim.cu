@@ -398,8 +398,8 @@ __global__ void __launch_bounds__(kThreads, MINB) oim_chain_kernel(const ChainAr
 template <typename T>
 __global__ void __launch_bounds__(256) oim_emit_kernel(const void* tokens_v, const float* acc, const int32_t* cell,
                                                        const int32_t* size, int32_t* cellpos, void* out_v,
-                                                       int32_t* out_sizes, int HW, int target, int D,
-                                                       long long total_cells) {
+                                                       int32_t* out_sizes, float* out_log_sizes, int HW, int target,
+                                                       int D, long long total_cells) {
     constexpr int V = Elem<T>::kVec;
     const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -411,7 +411,11 @@ __global__ void __launch_bounds__(256) oim_emit_kernel(const void* tokens_v, con
     const T* tok = reinterpret_cast<const T*>(tokens_v) + (img + root) * D;
     const float* arow = acc + (img + root) * D;
     T* out = reinterpret_cast<T*>(out_v) + ((size_t)b * target + c) * D;
-    if (lane == 0) { out_sizes[(size_t)b * target + c] = s; cellpos[img + root] = c; }
+    if (lane == 0) {
+        out_sizes[(size_t)b * target + c] = s;
+        cellpos[img + root] = c;
+        if (out_log_sizes != nullptr) out_log_sizes[(size_t)b * target + c] = logf((float)s);   // Eq. 2's log s
+    }
     if (s == 1) {
         for (int e = lane * V; e < D; e += 32 * V)
             *reinterpret_cast<uint4*>(out + e) = __ldg(reinterpret_cast<const uint4*>(tok + e));
@@ -605,11 +609,56 @@ static int oim_run_typed(const OimProblem& p) {
     const int32_t* final_cell = (n_steps & 1) ? ws.cell_b : ws.cell_a;
     const long long cells = (long long)p.B * target;
     oim_emit_kernel<T><<<(unsigned)((cells * 32 + 255) / 256), 256, 0, p.stream>>>(
-        p.tokens, ws.acc, final_cell, ws.size, ws.cellpos, p.out_tokens, p.out_sizes, HW, target, p.D, cells);
+        p.tokens, ws.acc, final_cell, ws.size, ws.cellpos, p.out_tokens, p.out_sizes, p.out_log_sizes, HW, target, p.D,
+        cells);
     count_launch();
     oim_map_kernel<<<(unsigned)((n + 255) / 256), 256, 0, p.stream>>>(ws.parent, ws.cellpos, p.out_map, HW, n);
     count_launch();
     phase_end(LUVC_PHASE_OIM_TOTAL, p.stream);
+    return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
+}
+
+// Value enhancement of Eq. 2: one warp per token row, 16 bytes per lane per trip.
+template <typename T>
+__global__ void __launch_bounds__(256) oim_value_enhance_kernel(const T* __restrict__ v, const int32_t* __restrict__ sizes,
+                                                                T* __restrict__ out, long long rows, int D) {
+    constexpr int V = 16 / sizeof(T);
+    const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const float bias = logf((float)sizes[row]);
+    const T* src = v + row * D;
+    T* dst = out + row * D;
+    for (int e = lane * V; e < D; e += 32 * V) {
+        if constexpr (sizeof(T) == 4) {
+            float4 f = *reinterpret_cast<const float4*>(src + e);
+            f.x += bias; f.y += bias; f.z += bias; f.w += bias;
+            *reinterpret_cast<float4*>(dst + e) = f;
+        } else {
+            const uint4 u = *reinterpret_cast<const uint4*>(src + e);
+            const unsigned w[4] = {u.x, u.y, u.z, u.w};
+            unsigned r[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const __nv_bfloat162 pr = __floats2bfloat162_rn(__uint_as_float(w[q] << 16) + bias,
+                                                                __uint_as_float(w[q] & 0xffff0000u) + bias);
+                r[q] = *reinterpret_cast<const unsigned*>(&pr);
+            }
+            *reinterpret_cast<uint4*>(dst + e) = make_uint4(r[0], r[1], r[2], r[3]);
+        }
+    }
+}
+
+int oim_value_enhance(const void* values, const int32_t* sizes, long long rows, int D, int dtype, void* out,
+                      cudaStream_t stream) {
+    const unsigned grid = (unsigned)((rows * 32 + 255) / 256);
+    if (dtype == LUVC_F32)
+        oim_value_enhance_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(values), sizes,
+                                                                  static_cast<float*>(out), rows, D);
+    else
+        oim_value_enhance_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(values), sizes,
+                                                                          static_cast<__nv_bfloat16*>(out), rows, D);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
 

@@ -126,3 +126,21 @@ def test_host_buffer_entry_point(luvc, oracle_mod):
     luvc.oim_merge_host(x, 16, tok, sizes, mp)
     ref = luvc.oim_merge(x.cuda(), 16)
     assert torch.equal(tok, ref[0].cpu()) and torch.equal(sizes, ref[1].cpu()) and torch.equal(mp, ref[2].cpu())
+
+
+def test_value_enhancement_bias(luvc, oracle_mod):
+    # Eq. 2: V + log s.  log s as an optional output of the merge, and the row-wise add as its own call
+    g = torch.Generator().manual_seed(11)
+    for dtype in (torch.float32, torch.bfloat16):
+        x = torch.randn((2, 10, 10, 64), generator=g).to(dtype).cuda()
+        tok, sizes, mp, logs = luvc.oim_merge(x, 25, want_log_sizes=True)
+        np.testing.assert_allclose(logs.cpu().numpy(), np.log(sizes.cpu().numpy().astype(np.float64)), rtol=2e-7, atol=1e-7)
+        assert sizes.max().item() > 1
+        enhanced = luvc.oim_value_enhance(tok, sizes)
+        ref = oracle_mod.oim_value_enhance(tok.float().cpu().numpy(), sizes.cpu().numpy())
+        from _compare import assert_values_close
+        assert_values_close(enhanced.float().cpu().numpy(), ref, _name(x), "enhanced values")
+        # in place
+        tok2 = tok.clone()
+        luvc.oim_value_enhance(tok2, sizes, out=tok2)
+        assert torch.equal(tok2, enhanced)

@@ -238,3 +238,13 @@ def test_config0_shapes_and_near_ties(oracle_mod):
     # smooth high-dimensional fields make near-ties common: the reason the GPU comparison
     # replays decisions instead of demanding an identical map everywhere
     assert r["stats"][0, 0] < 1e-3
+
+
+def test_value_enhancement_is_the_log_of_the_size(oracle_mod):
+    # Eq. 2 with uniform attention over n tokens: a token of size s with bias log s weighs like s unit tokens
+    v = np.array([[[1.0, 2.0], [3.0, 5.0]]])
+    s = np.array([[1, 4]])
+    e = oracle_mod.oim_value_enhance(v, s)
+    np.testing.assert_allclose(e[0, 0], v[0, 0])                      # log 1 = 0
+    np.testing.assert_allclose(e[0, 1] - v[0, 1], np.log(4.0))
+    np.testing.assert_allclose(np.exp(e - v)[0, :, 0], s[0])          # the bias exponentiates back to the size
