@@ -225,6 +225,23 @@ int luvc_spu_prune_ex(const void* hidden, int B, int N, int D, float cutoff, int
 int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, int keep, int dtype,
                         int32_t* out_idx, void* out_hidden);
 
+/*
+ * Cascade of prunes (Section 3.3: the unit is applied again every few layers, each time to the
+ * visual tokens that are left; appendix "Hyper-parameters of SPU": start layer and interval).
+ * Runs n_stages prunes back to back: stage t keeps keeps[t] of the keeps[t-1] survivors (N for
+ * t = 0) with cutoffs[t] (cutoffs == NULL or an entry <= 0: the default).  What the LLM does to the
+ * hidden states between two stages is the caller's business and not modelled: every stage sees
+ * the rows of `hidden`.
+ *
+ * keeps, cutoffs  HOST arrays of n_stages entries; 1 <= keeps[t] <= keeps[t-1] <= N
+ * out_idx     [B, keeps[n_stages-1]] int32  surviving tokens as indices into the ORIGINAL sequence, ascending
+ * out_hidden  [B, keeps[n_stages-1], D]     their rows, bit-exact copies
+ * Intermediate survivors live in library-owned scratch (grown with cudaMalloc on demand).
+ * Dropping the last survivors altogether, as the paper does at the final layer, needs no kernel.
+ */
+int luvc_spu_cascade(const void* hidden, int B, int N, int D, int n_stages, const int* keeps, const float* cutoffs,
+                     int dtype, void* cuda_stream, int32_t* out_idx, void* out_hidden);
+
 /* ---- SPU without any allocation ------------------------------------------- */
 
 /* Largest workspace (luvc_spu_workspace_bytes) luvc_spu_prune_static accepts: 32 MiB. */

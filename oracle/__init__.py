@@ -208,3 +208,19 @@ def spu(hidden, cutoff=None, keep=None, hamming=True, method="fft", nthreads=Non
     idx = np.stack([spu_select(scores[b], keep) for b in range(B)])
     kept = np.stack([x[b][idx[b]] for b in range(B)])
     return dict(scores=scores, idx=idx, hidden=kept, sigma=sigma)
+
+
+def spu_cascade(hidden, keeps, cutoffs=None, hamming=True):
+    """Section 3.3's progressive pruning as a plain loop: stage t applies Algorithm 2 to the survivors of
+    stage t-1.  Returns per stage the scores and kept indices (in that stage's coordinates) and, at the
+    end, the survivors as indices into the original sequence and their rows."""
+    x = _f32(hidden)
+    B = x.shape[0]
+    total = np.tile(np.arange(x.shape[1], dtype=np.int32), (B, 1))
+    stages = []
+    for t, keep in enumerate(keeps):
+        r = spu(x, cutoff=None if cutoffs is None else cutoffs[t], keep=int(keep), hamming=hamming)
+        stages.append(r)
+        total = np.stack([total[b][r["idx"][b]] for b in range(B)])
+        x = r["hidden"]
+    return dict(idx=total, hidden=x, stages=stages)

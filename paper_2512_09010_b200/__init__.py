@@ -29,7 +29,7 @@ EXPORTS = (
     "luvc_profile_enable", "luvc_profile_read", "luvc_check_status",
     "luvc_oim_plan", "luvc_oim_workspace_bytes", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
     "luvc_oim_merge_host", "luvc_oim_value_enhance", "luvc_spu_sigma", "luvc_spu_workspace_bytes", "luvc_spu_prune",
-    "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host", "luvc_spu_prune_static",
+    "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host", "luvc_spu_prune_static", "luvc_spu_cascade",
 )
 
 
@@ -90,6 +90,7 @@ def _load() -> ctypes.CDLL:
     L.luvc_spu_prune_ex.argtypes = [p, i, i, i, f, i, p, p, ctypes.POINTER(SpuOpts)]
     L.luvc_spu_prune_host.argtypes = [p, i, i, i, f, i, i, p, p]
     L.luvc_spu_prune_static.argtypes = [p, i, i, i, f, i, i, p, p, p]
+    L.luvc_spu_cascade.argtypes = [p, i, i, i, i, ctypes.POINTER(i), ctypes.POINTER(f), i, p, p, p]
     return L
 
 
@@ -265,6 +266,23 @@ def spu_prune_plain(hidden: torch.Tensor, keep: int, cutoff: float = 0.0):
         fn = lib.luvc_spu_prune if _dtype_code(hidden) == BF16 else lib.luvc_spu_prune_f32
         _check(fn(hidden.data_ptr(), B, N, D, float(cutoff), int(keep), out_idx.data_ptr(), out_hidden.data_ptr()),
                "luvc_spu_prune")
+    return out_idx, out_hidden
+
+
+def spu_cascade(hidden: torch.Tensor, keeps, cutoffs=None):
+    """luvc_spu_cascade: prunes back to back, stage t on the survivors of stage t-1.  Returns
+    (out_idx [B, keeps[-1]] int32 into the original sequence, out_hidden [B, keeps[-1], D])."""
+    hidden = hidden.contiguous()
+    B, N, D = hidden.shape
+    dev = hidden.device
+    n = len(keeps)
+    k_arr = (ctypes.c_int * n)(*[int(k) for k in keeps])
+    c_arr = (ctypes.c_float * n)(*[float(c) for c in cutoffs]) if cutoffs is not None else None
+    with torch.cuda.device(dev):
+        out_idx = torch.empty((B, int(keeps[-1])), dtype=torch.int32, device=dev)
+        out_hidden = torch.empty((B, int(keeps[-1]), D), dtype=hidden.dtype, device=dev)
+        _check(lib.luvc_spu_cascade(hidden.data_ptr(), B, N, D, n, k_arr, c_arr, _dtype_code(hidden), _stream_ptr(dev),
+                                    out_idx.data_ptr(), out_hidden.data_ptr()), "luvc_spu_cascade")
     return out_idx, out_hidden
 
 

@@ -42,7 +42,7 @@ thread_local cudaStream_t t_stream = nullptr;
 // Library-owned scratch: one growing buffer per purpose, shared by all threads.
 // Calls that use it from several host threads at once must use different streams'
 // work serially; the plain entry points take this lock only while (re)allocating.
-enum Slot { kOimWs = 0, kSpuWs, kIoIn, kIoOut, kStatus, kSlots };
+enum Slot { kOimWs = 0, kSpuWs, kIoIn, kIoOut, kStatus, kCascade, kSlots };
 struct Scratch { void* ptr = nullptr; size_t bytes = 0; };
 Scratch g_scratch[kSlots];
 std::mutex g_mutex;
@@ -327,6 +327,45 @@ int luvc_spu_prune_f32(const float* hidden, int B, int N, int D, float cutoff, i
     luvc_spu_opts o = {};
     o.dtype = LUVC_F32; o.stream = t_stream;
     return luvc_spu_prune_ex(hidden, B, N, D, cutoff, keep, out_idx, out_hidden, &o);
+}
+
+int luvc_spu_cascade(const void* hidden, int B, int N, int D, int n_stages, const int* keeps, const float* cutoffs,
+                     int dtype, void* cuda_stream, int32_t* out_idx, void* out_hidden) {
+    if (!hidden || !keeps || !out_idx || !out_hidden) return LUVC_ERR_NULL;
+    if (dtype != LUVC_BF16 && dtype != LUVC_F32) return LUVC_ERR_DTYPE;
+    if (B < 1 || N < 1 || D < 1 || n_stages < 1) return LUVC_ERR_SHAPE;
+    int prev = N;
+    for (int t = 0; t < n_stages; ++t) {
+        if (keeps[t] < 1 || keeps[t] > prev) return LUVC_ERR_KEEP;
+        if (cutoffs && (cutoffs[t] != cutoffs[t] || cutoffs[t] > 1.0f)) return LUVC_ERR_CUTOFF;
+        prev = keeps[t];
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    luvc_spu_opts o = {};
+    o.dtype = dtype; o.stream = cuda_stream;
+    if (n_stages == 1) return luvc_spu_prune_ex(hidden, B, N, D, cutoffs ? cutoffs[0] : 0.f, keeps[0], out_idx, out_hidden, &o);
+    // scratch: two buffers of survivors' rows (ping-pong) and three index arrays (stage, total so far, new total)
+    const size_t es = elem_size(dtype);
+    const size_t rows = align_up((size_t)B * keeps[0] * D * es), idxb = align_up((size_t)B * keeps[0] * 4);
+    unsigned char* sc = static_cast<unsigned char*>(scratch(kCascade, 2 * rows + 3 * idxb));
+    if (!sc) return LUVC_ERR_CUDA;
+    void* buf[2] = {sc, sc + rows};
+    int32_t* idx_stage = reinterpret_cast<int32_t*>(sc + 2 * rows);
+    int32_t* idx_tot[2] = {reinterpret_cast<int32_t*>(sc + 2 * rows + idxb), reinterpret_cast<int32_t*>(sc + 2 * rows + 2 * idxb)};
+    const void* in = hidden;
+    int n_in = N;
+    for (int t = 0; t < n_stages; ++t) {
+        const bool last = t == n_stages - 1;
+        void* out_rows = last ? out_hidden : buf[t & 1];
+        int rc = luvc_spu_prune_ex(in, B, n_in, D, cutoffs ? cutoffs[t] : 0.f, keeps[t], idx_stage, out_rows, &o);
+        if (rc) return rc;
+        int32_t* tot = last ? out_idx : idx_tot[t & 1];
+        rc = spu_compose_indices(t == 0 ? nullptr : idx_tot[(t - 1) & 1], idx_stage, tot, B, t == 0 ? 0 : keeps[t - 1], keeps[t], st);
+        if (rc) return rc;
+        in = out_rows;
+        n_in = keeps[t];
+    }
+    return LUVC_OK;
 }
 
 int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, int keep, int dtype,

@@ -63,6 +63,9 @@ struct SpuProblem {
 };
 size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype);
 int spu_run(const SpuProblem& p);
+// out[b][j] = prev[b][cur[b][j]] (prev == nullptr: out = cur)
+int spu_compose_indices(const int32_t* prev, const int32_t* cur, int32_t* out, int B, int n_prev, int keep,
+                        cudaStream_t stream);
 
 // Tensor-core contraction of the bf16 path (spu_tc.cu).
 struct SpuTcPlan {

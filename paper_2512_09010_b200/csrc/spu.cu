@@ -480,6 +480,23 @@ static int spu_run_typed(const SpuProblem& p) {
     return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
 
+__global__ void spu_compose_kernel(const int32_t* __restrict__ prev, const int32_t* __restrict__ cur,
+                                   int32_t* __restrict__ out, int n_prev, int keep, long long total) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int b = (int)(i / keep);
+    const int c = cur[i];
+    out[i] = prev ? prev[(size_t)b * n_prev + c] : c;
+}
+
+int spu_compose_indices(const int32_t* prev, const int32_t* cur, int32_t* out, int B, int n_prev, int keep,
+                        cudaStream_t stream) {
+    const long long total = (long long)B * keep;
+    spu_compose_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(prev, cur, out, n_prev, keep, total);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
+}
+
 int spu_run(const SpuProblem& p) {
     return p.dtype == LUVC_F32 ? spu_run_typed<float>(p) : spu_run_typed<__nv_bfloat16>(p);
 }

@@ -157,3 +157,34 @@ def test_stress_configuration_sampled(luvc, oracle_mod):
             assert len(idx_h[b]) == keep and np.all(np.diff(idx_h[b]) > 0)
             assert sc_h[b][kept].min() >= sc_h[b][~kept].max()
             assert torch.equal(hid[b], x[b][idx[b].long()])
+
+
+def test_cascade_entry_point(luvc, oracle_mod):
+    # luvc_spu_cascade against the same stages composed by hand, and against the oracle's loop where
+    # every stage of the oracle has a unique answer
+    g = torch.Generator().manual_seed(21)
+    for dtype, shape, keeps, cutoffs in ((torch.bfloat16, (2, 1296, 136), (324, 130, 65), None),
+                                         (torch.float32, (1, 200, 64), (120, 60, 7), (0.3, 0.0, 1.0)),
+                                         (torch.bfloat16, (3, 96, 72), (40,), (0.25,))):
+        x = torch.randn(shape, generator=g).to(dtype)
+        idx, hid = luvc.spu_cascade(x.cuda(), keeps, cutoffs)
+        torch.cuda.synchronize()
+        cur, tot = x.cuda(), None
+        for t, k in enumerate(keeps):
+            i_t, cur = luvc.spu_prune(cur, k, 0.0 if cutoffs is None else cutoffs[t])
+            tot = i_t.long() if tot is None else torch.gather(tot, 1, i_t.long())
+        assert torch.equal(idx.long(), tot) and torch.equal(hid, cur)
+        assert torch.equal(hid.cpu(), torch.stack([x[b][idx[b].long().cpu()] for b in range(shape[0])]))
+        assert bool((idx[:, 1:] > idx[:, :-1]).all())
+        ref = oracle_mod.spu_cascade(x.float().numpy(), keeps, cutoffs)
+        unique = True
+        for r, k in zip(ref["stages"], keeps):
+            for b in range(shape[0]):
+                order = np.sort(r["scores"][b])[::-1]
+                if k < len(order) and not order[k - 1] > order[k] * (1 + 1e-4):
+                    unique = False
+        if unique:
+            np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
+    with pytest.raises(luvc.LuvcError) as e:
+        luvc.spu_cascade(torch.zeros((1, 16, 8), dtype=torch.bfloat16).cuda(), (8, 9))
+    assert e.value.status == 4

@@ -174,3 +174,14 @@ def test_spu_end_to_end_gathers_original_rows(oracle_mod):
     for b in range(2):
         assert np.all(np.diff(r["idx"][b]) > 0)
         np.testing.assert_array_equal(r["hidden"][b], x[b][r["idx"][b]])   # the unfiltered tokens
+
+
+def test_cascade_is_the_composition_of_single_prunes(oracle_mod):
+    x = _signal(60, 6, 9)[None]
+    r = oracle_mod.spu_cascade(x, (30, 12, 5), (0.5, 0.25, 1.0))
+    a = oracle_mod.spu(x, cutoff=0.5, keep=30)
+    b = oracle_mod.spu(a["hidden"], cutoff=0.25, keep=12)
+    c = oracle_mod.spu(b["hidden"], cutoff=1.0, keep=5)
+    np.testing.assert_array_equal(r["idx"][0], a["idx"][0][b["idx"][0]][c["idx"][0]])
+    np.testing.assert_array_equal(r["hidden"], x[:, r["idx"][0]])
+    assert np.all(np.diff(r["idx"][0]) > 0)                      # the original order survives every stage
