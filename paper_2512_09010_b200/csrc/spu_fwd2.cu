@@ -81,6 +81,12 @@ __device__ __forceinline__ float2 root_neg(unsigned num, unsigned den) {
     sincospif(2.0f * (float)num / (float)den, &s, &c);
     return make_float2(c, -s);
 }
+// A table entry g = e^{-2 pi i num / den} in the form the packed complex multiply-add wants:
+// (g.x, g.x, -g.y, g.y), so that y += g w is two packed FMAs, (g.x, g.x) * (w.x, w.y) and (-g.y, g.y) * (w.y, w.x).
+__device__ __forceinline__ float4 root_neg_packed(unsigned num, unsigned den) {
+    const float2 g = root_neg(num, den);
+    return make_float4(g.x, g.x, -g.y, g.y);
+}
 
 template <int NCOL> __device__ __forceinline__ void tmem_load(uint32_t addr, uint32_t (&v)[NCOL]) {
     if constexpr (NCOL == 2) tmem_ld2(addr, v);
@@ -108,9 +114,9 @@ template <int CH> __device__ __forceinline__ void store_row(float* dst, const fl
 // -i is folded into its rotation; the pair of rows 0 / 1 holds the two real values A[0], A[P/2] (c = 0).
 // `tab` holds e^{-2 pi i q k2 / Q} for the tile's tokens.
 template <int KB, int CH, int NB>
-__device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float2* __restrict__ tab, float2& rot,
+__device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float4* __restrict__ tab, float2& rot,
                                             float2 step, float cg, bool warp_active, uint32_t acc_empty_bar,
-                                            int lane, float (&y)[KB][2 * CH][2]) {
+                                            int lane, float2 (&y)[KB][2 * CH]) {
     constexpr int C = 8 * CH, W = 2 * CH;
     uint32_t v[W], vn[W];
     tmem_load<W>(taddr, vn);
@@ -126,18 +132,42 @@ __device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float2
             if (lane == 0) mbar_arrive(acc_empty_bar);
         }
         if (!warp_active) continue;
-        float2 g[NB];
+        // packed fp32 arithmetic (two FMAs per instruction): a complex product a b is
+        // (a.x, a.x) * (b.x, b.y) + (-a.y, a.y) * (b.y, b.x)
+        const float2 rxx = make_float2(rot.x, rot.x), ryy = make_float2(-rot.y, rot.y);
+        if constexpr (NB <= 6) {            // few bins: the table row stays in registers across the channels
+            float4 g[NB];
 #pragma unroll
-        for (int t = 0; t < NB; ++t) g[t] = tab[ql * KB + t];
+            for (int t = 0; t < NB; ++t) g[t] = tab[ql * KB + t];
 #pragma unroll
-        for (int c = 0; c < W; ++c) {
-            const float own = __uint_as_float(v[c]);
-            const float other = cg * __shfl_xor_sync(0xffffffffu, own, 1);
-            const float2 w = cmul(rot, make_float2(own, other));
+            for (int c = 0; c < W; ++c) {
+                const float own = __uint_as_float(v[c]);
+                const float other = cg * __shfl_xor_sync(0xffffffffu, own, 1);
+                const float2 w = __ffma2_rn(rxx, make_float2(own, other), __fmul2_rn(ryy, make_float2(other, own)));
+                const float2 ws = make_float2(w.y, w.x);
+#pragma unroll
+                for (int t = 0; t < NB; ++t) {
+                    y[t][c] = __ffma2_rn(make_float2(g[t].x, g[t].y), w, y[t][c]);
+                    y[t][c] = __ffma2_rn(make_float2(g[t].z, g[t].w), ws, y[t][c]);
+                }
+            }
+        } else {                            // many bins, few channels: the rotated values stay, the table streams
+            float2 w[W], ws[W];
+#pragma unroll
+            for (int c = 0; c < W; ++c) {
+                const float own = __uint_as_float(v[c]);
+                const float other = cg * __shfl_xor_sync(0xffffffffu, own, 1);
+                w[c] = __ffma2_rn(rxx, make_float2(own, other), __fmul2_rn(ryy, make_float2(other, own)));
+                ws[c] = make_float2(w[c].y, w[c].x);
+            }
 #pragma unroll
             for (int t = 0; t < NB; ++t) {
-                y[t][c][0] = fmaf(g[t].x, w.x, fmaf(-g[t].y, w.y, y[t][c][0]));
-                y[t][c][1] = fmaf(g[t].x, w.y, fmaf(g[t].y, w.x, y[t][c][1]));
+                const float4 g = tab[ql * KB + t];
+#pragma unroll
+                for (int c = 0; c < W; ++c) {
+                    y[t][c] = __ffma2_rn(make_float2(g.x, g.y), w[c], y[t][c]);
+                    y[t][c] = __ffma2_rn(make_float2(g.z, g.w), ws[c], y[t][c]);
+                }
             }
         }
         rot = cmul(rot, step);
@@ -168,7 +198,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     unsigned char* s_fhi = smem;
     unsigned char* s_flo = smem + f_bytes;
     unsigned char* s_x = smem + 2 * f_bytes;
-    float2* s_tab = reinterpret_cast<float2*>(s_x + 2 * stage_bytes);   // [2][QT * KB]
+    float4* s_tab = reinterpret_cast<float4*>(s_x + 2 * stage_bytes);   // [Q * KB] or [2][QT * KB]
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -209,7 +239,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     if (a.static_tab)
         for (int e = tid; e < Q * KB; e += kThreads) {
             const int q = e / KB, k2 = e - q * KB;
-            s_tab[e] = root_neg(((unsigned)q * (unsigned)k2) % (unsigned)Q, Q);
+            s_tab[e] = root_neg_packed(((unsigned)q * (unsigned)k2) % (unsigned)Q, Q);
         }
     fence_proxy_async();
     tc_fence_before();
@@ -290,22 +320,22 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
             int nb = (active && kf <= sigma) ? (sigma - kf) / P + 1 - k2_lo : 0;
             nb = max(0, min(KB, nb));
             const int nb_w = __reduce_max_sync(0xffffffffu, nb);
-            float y[KB][2 * CH][2];
+            float2 y[KB][2 * CH];
 #pragma unroll
             for (int t = 0; t < KB; ++t)
 #pragma unroll
-                for (int c = 0; c < 2 * CH; ++c) y[t][c][0] = y[t][c][1] = 0.f;
+                for (int c = 0; c < 2 * CH; ++c) y[t][c] = make_float2(0.f, 0.f);
 
             float2 rot = make_float2(1.f, 0.f);
             for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
                 const int q0 = tile * QT, nq = min(QT, Q - q0), buf = u & 1, par = (u >> 1) & 1;
                 // table of e^{-2 pi i q k2 / Q} for the tile's tokens and the slice's k2
-                const float2* tab = s_tab + q0 * KB;
+                const float4* tab = s_tab + q0 * KB;
                 if (!a.static_tab) {
-                    float2* tw = s_tab + buf * (QT * KB);
+                    float4* tw = s_tab + buf * (QT * KB);
                     for (int e = tid; e < QT * KB; e += kEpiThreads) {
                         const int ql = e / KB, k2 = k2_lo + (e - ql * KB);
-                        tw[e] = root_neg(((unsigned)(q0 + ql) * (unsigned)k2) % (unsigned)Q, Q);
+                        tw[e] = root_neg_packed(((unsigned)(q0 + ql) * (unsigned)k2) % (unsigned)Q, Q);
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kBarTab + buf));
@@ -353,7 +383,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                         if (h == 1 && !second) continue;
                         float vr[CH], vi[CH];
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) { vr[c] = cr * y[t][h * CH + c][0]; vi[c] = ci * y[t][h * CH + c][1]; }
+                        for (int c = 0; c < CH; ++c) { vr[c] = cr * y[t][h * CH + c].x; vi[c] = ci * y[t][h * CH + c].y; }
                         store_row<CH>(Yb + (size_t)k * D + h * CH, vr);          // aligned vector stores
                         if (k >= 1) store_row<CH>(Yb + (size_t)(sigma + k) * D + h * CH, vi);
                     }
@@ -425,7 +455,7 @@ cudaError_t launch_fwd2(const FwdArgs& a, const SpuFwd2Plan& pl, cudaStream_t st
                CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
-    const size_t tab_bytes = a.static_tab ? (size_t)a.Q * KB * sizeof(float2) : (size_t)2 * QT * KB * sizeof(float2);
+    const size_t tab_bytes = a.static_tab ? (size_t)a.Q * KB * sizeof(float4) : (size_t)2 * QT * KB * sizeof(float4);
     const size_t smem = 1024 + (size_t)2 * KT * 256 + (size_t)2 * kNmma * KT * 2 + tab_bytes;
     static int sms = 0;
     if (!sms) {
@@ -477,7 +507,7 @@ int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, 
     a.B = B; a.N = N; a.D = D; a.P = pl.P; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
     a.nblk = pl.nblk;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
-    a.static_tab = (pl.slices == 1 && (size_t)pl.Q * pl.KB * sizeof(float2) <= (size_t)kStaticTabBytes) ? 1 : 0;
+    a.static_tab = (pl.slices == 1 && (size_t)pl.Q * pl.KB * sizeof(float4) <= (size_t)kStaticTabBytes) ? 1 : 0;
     cudaError_t err;
     if (pl.KB == 2) err = launch_fwd2<2, 8>(a, pl, stream);
     else if (pl.KB == 4) err = launch_fwd2<4, 4>(a, pl, stream);
