@@ -202,15 +202,17 @@ __global__ void __launch_bounds__(128) spu_coarse_spectrum_kernel(const float* _
     gpart[((size_t)b * gridDim.y + chunk) * (F + 1) + f] = make_float2(gr, gi);
 }
 
-// E[b][n] = sqrt(max(0, S(n))), the coefficient partials summed in chunk order.
+// E[b][n] = sqrt(max(0, S(n))), the coefficient partials summed in chunk order.  A thread forms
+// A = sum g.x cos and B = sum g.y sin once and writes two tokens: S(n) = A - B, S(N - n) = A + B.
 constexpr int kSynthTile = 2048;   // coefficients staged in shared memory at a time
 __global__ void __launch_bounds__(256) spu_coarse_synthesis_kernel(const float2* __restrict__ gpart, float* __restrict__ E,
                                                                    int N, int L, int F, int chunks) {
     __shared__ float2 s_g[kSynthTile];
     const int b = blockIdx.y, n = blockIdx.x * 256 + threadIdx.x;
+    const bool live = n <= N / 2;
     const float inv_l = 1.0f / (float)L;
-    const float2 step = unit_root(n < N ? n : 0, N);
-    float acc = 0.f;
+    const float2 step = unit_root(live ? n : 0, N);
+    float sa = 0.f, sb = 0.f;
     for (int f0 = 0; f0 <= F; f0 += kSynthTile) {
         const int cnt = min(kSynthTile, F + 1 - f0);
         __syncthreads();
@@ -224,20 +226,23 @@ __global__ void __launch_bounds__(256) spu_coarse_synthesis_kernel(const float2*
             s_g[i] = make_float2(gr * m, gi * m);
         }
         __syncthreads();
-        if (n < N) {
+        if (live) {
             float2 w = make_float2(1.f, 0.f);
             for (int i = 0; i < cnt; ++i) {
                 if ((i % kReseed) == 0) w = unit_root((long long)(f0 + i) * n, N);
                 const float2 g = s_g[i];
-                acc = fmaf(g.x, w.x, acc);
-                acc = fmaf(-g.y, w.y, acc);
+                sa = fmaf(g.x, w.x, sa);
+                sb = fmaf(g.y, w.y, sb);
                 const float nx = w.x * step.x - w.y * step.y;
                 w.y = fmaf(w.x, step.y, w.y * step.x);
                 w.x = nx;
             }
         }
     }
-    if (n < N) E[(size_t)b * N + n] = sqrtf(fmaxf(acc, 0.f));
+    if (live) {
+        E[(size_t)b * N + n] = sqrtf(fmaxf(sa - sb, 0.f));
+        if (n > 0 && n < N - n) E[(size_t)b * N + (N - n)] = sqrtf(fmaxf(sa + sb, 0.f));
+    }
 }
 
 // ---- order-preserving top-k ---------------------------------------------------
@@ -455,7 +460,7 @@ static int spu_run_typed(const SpuProblem& p) {
             const long long bl = (long long)B * L;
             spu_energy_kernel<<<(unsigned)((bl + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, ws.S, L, mode.n_parts, bl, 1);
             spu_coarse_spectrum_kernel<<<dim3((F + 128) / 128, chunks, B), 128, 0, p.stream>>>(ws.S, ws.gpart, L, F);
-            spu_coarse_synthesis_kernel<<<dim3((N + 255) / 256, B), 256, 0, p.stream>>>(ws.gpart, E, N, L, F, chunks);
+            spu_coarse_synthesis_kernel<<<dim3((N / 2 + 256) / 256, B), 256, 0, p.stream>>>(ws.gpart, E, N, L, F, chunks);
             count_launch(3);
         }
     } else {

@@ -82,3 +82,22 @@ def test_argument_errors_are_reported_before_any_device_work(luvc):
     assert L.luvc_spu_prune_ex(fake, 1, 8, 4, 0.5, 2, fake, fake, ctypes.byref(s)) == 6             # 8-byte rows
     assert L.luvc_oim_workspace_bytes(1, 24, 24, 1024, 0) >= 576 * 1024 * 4
     assert L.luvc_spu_workspace_bytes(1, 144, 4096, 0.0, 0) > 0
+
+
+def test_argument_errors_of_the_added_entry_points(luvc):
+    L = luvc.lib
+    fake = ctypes.c_void_p(4096)
+    assert L.luvc_oim_value_enhance(None, fake, 1, 4, 8, 0, fake, None) == 1
+    assert L.luvc_oim_value_enhance(fake, fake, 0, 4, 8, 0, fake, None) == 2
+    assert L.luvc_oim_value_enhance(fake, fake, 1, 4, 12, 0, fake, None) == 6          # 24-byte rows
+    assert L.luvc_oim_value_enhance(fake, fake, 1, 4, 8, 3, fake, None) == 7
+    keeps = (ctypes.c_int * 2)(8, 9)
+    assert L.luvc_spu_cascade(fake, 1, 16, 8, 2, keeps, None, 0, None, fake, fake) == 4  # stage 2 keeps more than stage 1
+    keeps = (ctypes.c_int * 2)(8, 4)
+    cut = (ctypes.c_float * 2)(0.5, 2.0)
+    assert L.luvc_spu_cascade(fake, 1, 16, 8, 2, keeps, cut, 0, None, fake, fake) == 5
+    assert L.luvc_spu_cascade(fake, 1, 16, 8, 0, keeps, None, 0, None, fake, fake) == 2
+    assert L.luvc_spu_cascade(None, 1, 16, 8, 2, keeps, None, 0, None, fake, fake) == 1
+    # the allocation-free prune checks its size limit before it touches the device
+    assert L.luvc_spu_prune_static(fake, 8, 16384, 4096, 0.0, 4, 0, None, fake, fake) == 8
+    assert L.luvc_spu_prune_static(fake, 1, 16, 8, 0.0, 17, 0, None, fake, fake) == 4
