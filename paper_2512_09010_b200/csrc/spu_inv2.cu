@@ -6,14 +6,19 @@
 // uniform points t = p Q + jj Q / J of the period (J = Q: the tokens themselves; J < Q: the coarse
 // grid from which the squared energies are interpolated).  With k = k1 + P k2:
 //   stage 2'  C_jj[k1] = e^{2 pi i k1 jj / L} sum_{k2} Y_{k1 + P k2} e^{2 pi i k2 jj / J}     CUDA cores
-//   stage 1'  x'[p, jj] = sum_{k1} cos(2 pi k1 p / P) Re C_jj[k1] - sin(2 pi k1 p / P) Im C_jj[k1]
-//             one tcgen05 contraction per tile: A = [cos | -sin] (128 x 2P, bf16 pair, built once per
-//             CTA), B = [Re C ; Im C] for a tile of 64 columns (points x channels), written to shared
-//             memory as a bf16 pair by the threads that computed it (three products: hi*hi, hi*lo, lo*hi)
-//   energy    S[p J + jj] += sum over the tile's channels of x'^2, read back from TMEM.
-// The thread that owns row k1 keeps the band bins Y_{k1 + P k2} of its channels in registers for
-// the whole work item (sequence x channel tile).  As in the forward kernel, P <= 64 puts 128 / P
-// channel blocks on the diagonal of the 128-row operand.  Every mbarrier wait is bounded.
+//   stage 1'  x'[p, jj] = sum_{k1 < P} Re(e^{2 pi i k1 p / P} C_jj[k1])
+//                       = sum_r F[r][p] G_jj[r],  the real P x P matrix of the forward kernel with
+//             G[0] = Re C[0], G[1] = Re C[P/2], G[2i] = Re C[i] + Re C[P-i], G[2i+1] = Im C[i] - Im C[P-i]
+//             one tcgen05 contraction per tile: A = F transposed (bf16 pair, built once per CTA),
+//             B = G for a tile of 64 columns (points x channels), written to shared memory as a bf16
+//             pair by the threads that computed it (three products: hi*hi, hi*lo, lo*hi); B and the
+//             accumulator are double buffered, so the MMAs of a tile run under the arithmetic of the next
+//   energy    S[p J + jj] = sum over the tile's channels of x'^2, read back from TMEM.
+// As in the forward kernel the even lane of a pair owns the frequency k1 = i and row 2i, the odd lane
+// P - i and row 2i + 1 (they swap one value per column to form G), each keeps its band bins
+// Y_{k + P k2} of its warp's channels in registers for the whole work item (sequence x channel tile),
+// and P <= 64 puts 128 / P channel blocks on the diagonal of the 128-row operand.  Every mbarrier
+// wait is bounded.
 
 #include <cuda_bf16.h>
 
@@ -29,13 +34,11 @@ constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
 constexpr int kNcol = 64;                     // columns of a tile: TJ points x C channels
 constexpr int kTmemCols = 128;                // two accumulator buffers
-constexpr int kBSbo = 4096;                   // distance between 8-column groups of the B tile (32 K groups x 128 B)
-constexpr int kBPart = 8 * kBSbo;             // one part (hi or lo) of the B tile
 constexpr int kSpin = 1 << 22;
 
 struct InvArgs {
     const float* Y;      // [B][R][D]
-    float* part;         // [B][n_ctiles * nblk * (2 if C = 32)][L]
+    float* part;         // [B][n_parts][L]
     int* status;
     int B, N, D, P, Q, sigma, R, nblk, J, L;
     int n_ctiles, n_items;
@@ -70,77 +73,91 @@ __device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) 
     return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
 }
 
-// C_jj[k1] of the tile's points for one thread's channels, as bf16 pairs into the B tile.
-// NA: number of band bins of this row that are summed (compile time).
-template <int KB, int CHT, int NA>
-__device__ __forceinline__ void stage2_tile(const float (&yv)[KB][CHT][2], const float2* __restrict__ w_tab, int jj0, int J,
-                                            float2 rot, float2 step, unsigned char* b_hi, unsigned char* b_lo,
-                                            int row_re, int row_im, int col0) {
-    constexpr int C = 4 * CHT, TJ = kNcol / C;
+// NV bf16 values (NV / 2 packed words) to shared memory
+template <int NV> __device__ __forceinline__ void store_bf16(unsigned char* dst, const uint32_t (&v)[NV / 2]) {
+    if constexpr (NV == 8) *reinterpret_cast<uint4*>(dst) = make_uint4(v[0], v[1], v[2], v[3]);
+    else if constexpr (NV == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(v[0], v[1]);
+    else *reinterpret_cast<uint32_t*>(dst) = v[0];
+}
+
+// Row `row` of G for the tile's points and this thread's W channels, as a bf16 pair into the B tile.
+// NB bins of this lane's frequency are summed (compile time).  G = ga C.x + gb C.y + gc (partner's value).
+template <int KB, int W, int NB>
+__device__ __forceinline__ void stage2_tile(const float2 (&y)[KB][W], const float4* __restrict__ w_tab, int jj0, int J,
+                                            float2 rot, float2 step, float ga, float gb, float gc, bool odd,
+                                            unsigned char* b_hi, unsigned char* b_lo, int sbo, int row, int col0) {
+    constexpr int C = 4 * W, TJ = kNcol / C;
+    constexpr int HV = W >= 8 ? 8 : W;        // bf16 values per store
 #pragma unroll 1
     for (int jl = 0; jl < TJ; ++jl) {
         const int jj = jj0 + jl;
-        float re[CHT], im[CHT];
+        float g[W];
         if (jj < J) {
-            float2 g[NA];
+            const float2 rxx = make_float2(rot.x, rot.x), ryy = make_float2(-rot.y, rot.y);
+            // s = sum_t y_t w_t as packed FMAs: (w.x, w.x) * (y.x, y.y) + (-w.y, w.y) * (y.y, y.x)
+            float2 s[W];
+            if constexpr (NB <= 6) {            // few bins: the table row stays in registers across the channels
+                float4 tw[NB];
 #pragma unroll
-            for (int t = 0; t < NA; ++t) g[t] = w_tab[jj * KB + t];
+                for (int t = 0; t < NB; ++t) tw[t] = w_tab[jj * KB + t];
 #pragma unroll
-            for (int c = 0; c < CHT; ++c) {
-                float sr = 0.f, si = 0.f;
+                for (int c = 0; c < W; ++c) {
+                    s[c] = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int t = 0; t < NA; ++t) {
-                    sr = fmaf(g[t].x, yv[t][c][0], fmaf(-g[t].y, yv[t][c][1], sr));
-                    si = fmaf(g[t].x, yv[t][c][1], fmaf(g[t].y, yv[t][c][0], si));
+                    for (int t = 0; t < NB; ++t) {
+                        s[c] = __ffma2_rn(make_float2(tw[t].x, tw[t].y), y[t][c], s[c]);
+                        s[c] = __ffma2_rn(make_float2(tw[t].z, tw[t].w), make_float2(y[t][c].y, y[t][c].x), s[c]);
+                    }
                 }
-                re[c] = rot.x * sr - rot.y * si;
-                im[c] = fmaf(rot.x, si, rot.y * sr);
+            } else {                            // many bins, few channels: the table streams
+#pragma unroll
+                for (int c = 0; c < W; ++c) s[c] = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int t = 0; t < NB; ++t) {
+                    const float4 tw = w_tab[jj * KB + t];
+#pragma unroll
+                    for (int c = 0; c < W; ++c) {
+                        s[c] = __ffma2_rn(make_float2(tw.x, tw.y), y[t][c], s[c]);
+                        s[c] = __ffma2_rn(make_float2(tw.z, tw.w), make_float2(y[t][c].y, y[t][c].x), s[c]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < W; ++c) {
+                const float2 cv = __ffma2_rn(rxx, s[c], __fmul2_rn(ryy, make_float2(s[c].y, s[c].x)));   // C = rot * s
+                const float got = __shfl_xor_sync(0xffffffffu, odd ? cv.x : cv.y, 1);
+                g[c] = fmaf(ga, cv.x, fmaf(gb, cv.y, gc * got));
             }
             rot = cmul(rot, step);
         } else {
 #pragma unroll
-            for (int c = 0; c < CHT; ++c) re[c] = im[c] = 0.f;
+            for (int c = 0; c < W; ++c) g[c] = 0.f;
         }
-        // element (K row r, column n) of a part sits at (n/8) kBSbo + (r/8) 128 + (r%8) 16 + (n%8) 2
+        if (row < 0) continue;                 // a lane past the rows in use only takes part in the exchange
+        // element (K row r, column n) of a part sits at (n/8) sbo + (r/8) 128 + (r%8) 16 + (n%8) 2
         const int n = jl * C + col0;
-        const int off_n = (n >> 3) * kBSbo + (n & 7) * 2;
-        const int off_re = off_n + (row_re >> 3) * 128 + (row_re & 7) * 16;
-        const int off_im = off_n + (row_im >> 3) * 128 + (row_im & 7) * 16;
-        uint32_t hr[CHT / 2], lr[CHT / 2], hi_[CHT / 2], li[CHT / 2];
+        const int off = (n >> 3) * sbo + (n & 7) * 2 + (row >> 3) * 128 + (row & 7) * 16;
 #pragma unroll
-        for (int c = 0; c < CHT; c += 2) {
-            const __nv_bfloat16 a0 = __float2bfloat16_rn(re[c]), a1 = __float2bfloat16_rn(re[c + 1]);
-            const __nv_bfloat16 b0 = __float2bfloat16_rn(im[c]), b1 = __float2bfloat16_rn(im[c + 1]);
-            hr[c / 2] = pack_bf16(a0, a1);
-            hi_[c / 2] = pack_bf16(b0, b1);
-            lr[c / 2] = pack_bf16(__float2bfloat16_rn(re[c] - __bfloat162float(a0)),
-                                  __float2bfloat16_rn(re[c + 1] - __bfloat162float(a1)));
-            li[c / 2] = pack_bf16(__float2bfloat16_rn(im[c] - __bfloat162float(b0)),
-                                  __float2bfloat16_rn(im[c + 1] - __bfloat162float(b1)));
-        }
-        if constexpr (CHT == 8) {
-            *reinterpret_cast<uint4*>(b_hi + off_re) = make_uint4(hr[0], hr[1], hr[2], hr[3]);
-            *reinterpret_cast<uint4*>(b_lo + off_re) = make_uint4(lr[0], lr[1], lr[2], lr[3]);
-            *reinterpret_cast<uint4*>(b_hi + off_im) = make_uint4(hi_[0], hi_[1], hi_[2], hi_[3]);
-            *reinterpret_cast<uint4*>(b_lo + off_im) = make_uint4(li[0], li[1], li[2], li[3]);
-        } else if constexpr (CHT == 4) {
-            *reinterpret_cast<uint2*>(b_hi + off_re) = make_uint2(hr[0], hr[1]);
-            *reinterpret_cast<uint2*>(b_lo + off_re) = make_uint2(lr[0], lr[1]);
-            *reinterpret_cast<uint2*>(b_hi + off_im) = make_uint2(hi_[0], hi_[1]);
-            *reinterpret_cast<uint2*>(b_lo + off_im) = make_uint2(li[0], li[1]);
-        } else {
-            *reinterpret_cast<uint32_t*>(b_hi + off_re) = hr[0];
-            *reinterpret_cast<uint32_t*>(b_lo + off_re) = lr[0];
-            *reinterpret_cast<uint32_t*>(b_hi + off_im) = hi_[0];
-            *reinterpret_cast<uint32_t*>(b_lo + off_im) = li[0];
+        for (int h = 0; h < W / HV; ++h) {     // W = 16: two column groups
+            uint32_t hv[HV / 2], lv[HV / 2];
+#pragma unroll
+            for (int c = 0; c < HV; c += 2) {
+                const float x0 = g[h * HV + c], x1 = g[h * HV + c + 1];
+                const __nv_bfloat16 a0 = __float2bfloat16_rn(x0), a1 = __float2bfloat16_rn(x1);
+                hv[c / 2] = pack_bf16(a0, a1);
+                lv[c / 2] = pack_bf16(__float2bfloat16_rn(x0 - __bfloat162float(a0)),
+                                      __float2bfloat16_rn(x1 - __bfloat162float(a1)));
+            }
+            store_bf16<HV>(b_hi + off + h * sbo, hv);
+            store_bf16<HV>(b_lo + off + h * sbo, lv);
         }
     }
 }
 
-// KB: band bins per row held by a thread; CHT: channels per thread (C = 4 CHT per channel block).
-template <int KB, int CHT>
+// KB: band bins per lane; W: channels per thread (C = 4 W per channel block, TJ = 64 / C points per tile).
+template <int KB, int W>
 __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) {
-    constexpr int C = 4 * CHT, TJ = kNcol / C;
+    constexpr int C = 4 * W, TJ = kNcol / C;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long s_bar[kBars];
     __shared__ uint32_t s_tmem;
@@ -148,13 +165,14 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int P = a.P, D = a.D, sigma = a.sigma, J = a.J, L = a.L;
-    const int KT = a.nblk * P;                   // rows in use; the contraction runs over 2 KT (real, imaginary)
-    const int f_bytes = 2 * KT * 256;            // one part of A: 2 KT / 8 K chunks x 128 rows x 16 B
+    const int KT = a.nblk * P;                   // rows in use = K extent of the contraction
+    const int f_bytes = KT * 256;                // one part of A: KT / 8 K chunks x 128 rows x 16 B
+    const int sbo = KT * 16;                     // B: distance between 8-column groups (KT / 8 K groups x 128 B)
+    const int b_part = 8 * sbo, b_buf = 2 * b_part;
     unsigned char* s_fhi = smem;
     unsigned char* s_flo = smem + f_bytes;
-    unsigned char* s_bhi = smem + 2 * f_bytes;
-    unsigned char* s_blo = s_bhi + kBPart;
-    float2* s_w = reinterpret_cast<float2*>(s_blo + kBPart);   // [J][KB]: e^{2 pi i k2 jj / J}
+    unsigned char* s_b = smem + 2 * f_bytes;     // [2 buffers][hi, lo][8 column groups][KT / 8][128 B]
+    float4* s_w = reinterpret_cast<float4*>(s_b + 2 * b_buf);   // [J][KB]: e^{2 pi i k2 jj / J}, packed for FMA pairs
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -168,17 +186,20 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     }
     if (warp == 0) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
 
-    // A = [cos | -sin], K-major: element (row m, column kk) at (m/8)*128 + (kk/8)*2048 + (m%8)*16 + (kk%8)*2;
-    // row m = jb P + p meets column (part, jb', k1) only for jb == jb'
-    for (int idx = tid; idx < 128 * 2 * KT; idx += kThreads) {
-        const int m = idx / (2 * KT), kk = idx - m * (2 * KT);
-        const int part = kk / KT, kr = kk - part * KT;
-        const int jb = m / P, p = m - jb * P, kb = kr / P, k1 = kr - kb * P;
+    // A[m][kk] = F[kk mod P][m mod P] where row m = jb P + p and column kk = kb P + r share the block
+    // (jb == kb), K-major: element at (m/8)*128 + (kk/8)*2048 + (m%8)*16 + (kk%8)*2
+    for (int idx = tid; idx < 128 * KT; idx += kThreads) {
+        const int m = idx / KT, kk = idx - m * KT;
+        const int jb = m / P, p = m - jb * P, kb = kk / P, r = kk - kb * P;
         float v = 0.f;
         if (m < KT && jb == kb) {
-            float s, c;
-            sincospif(2.0f * (float)((k1 * p) % P) / (float)P, &s, &c);
-            v = part ? -s : c;
+            if (r == 0) v = 1.f;
+            else if (r == 1) v = (p & 1) ? -1.f : 1.f;
+            else {
+                float s, c;
+                sincospif(2.0f * (float)(((r >> 1) * p) % P) / (float)P, &s, &c);
+                v = (r & 1) ? -s : c;
+            }
         }
         const __nv_bfloat16 h = __float2bfloat16_rn(v);
         const int off = (m >> 3) * 128 + (kk >> 3) * 2048 + (m & 7) * 16 + (kk & 7) * 2;
@@ -187,10 +208,9 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     }
     for (int e = tid; e < J * KB; e += kThreads) {
         const int jj = e / KB, k2 = e - jj * KB;
-        s_w[e] = root_pos(((unsigned)jj * (unsigned)k2) % (unsigned)J, J);
+        const float2 w = root_pos(((unsigned)jj * (unsigned)k2) % (unsigned)J, J);
+        s_w[e] = make_float4(w.x, w.x, -w.y, w.y);
     }
-    // rows of B that no thread writes (KT < 128 never happens for the K extent 2 KT, which is all
-    // the MMAs read), columns of points past J are written as zeros by their owners
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -199,22 +219,26 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     volatile int* fail = &s_fail;
 
     const int quarter = warp & 3, grp = warp >> 2;
-    const int j = quarter * 32 + lane;               // row: (channel block jb, frequency k1) when producing B,
-    const int jb = j / P, k1 = j - jb * P;            //      (channel block jb, point p) when reading the result
-    const bool active = j < KT;
+    const int j = quarter * 32 + lane;               // row (channel block jb, r) of G; row (jb, point p) of the result
+    const int jb = j / P, jr = j - jb * P;
+    const bool active = j < KT, warp_active = quarter * 32 < KT;
+    const int i = jr >> 1;
+    const bool odd = jr & 1, special = i == 0;
+    const int kf = special ? (odd ? P / 2 : 0) : (odd ? P - i : i);       // this lane's frequency
+    const float ga = (odd && !special) ? 0.f : 1.f, gb = (odd && !special) ? -1.f : 0.f, gc = special ? 0.f : 1.f;
     const int tiles_per_item = (J + TJ - 1) / TJ;
     const int item_channels = a.nblk * C;
-    const float2 step = root_pos((unsigned)k1 % (unsigned)L, L);
+    const float2 step = root_pos((unsigned)kf % (unsigned)L, L);
     const uint32_t idesc = make_idesc_bf16(128, kNcol, false, true);
     const uint64_t a_hi0 = make_desc(smem_u32(s_fhi), 2048, 128), a_lo0 = make_desc(smem_u32(s_flo), 2048, 128);
-    const uint64_t b_hi0 = make_desc(smem_u32(s_bhi), 128, kBSbo), b_lo0 = make_desc(smem_u32(s_blo), 128, kBSbo);
+    const uint64_t b_d0 = make_desc(smem_u32(s_b), 128, sbo);
 
     // energies of tile `t` (accumulator t & 1) of the item (b, ctile), points jj0 ..: the warp of channel
     // group grp reads the 16 columns [16 grp, 16 grp + 16) of its rows with ONE TMEM load (a load's round
     // trip is long, so the 64 columns are spread over the four warps that share the lanes):
-    //   C = 32: point jl = grp / 2, channel half grp % 2 (two partial sums per point)
-    //   C = 16: point jl = grp;   C = 8: points 2 grp and 2 grp + 1
-    constexpr int SPLIT = C == 32 ? 2 : 1;           // partial sums per (channel block, point)
+    //   C = 64: the point's channel quarter grp;  C = 32: point grp / 2, channel half grp % 2
+    //   C = 16: point grp;                         C = 8: points 2 grp and 2 grp + 1
+    constexpr int SPLIT = C == 64 ? 4 : (C == 32 ? 2 : 1);          // partial sums per (channel block, point)
     auto read_tile = [&](int t, int b, int ctile, int jj0) {
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((t & 1) * kNcol + grp * 16);
         uint32_t v[16];
@@ -222,17 +246,17 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
         tmem_ld_wait_for(v);
         tc_fence_before();
         if (!active) return;
-        const int half = C == 32 ? (grp & 1) : 0;
-        float* out = a.part + ((size_t)b * (a.n_ctiles * a.nblk * SPLIT) + (ctile * a.nblk + jb) * SPLIT + half) * L +
-                     (size_t)k1 * J;
+        const int sub = C == 64 ? grp : (C == 32 ? (grp & 1) : 0);
+        float* out = a.part + ((size_t)b * (a.n_ctiles * a.nblk * SPLIT) + (ctile * a.nblk + jb) * SPLIT + sub) * L +
+                     (size_t)jr * J;
         constexpr int PTS = C >= 16 ? 1 : 2;          // points among the 16 columns
-        constexpr int W = 16 / PTS;                   // columns per point
+        constexpr int WP = 16 / PTS;                  // columns per point
 #pragma unroll
         for (int pt = 0; pt < PTS; ++pt) {
             float sum = 0.f;
 #pragma unroll
-            for (int q = 0; q < W; ++q) { const float x = __uint_as_float(v[pt * W + q]); sum = fmaf(x, x, sum); }
-            const int jl = C == 32 ? (grp >> 1) : (C == 16 ? grp : 2 * grp + pt);
+            for (int q = 0; q < WP; ++q) { const float x = __uint_as_float(v[pt * WP + q]); sum = fmaf(x, x, sum); }
+            const int jl = C == 64 ? 0 : (C == 32 ? (grp >> 1) : (C == 16 ? grp : 2 * grp + pt));
             if (jj0 + jl < J) out[jj0 + jl] = sum;
         }
     };
@@ -242,22 +266,21 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     bool ok = true;
     for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
         const int ctile = item % a.n_ctiles, b = item / a.n_ctiles;
-        const int ch0 = ctile * item_channels + jb * C + grp * CHT;
-        // band bins of this row: Y_k = (cos row k) + i (sin row sigma + k), k = k1 + P t
-        float yv[KB][CHT][2];
-        int nA = (active && k1 <= sigma) ? min(KB, (sigma - k1) / P + 1) : 0;
+        const int ch0 = ctile * item_channels + jb * C + grp * W;
+        // band bins of this lane: Y_k = (cos row k) + i (sin row sigma + k), k = kf + P t
+        float2 y[KB][W];
+        const int nb = (active && kf <= sigma) ? min(KB, (sigma - kf) / P + 1) : 0;
         const float* Yb = a.Y + (size_t)b * a.R * D + ch0;
+        constexpr int VEC = W >= 4 ? 4 : 2;
 #pragma unroll
         for (int q = 0; q < KB; ++q) {
-            const int k = k1 + P * q;
-            const bool have = q < nA && ch0 < D;          // ch0 is a multiple of CHT and D of 8: all CHT channels exist
+            const int k = kf + P * q;
             const float* yc = Yb + (size_t)k * D;
             const float* ys = Yb + (size_t)(sigma + k) * D;
-            constexpr int VEC = CHT >= 4 ? 4 : 2;
 #pragma unroll
-            for (int c = 0; c < CHT; c += VEC) {
+            for (int c = 0; c < W; c += VEC) {
                 float vc[4] = {0.f, 0.f, 0.f, 0.f}, vs[4] = {0.f, 0.f, 0.f, 0.f};
-                if (have) {
+                if (q < nb && ch0 + c < D) {          // D is a multiple of 8, ch0 + c of VEC: the vector is whole or absent
                     if constexpr (VEC == 4) {
                         const float4 t4 = __ldg(reinterpret_cast<const float4*>(yc + c));
                         vc[0] = t4.x; vc[1] = t4.y; vc[2] = t4.z; vc[3] = t4.w;
@@ -275,51 +298,42 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
                     }
                 }
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) { yv[q][c + e][0] = vc[e]; yv[q][c + e][1] = vs[e]; }
+                for (int e = 0; e < VEC; ++e) y[q][c + e] = make_float2(vc[e], vs[e]);
             }
         }
-        const int nA_w = __reduce_max_sync(0xffffffffu, nA);
+        const int nb_w = __reduce_max_sync(0xffffffffu, nb);
 
         for (int tile = 0; tile < tiles_per_item; ++tile, ++t) {
             const int jj0 = tile * TJ;
-            // the B tile is single: the MMAs of the previous tile must be done with it
-            if (t >= 1) ok = wait_bar(bar(kBarAccFull + ((t - 1) & 1)), ((t - 1) >> 1) & 1, fail, a.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            if (quarter * 32 < KT) {
-                const float2 rot = root_pos(((unsigned)k1 * (unsigned)jj0) % (unsigned)L, L);   // k1 jj0 < P J = L
-                unsigned char* bh = s_bhi;
-                unsigned char* bl = s_blo;
-                const int col0 = grp * CHT, rre = j, rim = KT + j;
-                if (!active) {
-                    // rows past KT of this warp: nothing to write (the MMAs read K rows below 2 KT only,
-                    // and row j >= KT as a real-part row is an imaginary-part row of another thread)
-                } else if (KB <= 4) {
-                    switch (nA_w) {
-                        case 1: stage2_tile<KB, CHT, 1>(yv, s_w, jj0, J, rot, step, bh, bl, rre, rim, col0); break;
-                        case 2: stage2_tile<KB, CHT, (KB >= 2 ? 2 : KB)>(yv, s_w, jj0, J, rot, step, bh, bl, rre, rim, col0); break;
-                        case 3: stage2_tile<KB, CHT, (KB >= 3 ? 3 : KB)>(yv, s_w, jj0, J, rot, step, bh, bl, rre, rim, col0); break;
-                        default: stage2_tile<KB, CHT, KB>(yv, s_w, jj0, J, rot, step, bh, bl, rre, rim, col0); break;
-                    }
-                } else {
-                    if (nA_w == KB - 1) stage2_tile<KB, CHT, KB - 1>(yv, s_w, jj0, J, rot, step, bh, bl, rre, rim, col0);
-                    else stage2_tile<KB, CHT, KB>(yv, s_w, jj0, J, rot, step, bh, bl, rre, rim, col0);
-                }
+            // buffer t & 1 of B is free: every warp has seen the MMAs of tile t - 2 finish (below, one tile ago)
+            if (warp_active) {
+                const float2 rot = root_pos(((unsigned)kf * (unsigned)jj0) % (unsigned)L, L);   // kf jj0 < P J = L
+                unsigned char* bh = s_b + (t & 1) * b_buf;
+                unsigned char* bl = bh + b_part;
+                const int col0 = grp * W;
+                // lanes past the rows in use take part in the exchange with zeros and store nothing
+                if (nb_w == KB)
+                    stage2_tile<KB, W, KB>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
+                else if (nb_w == KB - 1 || KB == 2)
+                    stage2_tile<KB, W, (KB > 1 ? KB - 1 : 1)>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
+                else if (KB >= 4 && nb_w <= KB / 2)
+                    stage2_tile<KB, W, (KB >= 4 ? KB / 2 : KB)>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
+                else
+                    stage2_tile<KB, W, KB>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
             }
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarReady + (t & 1)));
             if (tid == 0) {
-                // every warp has written its share (and has finished reading accumulator t & 1, which it
-                // last did for tile t - 2, before it came here): run the three products
+                // every warp has written its share of B (and, before that, read the last of accumulator
+                // t & 1, which held tile t - 2): run the three products
                 ok = wait_bar(bar(kBarReady + (t & 1)), (t >> 1) & 1, fail, a.status);
                 if (ok) {
                     tc_fence_after();
                     const uint32_t acc = tmem + (uint32_t)((t & 1) * kNcol);
-                    const int ksteps = 2 * KT / 16;
-                    uint64_t ah = a_hi0, al = a_lo0, bh_d = b_hi0, bl_d = b_lo0;   // advance by adding to the address field
-                    for (int ks = 0; ks < ksteps; ++ks) {
+                    uint64_t ah = a_hi0, al = a_lo0;             // advance by adding to the address field
+                    uint64_t bh_d = b_d0 + (uint64_t)(((t & 1) * b_buf) >> 4), bl_d = bh_d + (uint64_t)(b_part >> 4);
+                    for (int ks = 0; ks < KT / 16; ++ks) {
                         umma_bf16(acc, ah, bh_d, idesc, ks ? 1u : 0u);
                         umma_bf16(acc, ah, bl_d, idesc, 1u);
                         umma_bf16(acc, al, bh_d, idesc, 1u);
@@ -328,10 +342,14 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
                     umma_commit(bar(kBarAccFull + (t & 1)));
                 }
             }
+            // meanwhile: the energies of the previous tile, whose MMAs ran under the arithmetic above
+            if (t >= 1) ok = wait_bar(bar(kBarAccFull + ((t - 1) & 1)), ((t - 1) >> 1) & 1, fail, a.status) && ok;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            // meanwhile: the energies of the previous tile (its accumulator was awaited above)
-            if (t >= 1) read_tile(t - 1, pb, pct, pj0);
+            if (t >= 1) {
+                tc_fence_after();
+                read_tile(t - 1, pb, pct, pj0);
+            }
             pb = b; pct = ctile; pj0 = jj0;
         }
     }
@@ -349,19 +367,19 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <int KB, int CHT>
+template <int KB, int W>
 cudaError_t launch_inv2(const InvArgs& a, cudaStream_t stream) {
     const int KT = a.nblk * a.P;
-    const size_t smem = (size_t)2 * 2 * KT * 256 + 2 * kBPart + (size_t)a.J * KB * sizeof(float2);
+    const size_t smem = (size_t)2 * KT * 256 + (size_t)2 * KT * 256 + (size_t)a.J * KB * sizeof(float4);
     static int sms = 0;
     if (!sms) {
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    cudaFuncSetAttribute(spu_inv2_kernel<KB, CHT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncSetAttribute(spu_inv2_kernel<KB, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int grid = a.n_items < sms ? a.n_items : sms;
-    spu_inv2_kernel<KB, CHT><<<grid, kThreads, smem, stream>>>(a);
+    spu_inv2_kernel<KB, W><<<grid, kThreads, smem, stream>>>(a);
     return cudaGetLastError();
 }
 
@@ -379,17 +397,18 @@ SpuInv2Plan spu_inv2_plan(int B, int N, int D, int sigma) {
     pl.J = pl.coarse ? (int)jc : pl.Q;
     pl.L = pl.P * pl.J;
     const int nk2 = sigma / pl.P + 1;
-    if (nk2 <= 4) { pl.KB = 4; pl.CHT = 8; }
+    if (nk2 <= 2) { pl.KB = 2; pl.CHT = 16; }
+    else if (nk2 <= 4) { pl.KB = 4; pl.CHT = 8; }
     else if (nk2 <= 9) { pl.KB = 9; pl.CHT = 4; }
     else if (nk2 <= 17) { pl.KB = 17; pl.CHT = 2; }
     else return pl;
-    if ((size_t)pl.J * pl.KB * sizeof(float2) > 24 * 1024) return pl;
-    const int C = 4 * pl.CHT * pl.nblk;
-    pl.n_ctiles = (D + C - 1) / C;
+    if ((size_t)pl.J * pl.KB * sizeof(float4) > 24 * 1024) return pl;
+    const int C = 4 * pl.CHT;                          // channels of one block
+    pl.n_ctiles = (D + C * pl.nblk - 1) / (C * pl.nblk);
     const long long items = (long long)B * pl.n_ctiles;
     if (items > 0x7fffffffll) return pl;
     pl.n_items = (int)items;
-    pl.n_parts = pl.n_ctiles * pl.nblk * (pl.CHT == 8 ? 2 : 1);
+    pl.n_parts = pl.n_ctiles * pl.nblk * (C == 64 ? 4 : (C == 32 ? 2 : 1));
     pl.ok = 1;
     return pl;
 }
@@ -402,7 +421,8 @@ int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, in
     a.B = B; a.N = N; a.D = D; a.P = pl.P; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
     a.nblk = pl.nblk; a.J = pl.J; a.L = pl.L; a.n_ctiles = pl.n_ctiles; a.n_items = pl.n_items;
     cudaError_t err;
-    if (pl.KB == 4) err = launch_inv2<4, 8>(a, stream);
+    if (pl.KB == 2) err = launch_inv2<2, 16>(a, stream);
+    else if (pl.KB == 4) err = launch_inv2<4, 8>(a, stream);
     else if (pl.KB == 9) err = launch_inv2<9, 4>(a, stream);
     else err = launch_inv2<17, 2>(a, stream);
     count_launch();
