@@ -262,6 +262,27 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------- multi-rank bookkeeping
+
+
+def max_over_ranks(ms_local, world, device="cpu"):
+    """The slowest rank's time: every rank contributes its own device-timed milliseconds."""
+    if world <= 1:
+        return float(ms_local)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_second(tokens_per_rank, world, ms_per_step):
+    """Weak scaling: every rank runs the same per-GPU batch, units are independent, no collective in
+    the data path; the job's throughput is all ranks' tokens over the slowest rank's time."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 # ----------------------------------------------------------------------------- the GPU arm
 
 
@@ -326,12 +347,9 @@ def main():
     ms_total = ev0.elapsed_time(ev1)
     launches = luvc.kernel_launches() - launches0
     clocks = sampler.stop()
-    t = torch.tensor([ms_total], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, device)
     ms_per_step = ms_total / args.steps
-    value = world * spec["tokens"] / (ms_per_step * 1e-3)
+    value = whole_job_tokens_per_second(spec["tokens"], world, ms_per_step)
 
     # ---- per-phase pass: the library's own events around its phases, one step at a time
     luvc.profile_enable(True)
@@ -367,10 +385,7 @@ def main():
         e2e_step()
     ev1.record()
     barrier()
-    t = torch.tensor([ev0.elapsed_time(ev1) / e2e_reps], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1) / e2e_reps, world, device)
     h2d = x_host.numel() * 2 + y_host.numel() * 2
     d2h = sum(t_.numel() * t_.element_size() for t_ in (o_tok, o_sz, o_map, o_idx, o_hid))
 
@@ -419,7 +434,7 @@ def main():
         "config": {"workload": workload_name(spec), "l2": "inputs rotate over %d distinct sets (%.0f MB) > L2" % (
             sets, sets * (oim_in_bytes + spu_in_bytes) / 1e6), "parallelism": "batch split, no collective" if world > 1 else "1 GPU"},
         "clocks": clocks,
-        "e2e": {"value": world * spec["tokens"] / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_tokens_per_second(spec["tokens"], world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "phases_ms": phases,
