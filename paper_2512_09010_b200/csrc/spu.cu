@@ -152,14 +152,26 @@ __global__ void __launch_bounds__(kGemmThreads) spu_contract_kernel(const void* 
     }
 }
 
-// E[b][n] = sqrt(sum over the channel tiles, in tile order); with `squared` the sum itself.
-__global__ void spu_energy_kernel(const float* part, float* E, int N, int tiles, long long total, int squared) {
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    const int b = (int)(i / N), n = (int)(i % N);
+// E[b][n] = sqrt(sum over the channel tiles); with `squared` the sum itself.  The order of the sum is
+// fixed: thread group g adds tiles g, g + 8, ... in turn, then the eight group sums are added in order.
+__global__ void __launch_bounds__(256) spu_energy_kernel(const float* part, float* E, int N, int tiles, long long total,
+                                                         int squared) {
+    __shared__ float s_sum[8][33];
+    const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
+    const long long i = (long long)blockIdx.x * 32 + lane;
     float s = 0.f;
-    for (int t = 0; t < tiles; ++t) s += part[((size_t)b * tiles + t) * N + n];
-    E[i] = squared ? s : sqrtf(s);
+    if (i < total) {
+        const int b = (int)(i / N), n = (int)(i % N);
+        for (int t = g; t < tiles; t += 8) s += part[((size_t)b * tiles + t) * N + n];
+    }
+    s_sum[g][lane] = s;
+    __syncthreads();
+    if (g == 0 && i < total) {
+        float r = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) r += s_sum[q][lane];
+        E[i] = squared ? r : sqrtf(r);
+    }
 }
 
 // ---- squared energies from L uniform samples of the period to the N tokens --------------------
@@ -302,14 +314,32 @@ __global__ void __launch_bounds__(kSelThreads) spu_select_kernel(const float* __
             if ((key & himask) == prefix) atomicAdd(&s_hist[(key >> (8 * pass)) & 255u], 1);
         }
         __syncthreads();
-        if (tid == 0) {
-            int rem = s_remaining, bucket = 255;
-            for (; bucket > 0; --bucket) {
-                if (s_hist[bucket] >= rem) break;
-                rem -= s_hist[bucket];
+        if (tid < 32) {
+            // the bucket in which the count from the top reaches `rem`: lane l owns buckets 8l .. 8l+7
+            const int rem = s_remaining;
+            int h[8], mine = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { h[q] = s_hist[tid * 8 + q]; mine += h[q]; }
+            int above = mine;                                  // inclusive sum over lanes >= tid
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_down_sync(0xffffffffu, above, o);
+                if (tid + o < 32) above += v;
             }
-            s_prefix = prefix | ((unsigned)bucket << (8 * pass));
-            s_remaining = rem;
+            above -= mine;                                     // keys in the buckets of the lanes above this one
+            const bool here = above < rem && above + mine >= rem;
+            const unsigned who = __ballot_sync(0xffffffffu, here);
+            if (who == 0u) {                                   // fewer keys than asked for (cannot happen): bucket 0
+                if (tid == 0) { s_prefix = prefix; s_remaining = rem; }
+            } else if (tid == 31 - __clz(who)) {
+                int r = rem - above, bucket = 7;
+                for (; bucket > 0; --bucket) {
+                    if (h[bucket] >= r) break;
+                    r -= h[bucket];
+                }
+                s_prefix = prefix | ((unsigned)(tid * 8 + bucket) << (8 * pass));
+                s_remaining = r;
+            }
         }
         __syncthreads();
     }
@@ -453,12 +483,12 @@ static int spu_run_typed(const SpuProblem& p) {
                                               p.stream, mode.fwd2);
         if (rc != LUVC_OK) return rc;
         if (!mode.coarse) {
-            spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, E, N, mode.n_parts, bn, 0);
+            spu_energy_kernel<<<(unsigned)((bn + 31) / 32), 256, 0, p.stream>>>(ws.tc.part, E, N, mode.n_parts, bn, 0);
             count_launch();
         } else {
             const int L = mode.L, F = 2 * sigma, chunks = (L + kSpecChunk - 1) / kSpecChunk;
             const long long bl = (long long)B * L;
-            spu_energy_kernel<<<(unsigned)((bl + 255) / 256), 256, 0, p.stream>>>(ws.tc.part, ws.S, L, mode.n_parts, bl, 1);
+            spu_energy_kernel<<<(unsigned)((bl + 31) / 32), 256, 0, p.stream>>>(ws.tc.part, ws.S, L, mode.n_parts, bl, 1);
             spu_coarse_spectrum_kernel<<<dim3((F + 128) / 128, chunks, B), 128, 0, p.stream>>>(ws.S, ws.gpart, L, F);
             spu_coarse_synthesis_kernel<<<dim3((N / 2 + 256) / 256, B), 256, 0, p.stream>>>(ws.gpart, E, N, L, F, chunks);
             count_launch(3);
@@ -469,7 +499,7 @@ static int spu_run_typed(const SpuProblem& p) {
             p.hidden, ws.Y, ws.tw, ws.scale, N, D, sigma);
         spu_contract_kernel<T, false><<<dim3(tiles, (N + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
             ws.Y, ws.part, ws.tw, ws.scale, N, D, sigma);
-        spu_energy_kernel<<<(unsigned)((bn + 255) / 256), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn, 0);
+        spu_energy_kernel<<<(unsigned)((bn + 31) / 32), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn, 0);
         count_launch(3);
     }
     phase_end(LUVC_PHASE_SPU_TRANSFORM, p.stream);
