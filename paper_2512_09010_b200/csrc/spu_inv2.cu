@@ -94,7 +94,8 @@ __device__ __forceinline__ void stage2_tile(const float2 (&y)[KB][W], const floa
         float g[W];
         if (jj < J) {
             const float2 rxx = make_float2(rot.x, rot.x), ryy = make_float2(-rot.y, rot.y);
-            // s = sum_t y_t w_t as packed FMAs: (w.x, w.x) * (y.x, y.y) + (-w.y, w.y) * (y.y, y.x)
+            // s = sum_t y_t w_t with packed FMAs and no operand swaps: sa += (w.x, w.x) * (y.x, y.y),
+            // sb += (w.y, w.y) * (y.x, y.y); then s = (sa.x - sb.y, sa.y + sb.x)
             float2 s[W];
             if constexpr (NB <= 6) {            // few bins: the table row stays in registers across the channels
                 float4 tw[NB];
@@ -102,25 +103,29 @@ __device__ __forceinline__ void stage2_tile(const float2 (&y)[KB][W], const floa
                 for (int t = 0; t < NB; ++t) tw[t] = w_tab[jj * KB + t];
 #pragma unroll
                 for (int c = 0; c < W; ++c) {
-                    s[c] = make_float2(0.f, 0.f);
+                    float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
 #pragma unroll
                     for (int t = 0; t < NB; ++t) {
-                        s[c] = __ffma2_rn(make_float2(tw[t].x, tw[t].y), y[t][c], s[c]);
-                        s[c] = __ffma2_rn(make_float2(tw[t].z, tw[t].w), make_float2(y[t][c].y, y[t][c].x), s[c]);
+                        sa = __ffma2_rn(make_float2(tw[t].x, tw[t].y), y[t][c], sa);
+                        sb = __ffma2_rn(make_float2(tw[t].z, tw[t].w), y[t][c], sb);
                     }
+                    s[c] = make_float2(sa.x - sb.y, sa.y + sb.x);
                 }
             } else {                            // many bins, few channels: the table streams
+                float2 sa[W], sb[W];
 #pragma unroll
-                for (int c = 0; c < W; ++c) s[c] = make_float2(0.f, 0.f);
+                for (int c = 0; c < W; ++c) sa[c] = sb[c] = make_float2(0.f, 0.f);
 #pragma unroll
                 for (int t = 0; t < NB; ++t) {
                     const float4 tw = w_tab[jj * KB + t];
 #pragma unroll
                     for (int c = 0; c < W; ++c) {
-                        s[c] = __ffma2_rn(make_float2(tw.x, tw.y), y[t][c], s[c]);
-                        s[c] = __ffma2_rn(make_float2(tw.z, tw.w), make_float2(y[t][c].y, y[t][c].x), s[c]);
+                        sa[c] = __ffma2_rn(make_float2(tw.x, tw.y), y[t][c], sa[c]);
+                        sb[c] = __ffma2_rn(make_float2(tw.z, tw.w), y[t][c], sb[c]);
                     }
                 }
+#pragma unroll
+                for (int c = 0; c < W; ++c) s[c] = make_float2(sa[c].x - sb[c].y, sa[c].y + sb[c].x);
             }
 #pragma unroll
             for (int c = 0; c < W; ++c) {
@@ -172,7 +177,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     unsigned char* s_fhi = smem;
     unsigned char* s_flo = smem + f_bytes;
     unsigned char* s_b = smem + 2 * f_bytes;     // [2 buffers][hi, lo][8 column groups][KT / 8][128 B]
-    float4* s_w = reinterpret_cast<float4*>(s_b + 2 * b_buf);   // [J][KB]: e^{2 pi i k2 jj / J}, packed for FMA pairs
+    float4* s_w = reinterpret_cast<float4*>(s_b + 2 * b_buf);   // [J][KB]: w = e^{2 pi i k2 jj / J} as (w.x, w.x, w.y, w.y)
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -209,7 +214,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     for (int e = tid; e < J * KB; e += kThreads) {
         const int jj = e / KB, k2 = e - jj * KB;
         const float2 w = root_pos(((unsigned)jj * (unsigned)k2) % (unsigned)J, J);
-        s_w[e] = make_float4(w.x, w.x, -w.y, w.y);
+        s_w[e] = make_float4(w.x, w.x, w.y, w.y);
     }
     fence_proxy_async();
     tc_fence_before();
