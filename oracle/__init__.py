@@ -49,7 +49,7 @@ def lib() -> ctypes.CDLL:
             P = ctypes.c_void_p
             L.oracle_oim_final_dims.argtypes = [c_int, c_int, c_int, P, P]
             L.oracle_oim_schedule.argtypes = [c_int] * 6 + [P, P, c_int]
-            L.oracle_oim_batch.argtypes = [P] + [c_int] * 8 + [P, P, P, P, c_dbl, P, P, c_int]
+            L.oracle_oim_batch.argtypes = [P] + [c_int] * 9 + [P, P, P, P, c_dbl, P, P, c_int]
             L.oracle_dft_naive.argtypes = [P, c_int, P, P]
             L.oracle_dft_naive.restype = None
             L.oracle_fft.argtypes = [P, P, c_int, c_int, P, P]
@@ -98,8 +98,13 @@ def oim_schedule(H, W, Hf, Wf, r=2, height_first=False):
     return [(int(axes[i]), int(ms[i])) for i in range(n)]
 
 
-def oim(tokens, target=None, out_hw=None, r=2, height_first=False, trace=None, tol=1e-4, nthreads=None):
+def oim(tokens, target=None, out_hw=None, r=2, height_first=False, trace=None, tol=1e-4, nthreads=None,
+        matching="adjacent"):
     """Run (or, with ``trace``, replay) OIM on tokens [B,H,W,D] (float32-exact values).
+
+    ``matching``: "adjacent" compares every even cell of a line with its one or two
+    neighbours; "bipartite" compares it with every odd cell of the line (the reading
+    behind the O(n_v^1.5 k) cost stated in Section 3.2).
 
     Returns a dict: tokens [B,T,D] float64, sizes [B,T] int32, map [B,H*W] int32,
     trace [B,H*W-T] int32, stats [B,4] = (min selection margin, min direction
@@ -118,7 +123,8 @@ def oim(tokens, target=None, out_hw=None, r=2, height_first=False, trace=None, t
     if trace is not None:
         tin = np.ascontiguousarray(np.asarray(trace, dtype=np.int32)).reshape(B, H * W - T)
     nt = nthreads or hardware_threads()
-    rc = lib().oracle_oim_batch(_ptr(x), B, H, W, D, Hf, Wf, r, int(height_first), _ptr(out_tokens),
+    rc = lib().oracle_oim_batch(_ptr(x), B, H, W, D, Hf, Wf, r, int(height_first),
+                                {"adjacent": 0, "bipartite": 1}[matching], _ptr(out_tokens),
                                 _ptr(out_sizes), _ptr(out_map), _ptr(tin), float(tol), _ptr(trace_out),
                                 _ptr(stats), nt)
     if rc:

@@ -13,9 +13,10 @@
 // Where the paper is silent the reading taken is stated next to the code.
 //
 // Parity unpinned (no value in the paper to check against): the default
-// low-pass cutoff, the adjacent-neighbour reading of "similarity calculations
-// and binary matching", the rule mapping a target count to a final grid, and
-// the axis order.  Everything else is pinned by the CPU tests.
+// low-pass cutoff, the two readings of "similarity calculations and binary
+// matching" (adjacent neighbours; every even cell against every odd cell of
+// its line), the rule mapping a target count to a final grid, and the axis
+// order.  Everything else is pinned by the CPU tests.
 //
 // Build: g++ -O2 -std=c++17 -shared -fPIC -pthread luvc_oracle.cpp -o libluvc_oracle.so
 
@@ -213,6 +214,128 @@ void oim_step(std::vector<Cell>& grid, int& h, int& w, int axis, int m,
     w = nw;
 }
 
+// The full-line reading of "similarity calculations and binary matching" (Section 3.2;
+// the O(n_v^1.5 k) cost the paper states for OIM corresponds to a similarity matrix per
+// line): the cells of a line are split into set A (even positions) and set B (odd
+// positions), every A cell is compared with EVERY B cell of its line and proposes the
+// most similar one (ties: the lowest position), and the m proposals with the highest
+// similarity (ties: the lowest A position) are merged, size-weighted, into the proposed
+// B cells; several A cells may end in the same B cell.  The line closes up in order.
+// Trace entries are (A position << 16) | B position.
+void oim_step_bipartite(std::vector<Cell>& grid, int& h, int& w, int axis, int m,
+                        const int32_t* trace_in, double tol, int32_t* trace_out, OimStats& st) {
+    const int nlines = axis == 0 ? h : w;
+    const int len = axis == 0 ? w : h;
+    auto at = [&](int line, int pos) -> Cell& {
+        return axis == 0 ? grid[(size_t)line * w + pos] : grid[(size_t)pos * w + line];
+    };
+    const int nh = axis == 0 ? h : h - m, nw = axis == 0 ? w - m : w;
+    std::vector<Cell> next((size_t)nh * nw);
+    const int na = (len + 1) / 2, nb = len / 2;
+
+    for (int line = 0; line < nlines; ++line) {
+        // similarity matrix S[i][j] = cos(cell 2i, cell 2j+1)
+        std::vector<double> S((size_t)na * nb);
+        for (int i = 0; i < na; ++i)
+            for (int j = 0; j < nb; ++j) S[(size_t)i * nb + j] = cosine(at(line, 2 * i).v, at(line, 2 * j + 1).v);
+        // proposal of every A cell: first maximum of its row
+        std::vector<int> prop(na, 0);
+        std::vector<double> score(na, -std::numeric_limits<double>::infinity());
+        for (int i = 0; i < na; ++i)
+            for (int j = 0; j < nb; ++j)
+                if (S[(size_t)i * nb + j] > score[i]) { score[i] = S[(size_t)i * nb + j]; prop[i] = j; }
+        std::vector<int> order(na);
+        for (int i = 0; i < na; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return score[a] > score[b]; });
+
+        std::vector<int> src(m), dst(m);      // positions in the line
+        auto own_choice = [&]() {
+            for (int k = 0; k < m; ++k) { src[k] = 2 * order[k]; dst[k] = 2 * prop[order[k]] + 1; }
+        };
+        if (!trace_in) {
+            own_choice();
+        } else {
+            const int32_t* t = trace_in + (size_t)line * m;
+            std::vector<char> is_chosen(na, 0);
+            bool ok = true;
+            for (int k = 0; k < m; ++k) {
+                const int a = t[k] >> 16, b = t[k] & 0xffff;
+                const bool valid = t[k] >= 0 && a < len && a % 2 == 0 && b < len && b % 2 == 1 && !is_chosen[a / 2];
+                if (!valid) { ok = false; break; }
+                is_chosen[a / 2] = 1;
+                src[k] = a;
+                dst[k] = b;
+            }
+            if (!ok) {
+                st.violations++;
+                own_choice();
+            } else {
+                double min_chosen = std::numeric_limits<double>::infinity();
+                double max_unchosen = -std::numeric_limits<double>::infinity();
+                for (int i = 0; i < na; ++i) {
+                    if (is_chosen[i]) min_chosen = std::min(min_chosen, score[i]);
+                    else max_unchosen = std::max(max_unchosen, score[i]);
+                }
+                if (m > 0 && min_chosen < max_unchosen - tol) st.violations++;
+                bool differs = false;
+                for (int k = 0; k < m; ++k) {
+                    const int i = src[k] / 2, j = dst[k] / 2;
+                    if (S[(size_t)i * nb + j] < score[i] - tol) st.violations++;
+                    if (j != prop[i]) differs = true;
+                    bool in_top = false;
+                    for (int q = 0; q < m; ++q) in_top |= order[q] == i;
+                    if (!in_top) differs = true;
+                }
+                if (differs) st.deviations++;
+            }
+        }
+
+        // margins of the oracle's own decisions on this state: between the last taken and the
+        // first refused proposal, and between the best and second-best B cell of a merged A cell
+        if (m > 0 && m < na)
+            st.min_sel_margin = std::min(st.min_sel_margin, score[order[m - 1]] - score[order[m]]);
+        for (int k = 0; k < m; ++k) {
+            const int i = src[k] / 2;
+            for (int j = 0; j < nb; ++j)
+                if (j != prop[i]) st.min_dir_margin = std::min(st.min_dir_margin, score[i] - S[(size_t)i * nb + j]);
+        }
+        if (trace_out)
+            for (int k = 0; k < m; ++k) trace_out[(size_t)line * m + k] = (src[k] << 16) | dst[k];
+
+        std::vector<char> removed(len, 0);
+        std::vector<std::vector<int>> incoming(len);
+        for (int k = 0; k < m; ++k) {
+            removed[src[k]] = 1;
+            incoming[dst[k]].push_back(src[k]);
+        }
+        int out_pos = 0;
+        for (int j = 0; j < len; ++j) {
+            if (removed[j]) continue;
+            Cell c = at(line, j);
+            if (!incoming[j].empty()) {
+                const size_t D = c.v.size();
+                std::vector<double> wsum(D);
+                long long stot = c.s;
+                for (size_t i = 0; i < D; ++i) wsum[i] = (double)c.s * c.v[i];
+                for (int a : incoming[j]) {
+                    const Cell& ca = at(line, a);
+                    for (size_t i = 0; i < D; ++i) wsum[i] += (double)ca.s * ca.v[i];
+                    stot += ca.s;
+                    c.src.insert(c.src.end(), ca.src.begin(), ca.src.end());
+                }
+                for (size_t i = 0; i < D; ++i) c.v[i] = wsum[i] / (double)stot;
+                c.s = stot;
+            }
+            if (axis == 0) next[(size_t)line * nw + out_pos] = std::move(c);
+            else next[(size_t)out_pos * nw + line] = std::move(c);
+            ++out_pos;
+        }
+    }
+    grid.swap(next);
+    h = nh;
+    w = nw;
+}
+
 // ----------------------------------------------------------------------------
 // SPU
 // ----------------------------------------------------------------------------
@@ -364,11 +487,12 @@ int oracle_oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first,
 // OIM on one image.  tokens: [H*W][D] (exact input values as float).
 // out_tokens: [Hf*Wf][D] double; out_sizes: [Hf*Wf]; out_map: [H*W] (final
 // row-major cell of every source token).  trace_in == NULL: the oracle decides.
-// Otherwise the decisions in trace_in (one int per merge, pos*2+dir, ordered by
-// step, line, rank) are checked against `tol` and applied.  trace_out (may be
+// Otherwise the decisions in trace_in (one int per merge, ordered by step, line,
+// rank; pos*2+dir for matching 0, (A position << 16) | B position for matching 1,
+// the full-line bipartite reading) are checked against `tol` and applied.  trace_out (may be
 // NULL) gets the applied decisions.  stats[0..3] = minimum selection margin,
 // minimum direction margin, violations, deviations.
-int oracle_oim_image(const float* tokens, int H, int W, int D, int Hf, int Wf, int r, int height_first,
+int oracle_oim_image(const float* tokens, int H, int W, int D, int Hf, int Wf, int r, int height_first, int matching,
                      double* out_tokens, int32_t* out_sizes, int32_t* out_map,
                      const int32_t* trace_in, double tol, int32_t* trace_out, double* stats) {
     std::vector<int32_t> axes(2 * (size_t)(H + W) + 4), ms(axes.size());
@@ -385,8 +509,8 @@ int oracle_oim_image(const float* tokens, int H, int W, int D, int Hf, int Wf, i
     OimStats st;
     for (int s = 0; s < nsteps; ++s) {
         const int nlines = axes[s] == 0 ? h : w;
-        oim_step(grid, h, w, axes[s], ms[s], trace_in ? trace_in + off : nullptr, tol,
-                 trace_out ? trace_out + off : nullptr, st);
+        (matching == 1 ? oim_step_bipartite : oim_step)(grid, h, w, axes[s], ms[s], trace_in ? trace_in + off : nullptr,
+                                                        tol, trace_out ? trace_out + off : nullptr, st);
         off += (size_t)nlines * ms[s];
     }
     for (int c = 0; c < Hf * Wf; ++c) {
@@ -402,14 +526,14 @@ int oracle_oim_image(const float* tokens, int H, int W, int D, int Hf, int Wf, i
 }
 
 // A batch of images on `nthreads` host threads (images are independent).
-int oracle_oim_batch(const float* tokens, int B, int H, int W, int D, int Hf, int Wf, int r, int height_first,
+int oracle_oim_batch(const float* tokens, int B, int H, int W, int D, int Hf, int Wf, int r, int height_first, int matching,
                      double* out_tokens, int32_t* out_sizes, int32_t* out_map,
                      const int32_t* trace_in, double tol, int32_t* trace_out, double* stats, int nthreads) {
     const size_t ntrace = (size_t)H * W - (size_t)Hf * Wf;
     std::vector<int> rc((size_t)B, 0);
     auto work = [&](int t) {
         for (int b = t; b < B; b += nthreads)
-            rc[b] = oracle_oim_image(tokens + (size_t)b * H * W * D, H, W, D, Hf, Wf, r, height_first,
+            rc[b] = oracle_oim_image(tokens + (size_t)b * H * W * D, H, W, D, Hf, Wf, r, height_first, matching,
                                      out_tokens + (size_t)b * Hf * Wf * D, out_sizes + (size_t)b * Hf * Wf,
                                      out_map + (size_t)b * H * W,
                                      trace_in ? trace_in + (size_t)b * ntrace : nullptr, tol,
