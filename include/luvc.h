@@ -116,6 +116,23 @@ int luvc_oim_plan(int H, int W, int target_count, int merge_per_step,
 /* Bytes of workspace luvc_oim_merge_ex needs for this problem. */
 size_t luvc_oim_workspace_bytes(int B, int H, int W, int D, int dtype);
 
+/*
+ * The two readings of "similarity calculations and binary matching" (Section 3.2).
+ * ADJACENT: a cell at an even position of a line is compared with its one or two
+ * neighbours in the line.  BIPARTITE: the line is split into its even-position cells
+ * (set A) and odd-position cells (set B), every A cell is compared with EVERY B cell
+ * of the line (one ceil(len/2) x floor(len/2) similarity matrix per line, the
+ * O(n_v^1.5 k) cost the section states), proposes the most similar one (ties: lowest
+ * position), and the m best proposals (ties: lowest A position) are merged; several A
+ * cells may merge into one B cell.  BIPARTITE needs H <= 256 and W <= 256
+ * (LUVC_ERR_SHAPE otherwise), and its trace entries are
+ * (position of the merged A cell << 16) | position of the B cell it merged into.
+ */
+typedef enum {
+    LUVC_OIM_MATCH_ADJACENT = 0,
+    LUVC_OIM_MATCH_BIPARTITE = 1
+} luvc_oim_matching;
+
 typedef struct {
     int dtype;               /* luvc_dtype of tokens and out_tokens */
     void* stream;            /* cudaStream_t; NULL = legacy default stream */
@@ -130,6 +147,8 @@ typedef struct {
                                 ordered by step, line, rank of the candidate */
     float* out_log_sizes;    /* optional device [B, target_count] fp32: log(s), the bias that the
                                 value enhancement of Eq. 2 adds to the values (V + log s) */
+    int matching;            /* LUVC_OIM_MATCH_ADJACENT (0) or LUVC_OIM_MATCH_BIPARTITE: which cells
+                                of a line are compared (see luvc_oim_matching) */
 } luvc_oim_opts;
 
 /*

@@ -45,7 +45,7 @@ class OimOpts(ctypes.Structure):
         ("dtype", ctypes.c_int), ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("out_h", ctypes.c_int), ("out_w", ctypes.c_int),
         ("merge_per_step", ctypes.c_int), ("height_first", ctypes.c_int), ("trace", ctypes.c_void_p),
-        ("out_log_sizes", ctypes.c_void_p),
+        ("out_log_sizes", ctypes.c_void_p), ("matching", ctypes.c_int),
     ]
 
 
@@ -159,9 +159,10 @@ def spu_sigma(N: int, cutoff: float = 0.0) -> int:
 
 def oim_merge(tokens: torch.Tensor, target_count: int, *, out_hw=None, merge_per_step: int = 0,
               height_first: bool = False, want_trace: bool = False, workspace: torch.Tensor | None = None,
-              want_log_sizes: bool = False):
+              want_log_sizes: bool = False, matching: str = "adjacent"):
     """luvc_oim_merge_ex on a CUDA tensor [B,H,W,D]; returns (out_tokens [B,T,D], out_sizes [B,T] int32,
-    out_map [B,H*W] int32) and, with want_trace, the per-merge decision log [B,H*W-T] int32."""
+    out_map [B,H*W] int32) and, with want_trace, the per-merge decision log [B,H*W-T] int32.
+    matching: "adjacent" or "bipartite" (luvc_oim_matching)."""
     if not tokens.is_cuda:
         raise ValueError("tokens must live on a CUDA device; host buffers go through oim_merge_host")
     tokens = tokens.contiguous()
@@ -182,6 +183,7 @@ def oim_merge(tokens: torch.Tensor, target_count: int, *, out_hw=None, merge_per
             o.out_h, o.out_w = int(out_hw[0]), int(out_hw[1])
         o.merge_per_step = int(merge_per_step)
         o.height_first = int(bool(height_first))
+        o.matching = {"adjacent": 0, "bipartite": 1}[matching]
         o.trace = trace.data_ptr() if (trace is not None and trace.numel()) else None
         log_sizes = torch.empty((B, max(T, 0)), dtype=torch.float32, device=dev) if want_log_sizes else None
         o.out_log_sizes = log_sizes.data_ptr() if log_sizes is not None else None

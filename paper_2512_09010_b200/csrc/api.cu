@@ -83,6 +83,8 @@ int check_oim(const void* tokens, int B, int H, int W, int D, int target, const 
         (reinterpret_cast<uintptr_t>(out_map) & 3u))
         return LUVC_ERR_ALIGN;
     if (o.merge_per_step < 0) return LUVC_ERR_TARGET;
+    if (o.matching != LUVC_OIM_MATCH_ADJACENT && o.matching != LUVC_OIM_MATCH_BIPARTITE) return LUVC_ERR_SHAPE;
+    if (o.matching == LUVC_OIM_MATCH_BIPARTITE && (H > 256 || W > 256)) return LUVC_ERR_SHAPE;
     if (o.out_h || o.out_w) {
         if (o.out_h < 1 || o.out_w < 1 || o.out_h > H || o.out_w > W) return LUVC_ERR_TARGET;
         if ((long long)o.out_h * o.out_w != (long long)target) return LUVC_ERR_TARGET;
@@ -220,6 +222,7 @@ int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target
     p.dtype = opts->dtype;
     p.out_tokens = out_tokens; p.out_sizes = out_sizes; p.out_map = out_map; p.trace = opts->trace;
     p.out_log_sizes = opts->out_log_sizes;
+    p.matching = opts->matching;
     p.workspace = ws; p.stream = static_cast<cudaStream_t>(opts->stream);
     p.status = status_word();
     if (!p.status) return LUVC_ERR_CUDA;

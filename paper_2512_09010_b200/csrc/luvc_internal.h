@@ -35,6 +35,7 @@ bool oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first, OimStep
 struct OimProblem {
     const void* tokens;
     int B, H, W, D, Hf, Wf, r, height_first, dtype;
+    int matching;   // luvc_oim_matching
     void* out_tokens;
     int32_t* out_sizes;
     int32_t* out_map;

@@ -29,7 +29,8 @@ def assert_values_close(got, ref, dtype_name, what):
 
 
 def check_oim_against_oracle(oracle, x_host, gpu_tokens, gpu_sizes, gpu_map, gpu_trace, dtype_name, *,
-                             target=None, out_hw=None, r=2, height_first=False, images=None):
+                             target=None, out_hw=None, r=2, height_first=False, images=None,
+                             matching="adjacent"):
     """x_host: float32 numpy [B,H,W,D] holding exactly the values the GPU read.
     Replays the GPU's decisions in double precision: each must be the oracle's own or tie with it
     within DECISION_TOL; the map and sizes must then equal the replayed ones exactly and the tokens
@@ -38,7 +39,7 @@ def check_oim_against_oracle(oracle, x_host, gpu_tokens, gpu_sizes, gpu_map, gpu
     B = x_host.shape[0]
     images = list(range(B)) if images is None else list(images)
     xs = x_host[images]
-    kw = dict(target=target, out_hw=out_hw, r=r, height_first=height_first)
+    kw = dict(target=target, out_hw=out_hw, r=r, height_first=height_first, matching=matching)
     free = oracle.oim(xs, **kw)
     replay = oracle.oim(xs, trace=gpu_trace[images], tol=DECISION_TOL, **kw)
     exact = 0
@@ -54,9 +55,10 @@ def check_oim_against_oracle(oracle, x_host, gpu_tokens, gpu_sizes, gpu_map, gpu
     return exact
 
 
-def check_oim_invariants(x_host, gpu_tokens, gpu_sizes, gpu_map, dtype_name, grid_in, grid_out):
+def check_oim_invariants(x_host, gpu_tokens, gpu_sizes, gpu_map, dtype_name, grid_in, grid_out, local=True):
     """Properties that hold at any size: sizes are the map's histogram and sum to H*W, every merged
-    token is the mean of its sources, and no token moves against the compaction."""
+    token is the mean of its sources, and (local=True: adjacent matching, where a cell only ever
+    merges into a neighbour) no token moves against the compaction."""
     (H, W), (Hf, Wf) = grid_in, grid_out
     B, T = gpu_sizes.shape
     hh, ww = np.divmod(np.arange(H * W), W)
@@ -69,9 +71,10 @@ def check_oim_invariants(x_host, gpu_tokens, gpu_sizes, gpu_map, dtype_name, gri
         sums = np.zeros((T, x_host.shape[-1]), np.float64)
         np.add.at(sums, m, x_host[b].reshape(H * W, -1).astype(np.float64))
         assert_values_close(gpu_tokens[b], sums / counts[:, None], dtype_name, "image %d means" % b)
-        hf, wf = np.divmod(m, Wf)
-        assert np.all(hf <= hh) and np.all(hf >= hh - (H - Hf))
-        assert np.all(wf <= ww) and np.all(wf >= ww - (W - Wf))
+        if local:
+            hf, wf = np.divmod(m, Wf)
+            assert np.all(hf <= hh) and np.all(hf >= hh - (H - Hf))
+            assert np.all(wf <= ww) and np.all(wf >= ww - (W - Wf))
 
 
 def check_spu_selection(scores_ref, gpu_idx, keep):

@@ -1,0 +1,99 @@
+"""Parity of the full-line bipartite matching of luvc_oim_merge_ex (tensor-core similarity
+matrices, through the C ABI) with the CPU oracle's statement of the same reading."""
+import numpy as np
+import pytest
+import torch
+
+import luvc_inputs as gi
+from _compare import check_oim_against_oracle, check_oim_invariants
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def luvc():
+    import paper_2512_09010_b200 as luvc
+    assert torch.cuda.is_available()
+    return luvc
+
+
+def _run(luvc, x_dev, **kw):
+    tok, sizes, mp, trace = luvc.oim_merge(x_dev, want_trace=True, matching="bipartite", **kw)
+    torch.cuda.synchronize()
+    return tok.float().cpu().numpy(), sizes.cpu().numpy(), mp.cpu().numpy(), trace.cpu().numpy()
+
+
+def _name(x):
+    return "bf16" if x.dtype == torch.bfloat16 else "f32"
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B,H,W,D,out_hw", [
+    (2, 6, 6, 64, (3, 3)), (3, 8, 5, 8, (5, 2)), (1, 7, 9, 40, (3, 7)), (2, 1, 9, 16, (1, 4)),
+    (2, 9, 1, 16, (5, 1)), (1, 12, 12, 264, (4, 4)), (1, 3, 3, 8, (1, 1)), (2, 5, 5, 24, (5, 5)),
+    (1, 33, 31, 72, (16, 15)), (1, 4, 130, 8, (2, 65)), (1, 2, 256, 136, (2, 200)), (2, 70, 40, 1280, (35, 20)),
+])
+def test_random_grids_match_the_oracle(luvc, oracle_mod, dtype, B, H, W, D, out_hw):
+    g = torch.Generator().manual_seed(H * 1000 + W * 10 + D + 1)
+    x = torch.randn((B, H, W, D), generator=g).to(dtype)
+    target = out_hw[0] * out_hw[1]
+    got = _run(luvc, x.cuda(), target_count=target, out_hw=out_hw)
+    xh = x.float().numpy()
+    check_oim_against_oracle(oracle_mod, xh, *got, _name(x), out_hw=out_hw, matching="bipartite")
+    check_oim_invariants(xh, got[0], got[1], got[2], _name(x), (H, W), out_hw, local=False)
+
+
+def test_a_distant_twin_is_merged(luvc):
+    # one row of mutually orthogonal cells, except that cell 0 is parallel to cell 5
+    x = torch.zeros((1, 1, 8, 8))
+    for j in range(8):
+        x[0, 0, j, j] = 1.0 + j
+    x[0, 0, 0] = 3.0 * x[0, 0, 5]
+    x[0, 0, 6] = x[0, 0, 1] + 0.25 * x[0, 0, 6]
+    got = _run(luvc, x.cuda(), target_count=6, out_hw=(1, 6))
+    assert got[3][0].tolist() == [(0 << 16) | 5, (6 << 16) | 1]
+    assert got[2][0].tolist() == [4, 0, 1, 2, 3, 4, 0, 5]
+    assert got[1][0].tolist() == [2, 1, 1, 1, 2, 1]
+
+
+def test_options_ties_and_merge_number(luvc, oracle_mod):
+    x = torch.ones((1, 3, 9, 16))
+    got = _run(luvc, x.cuda(), target_count=21, out_hw=(3, 7))
+    ref = oracle_mod.oim(x.numpy(), out_hw=(3, 7), matching="bipartite")
+    np.testing.assert_array_equal(got[3], ref["trace"])
+    np.testing.assert_array_equal(got[2], ref["map"])
+    g = torch.Generator().manual_seed(16)
+    y = torch.randn((2, 10, 9, 32), generator=g)
+    for kw in (dict(height_first=True), dict(merge_per_step=3), dict(merge_per_step=5, height_first=True)):
+        got = _run(luvc, y.cuda(), target_count=20, out_hw=(5, 4), **kw)
+        check_oim_against_oracle(oracle_mod, y.numpy(), *got, "f32", out_hw=(5, 4), matching="bipartite",
+                                 r=kw.get("merge_per_step", 2) or 2, height_first=kw.get("height_first", False))
+
+
+def test_lines_longer_than_256_cells_are_refused(luvc):
+    x = torch.zeros((1, 1, 258, 8), device="cuda")
+    with pytest.raises(luvc.LuvcError) as e:
+        luvc.oim_merge(x, 129, matching="bipartite")
+    assert luvc.STATUS_NAMES[e.value.status] == "LUVC_ERR_SHAPE"
+
+
+@pytest.mark.parametrize("config", [0, 1])
+def test_small_configurations_full(luvc, oracle_mod, config):
+    c = gi.CONFIGS[config]
+    x = gi.oim_input(config, device="cuda")
+    got = _run(luvc, x, target_count=c["target"])
+    xh = x.float().cpu().numpy()
+    check_oim_against_oracle(oracle_mod, xh, *got, c["dtype"], target=c["target"], matching="bipartite")
+    Hf, Wf, _ = luvc.oim_plan(c["H"], c["W"], c["target"])
+    check_oim_invariants(xh, got[0], got[1], got[2], c["dtype"], (c["H"], c["W"]), (Hf, Wf), local=False)
+
+
+@pytest.mark.parametrize("config", [2, 3, 4])
+def test_large_configurations_sampled_replay_and_invariants(luvc, oracle_mod, config):
+    c = gi.CONFIGS[config]
+    x = gi.oim_input(config, device="cuda")
+    got = _run(luvc, x, target_count=c["target"])
+    xh = x.float().cpu().numpy()
+    Hf, Wf, _ = luvc.oim_plan(c["H"], c["W"], c["target"])
+    check_oim_invariants(xh, got[0], got[1], got[2], c["dtype"], (c["H"], c["W"]), (Hf, Wf), local=False)
+    check_oim_against_oracle(oracle_mod, xh, *got, c["dtype"], target=c["target"], images=[0], matching="bipartite")
