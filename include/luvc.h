@@ -113,8 +113,11 @@ int luvc_profile_read(float* ms, int count);
 int luvc_oim_plan(int H, int W, int target_count, int merge_per_step,
                   int* out_h, int* out_w, int* n_steps);
 
-/* Bytes of workspace luvc_oim_merge_ex needs for this problem. */
+/* Bytes of workspace luvc_oim_merge_ex needs for this problem with the adjacent matching;
+ * the _ex form takes the luvc_oim_matching (the bipartite matching also keeps a bf16
+ * hi + lo copy of every fp32 row).  0 for invalid arguments. */
 size_t luvc_oim_workspace_bytes(int B, int H, int W, int D, int dtype);
+size_t luvc_oim_workspace_bytes_ex(int B, int H, int W, int D, int dtype, int matching);
 
 /*
  * The two readings of "similarity calculations and binary matching" (Section 3.2).
@@ -125,7 +128,8 @@ size_t luvc_oim_workspace_bytes(int B, int H, int W, int D, int dtype);
  * O(n_v^1.5 k) cost the section states), proposes the most similar one (ties: lowest
  * position), and the m best proposals (ties: lowest A position) are merged; several A
  * cells may merge into one B cell.  BIPARTITE needs H <= 256 and W <= 256
- * (LUVC_ERR_SHAPE otherwise), and its trace entries are
+ * (LUVC_ERR_SHAPE otherwise) and D a multiple of 8 (LUVC_ERR_ALIGN), a larger workspace
+ * (luvc_oim_workspace_bytes_ex), and its trace entries are
  * (position of the merged A cell << 16) | position of the B cell it merged into.
  */
 typedef enum {

@@ -27,7 +27,7 @@ STATUS_NAMES = {
 EXPORTS = (
     "luvc_version", "luvc_status_string", "luvc_set_stream", "luvc_shutdown", "luvc_kernel_launches",
     "luvc_profile_enable", "luvc_profile_read", "luvc_check_status",
-    "luvc_oim_plan", "luvc_oim_workspace_bytes", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
+    "luvc_oim_plan", "luvc_oim_workspace_bytes", "luvc_oim_workspace_bytes_ex", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
     "luvc_oim_merge_host", "luvc_oim_value_enhance", "luvc_spu_sigma", "luvc_spu_workspace_bytes", "luvc_spu_prune",
     "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host", "luvc_spu_prune_static", "luvc_spu_cascade",
 )
@@ -77,6 +77,8 @@ def _load() -> ctypes.CDLL:
     L.luvc_oim_plan.argtypes = [i, i, i, i, ctypes.POINTER(i), ctypes.POINTER(i), ctypes.POINTER(i)]
     L.luvc_oim_workspace_bytes.restype = sz
     L.luvc_oim_workspace_bytes.argtypes = [i, i, i, i, i]
+    L.luvc_oim_workspace_bytes_ex.restype = sz
+    L.luvc_oim_workspace_bytes_ex.argtypes = [i, i, i, i, i, i]
     L.luvc_oim_merge.argtypes = [p, i, i, i, i, i, p, p, p]
     L.luvc_oim_merge_f32.argtypes = [p, i, i, i, i, i, p, p, p]
     L.luvc_oim_merge_ex.argtypes = [p, i, i, i, i, i, p, p, p, ctypes.POINTER(OimOpts)]

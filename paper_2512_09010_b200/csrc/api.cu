@@ -85,6 +85,7 @@ int check_oim(const void* tokens, int B, int H, int W, int D, int target, const 
     if (o.merge_per_step < 0) return LUVC_ERR_TARGET;
     if (o.matching != LUVC_OIM_MATCH_ADJACENT && o.matching != LUVC_OIM_MATCH_BIPARTITE) return LUVC_ERR_SHAPE;
     if (o.matching == LUVC_OIM_MATCH_BIPARTITE && (H > 256 || W > 256)) return LUVC_ERR_SHAPE;
+    if (o.matching == LUVC_OIM_MATCH_BIPARTITE && D % 8 != 0) return LUVC_ERR_ALIGN;
     if (o.out_h || o.out_w) {
         if (o.out_h < 1 || o.out_w < 1 || o.out_h > H || o.out_w > W) return LUVC_ERR_TARGET;
         if ((long long)o.out_h * o.out_w != (long long)target) return LUVC_ERR_TARGET;
@@ -201,13 +202,19 @@ size_t luvc_oim_workspace_bytes(int B, int H, int W, int D, int dtype) {
     return oim_workspace_bytes(B, H, W, D, dtype);
 }
 
+size_t luvc_oim_workspace_bytes_ex(int B, int H, int W, int D, int dtype, int matching) {
+    if (B < 1 || H < 1 || W < 1 || D < 1) return 0;
+    if (matching != LUVC_OIM_MATCH_ADJACENT && matching != LUVC_OIM_MATCH_BIPARTITE) return 0;
+    return oim_workspace_bytes(B, H, W, D, dtype, matching);
+}
+
 int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target_count, void* out_tokens,
                       int32_t* out_sizes, int32_t* out_map, const luvc_oim_opts* opts) {
     if (!opts) return LUVC_ERR_NULL;
     int Hf = 0, Wf = 0;
     const int rc = check_oim(tokens, B, H, W, D, target_count, out_tokens, out_sizes, out_map, *opts, &Hf, &Wf);
     if (rc) return rc;
-    const size_t need = oim_workspace_bytes(B, H, W, D, opts->dtype);
+    const size_t need = oim_workspace_bytes(B, H, W, D, opts->dtype, opts->matching);
     void* ws = opts->workspace;
     if (ws) {
         if (opts->workspace_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u)) return LUVC_ERR_WORKSPACE;

@@ -45,7 +45,7 @@ struct OimProblem {
     int* status;   // device status word shared by all calls (0 = ok, else a luvc_status)
     cudaStream_t stream;
 };
-size_t oim_workspace_bytes(int B, int H, int W, int D, int dtype);
+size_t oim_workspace_bytes(int B, int H, int W, int D, int dtype, int matching = 0);
 int oim_run(const OimProblem& p);
 int oim_value_enhance(const void* values, const int32_t* sizes, long long rows, int D, int dtype, void* out,
                       cudaStream_t stream);

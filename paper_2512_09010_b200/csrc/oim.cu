@@ -389,11 +389,13 @@ struct Workspace {
     StepDesc* steps;
     int* done;
     int* counters;   // [0] next item, [1] status
+    __nv_bfloat16* split;   // bipartite matching only
+    float* nrm2;            // bipartite matching only
 };
 
 size_t max_steps(int H, int W) { return (size_t)H + W + 2; }
 
-Workspace carve(void* ws, int B, int H, int W, int D) {
+Workspace carve(void* ws, int B, int H, int W, int D, int matching) {
     unsigned char* p = static_cast<unsigned char*>(ws);
     Workspace w;
     const size_t n = (size_t)B * H * W;
@@ -405,7 +407,13 @@ Workspace carve(void* ws, int B, int H, int W, int D) {
     w.cellpos = reinterpret_cast<int32_t*>(p); p += align_up(n * 4);
     w.steps = reinterpret_cast<StepDesc*>(p); p += align_up(max_steps(H, W) * sizeof(StepDesc));
     w.done = reinterpret_cast<int*>(p); p += align_up(max_steps(H, W) * B * sizeof(int));
-    w.counters = reinterpret_cast<int*>(p);
+    w.counters = reinterpret_cast<int*>(p); p += 256;
+    w.split = nullptr;
+    w.nrm2 = nullptr;
+    if (matching == LUVC_OIM_MATCH_BIPARTITE) {
+        w.split = reinterpret_cast<__nv_bfloat16*>(p); p += align_up(n * D * 2 * sizeof(__nv_bfloat16));
+        w.nrm2 = reinterpret_cast<float*>(p);
+    }
     return w;
 }
 
@@ -453,10 +461,12 @@ bool oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first, OimStep
     return true;
 }
 
-size_t oim_workspace_bytes(int B, int H, int W, int D, int /*dtype*/) {
+size_t oim_workspace_bytes(int B, int H, int W, int D, int /*dtype*/, int matching) {
     const size_t n = (size_t)B * H * W;
-    return align_up(n * D * sizeof(float)) + 5 * align_up(n * 4) + align_up(max_steps(H, W) * sizeof(StepDesc)) +
-           align_up(max_steps(H, W) * B * sizeof(int)) + 256;
+    size_t bytes = align_up(n * D * sizeof(float)) + 5 * align_up(n * 4) + align_up(max_steps(H, W) * sizeof(StepDesc)) +
+                   align_up(max_steps(H, W) * B * sizeof(int)) + 256;
+    if (matching == LUVC_OIM_MATCH_BIPARTITE) bytes += align_up(n * D * 2 * sizeof(__nv_bfloat16)) + align_up(n * 4);
+    return bytes;
 }
 
 template <typename T, int NCHUNK, int MINB>
@@ -492,7 +502,7 @@ template <typename T>
 static int oim_run_typed(const OimProblem& p) {
     const int HW = p.H * p.W, target = p.Hf * p.Wf;
     const long long n = (long long)p.B * HW;
-    Workspace ws = carve(p.workspace, p.B, p.H, p.W, p.D);
+    Workspace ws = carve(p.workspace, p.B, p.H, p.W, p.D, p.matching);
     const int cap = (int)max_steps(p.H, p.W);
     OimStep* steps = new OimStep[cap];
     int n_steps = 0;
@@ -516,7 +526,7 @@ static int oim_run_typed(const OimProblem& p) {
         ChainArgs a;
         a.tokens = p.tokens; a.acc = ws.acc; a.cell[0] = ws.cell_a; a.cell[1] = ws.cell_b;
         a.size = ws.size; a.parent = ws.parent; a.trace = p.trace; a.steps = ws.steps; a.done = ws.done;
-        a.next_item = ws.counters; a.status = p.status;
+        a.next_item = ws.counters; a.status = p.status; a.split = ws.split; a.nrm2 = ws.nrm2;
         a.B = p.B; a.HW = HW; a.D = p.D; a.n_steps = n_steps; a.total_items = (int)total_items;
         a.trace_stride = HW - target;
         const int chunk = 32 * Elem<T>::kVec;
@@ -524,7 +534,9 @@ static int oim_run_typed(const OimProblem& p) {
         const int max_len = p.H > p.W ? p.H : p.W;
         cudaError_t err;
         if (p.matching == LUVC_OIM_MATCH_BIPARTITE) {
-            err = oim_bipartite_launch(a, p.dtype, max_len, p.r, p.stream);
+            err = oim_bipartite_prepare(a, p.dtype, p.stream);
+            count_launch();
+            if (err == cudaSuccess) err = oim_bipartite_launch(a, p.dtype, max_len, p.r, p.stream);
         } else
         switch (nchunk) {
             case 4: err = launch_chain<T, 4>(a, max_len, p.r, p.stream); break;

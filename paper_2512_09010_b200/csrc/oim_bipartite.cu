@@ -6,19 +6,25 @@
 // similarity matrix S = A B^T (ceil(len/2) x floor(len/2), contraction over D) is a dense
 // contraction and runs on the tensor cores:
 //
-//   * the line's vectors are gathered through the cell grid (bf16 input rows, or fp32 sums of
-//     merged cells), split into bf16 hi + lo parts and written to shared memory as K-major
-//     operand tiles, 128 channels at a time, while each thread also accumulates the squared
-//     norms of the rows it handles;
-//   * one thread issues tcgen05.mma for hi*hi, lo*hi and hi*lo (fp32 accumulation in TMEM;
-//     a part that is zero for the whole line is skipped);
-//   * the rows of S are read back with tcgen05.ld, scaled to cosines, and each A row keeps its
-//     first maximum.
+//   * every vector the chain can meet exists in global memory as bf16 hi + lo parts with its
+//     squared norm: bf16 input rows are their own hi part (lo = 0), fp32 input rows are split
+//     by a preparation kernel, and the merge phase writes the parts and the norm of every sum
+//     it forms (next to the fp32 sum itself);
+//   * eight loader warps gather the line's rows through the cell grid with cp.async, 16 bytes
+//     at a time, straight into K-major operand tiles of 64 channels, several tiles in flight;
+//     the lo rows of an operand sit below its hi rows in the same tile;
+//   * a ninth warp issues tcgen05.mma (fp32 accumulation in TMEM): [A hi; A lo] x [B hi; B lo]^T
+//     is one instruction per 16 channels when both halves of A fit the 128 rows of the MMA, two
+//     otherwise; parts that are zero for the whole line are left out;
+//   * the rows of the product are read back with tcgen05.ld, the hi/lo blocks added, scaled to
+//     cosines, and each A row keeps its first maximum.
+// Loaders and the issuing warp meet only through mbarriers (tile landed / tile consumed).
 //
 // Ranking, the size-weighted merge and the compaction of the line follow; the data layout, the
 // work distribution (one persistent kernel, lines claimed through an atomic counter, bounded
 // waits on the image's previous step) and the emit / map kernels are those of the adjacent-pair
-// chain.  Every wait has an iteration limit and reports through the status word.
+// chain.  A line's phases are latency-bound, so several CTAs share an SM.  Every wait has an
+// iteration limit and reports through the status word.
 
 #include <cuda_bf16.h>
 #include <float.h>
@@ -32,12 +38,15 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
-constexpr int kKC = 128;                 // channels per operand tile
+constexpr int kLoaders = 256;            // threads that gather operand tiles (and do everything else)
+constexpr int kThreads = kLoaders + 32;  // plus the warp that issues the MMAs
+constexpr int kWarps = kLoaders / 32;
+constexpr int kIssueWarp = kWarps;
+constexpr int kKC = 64;                  // channels per operand tile
 constexpr int kPieces = kKC / 8;         // 16-byte pieces (8 bf16) per row and tile
-constexpr int kSlack = 2048;             // the M = 128 operand read may run this far past the last tile
+constexpr int kSlack = 4096;             // the M = 128 operand read may run this far past the last tile
 constexpr int kMaxLen = 256;             // 128 A rows (the MMA's M) and 128 B rows
+constexpr int kMaxStages = 7;
 constexpr int kWaitLimit = 1 << 22;
 
 // Operand tile of R rows (R a multiple of 8): piece p of row r sits at
@@ -48,9 +57,9 @@ __host__ __device__ constexpr int tile_lbo(int rows) { return rows * 16 + 16; }
 
 struct LineGeom {
     int na, nb;          // cells in A and B
-    int ra, rb;          // rows of the A and B tiles (na, nb rounded up to 8 and 16)
-    int lbo_a, lbo_b;
-    int off_alo, off_bhi, off_blo;   // byte offsets of the planes inside one stage (A hi at 0)
+    int ra, rb;          // rows of one half (hi or lo) of the A and B tiles: na, nb rounded up to 8 and 16
+    int lbo_a, lbo_b;    // tiles hold 2 * ra and 2 * rb rows: hi rows, then lo rows
+    int off_b;           // byte offset of the B tile inside one stage (the A tile is at 0)
     int stage_bytes;
 };
 
@@ -61,20 +70,18 @@ __host__ __device__ inline LineGeom line_geom(int len) {
     g.ra = (g.na + 7) & ~7;
     g.rb = (g.nb + 15) & ~15;
     if (g.rb < 16) g.rb = 16;
-    g.lbo_a = tile_lbo(g.ra);
-    g.lbo_b = tile_lbo(g.rb);
-    g.off_alo = kPieces * g.lbo_a;
-    g.off_bhi = 2 * kPieces * g.lbo_a;
-    g.off_blo = g.off_bhi + kPieces * g.lbo_b;
-    g.stage_bytes = g.off_blo + kPieces * g.lbo_b;
+    g.lbo_a = tile_lbo(2 * g.ra);
+    g.lbo_b = tile_lbo(2 * g.rb);
+    g.off_b = kPieces * g.lbo_a;
+    g.stage_bytes = g.off_b + kPieces * g.lbo_b;
     return g;
 }
 
 // Bounded wait on an mbarrier phase.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, int parity, int* status) {
     for (int it = 0; it < kWaitLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it > 1024) __nanosleep(64);
+        if (mbar_test_wait(bar, parity)) return true;
+        if (it > 4096) __nanosleep(64);
     }
     atomicCAS(status, 0, (int)LUVC_ERR_TIMEOUT);
     return false;
@@ -85,62 +92,79 @@ __device__ __forceinline__ unsigned pack_bf16(float a, float b) {
     return *reinterpret_cast<const unsigned*>(&p);
 }
 
-// x[0..7] -> bf16 hi parts and bf16 lo parts (x - hi), packed as 16 bytes each.
-__device__ __forceinline__ void split8(const float (&x)[8], uint4& hi, uint4& lo) {
-    unsigned h[4], l[4];
+// Writes the bf16 hi parts of x[0..V) and the bf16 lo parts (x - hi) to the two planes of a row, at channel e.
+template <int V>
+__device__ __forceinline__ void store_parts(__nv_bfloat16* hi_row, __nv_bfloat16* lo_row, int e, const float (&x)[V]) {
+    unsigned h[V / 2], l[V / 2];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < V / 2; ++q) {
         h[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
         l[q] = pack_bf16(x[2 * q] - bf16lo(h[q]), x[2 * q + 1] - bf16hi(h[q]));
     }
-    hi = make_uint4(h[0], h[1], h[2], h[3]);
-    lo = make_uint4(l[0], l[1], l[2], l[3]);
-}
-
-__device__ __forceinline__ void st_shared16(uint32_t addr, const uint4& v) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
-// Eight consecutive channels of a cell, starting at channel e, as fp32 (zeros past D).
-template <typename T>
-__device__ __forceinline__ void load_piece(const T* __restrict__ tok_row, const float* acc_row, bool merged, int e, int D,
-                                           float (&x)[8]) {
-    if (e >= D) {
-#pragma unroll
-        for (int q = 0; q < 8; ++q) x[q] = 0.f;
-        return;
-    }
-    if (merged || sizeof(T) == 4) {
-        const float* src = merged ? acc_row : reinterpret_cast<const float*>(tok_row);
-        float4 f0, f1 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (merged) {
-            f0 = __ldcg(reinterpret_cast<const float4*>(src + e));
-            if (e + 4 < D) f1 = __ldcg(reinterpret_cast<const float4*>(src + e + 4));
-        } else {
-            f0 = __ldg(reinterpret_cast<const float4*>(src + e));
-            if (e + 4 < D) f1 = __ldg(reinterpret_cast<const float4*>(src + e + 4));
-        }
-        x[0] = f0.x; x[1] = f0.y; x[2] = f0.z; x[3] = f0.w;
-        x[4] = f1.x; x[5] = f1.y; x[6] = f1.z; x[7] = f1.w;
+    if constexpr (V == 8) {
+        *reinterpret_cast<uint4*>(hi_row + e) = make_uint4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<uint4*>(lo_row + e) = make_uint4(l[0], l[1], l[2], l[3]);
     } else {
-        const uint4 u = __ldg(reinterpret_cast<const uint4*>(tok_row + e));
-        x[0] = bf16lo(u.x); x[1] = bf16hi(u.x); x[2] = bf16lo(u.y); x[3] = bf16hi(u.y);
-        x[4] = bf16lo(u.z); x[5] = bf16hi(u.z); x[6] = bf16lo(u.w); x[7] = bf16hi(u.w);
+        *reinterpret_cast<uint2*>(hi_row + e) = make_uint2(h[0], h[1]);
+        *reinterpret_cast<uint2*>(lo_row + e) = make_uint2(l[0], l[1]);
     }
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// cp.async.wait_group with a run-time count (0 .. 6 groups may stay pending).
+__device__ __forceinline__ void cp_async_wait_dyn(int n) {
+    switch (n) {
+        case 0: cp_async_wait<0>(); break;
+        case 1: cp_async_wait<1>(); break;
+        case 2: cp_async_wait<2>(); break;
+        case 3: cp_async_wait<3>(); break;
+        case 4: cp_async_wait<4>(); break;
+        case 5: cp_async_wait<5>(); break;
+        default: cp_async_wait<6>(); break;
+    }
+}
+
+// Preparation: squared norm of every input token and, for fp32 input, its bf16 hi + lo parts.
+template <typename T>
+__global__ void __launch_bounds__(256) oim_bipartite_prepare_kernel(const T* __restrict__ tokens, __nv_bfloat16* split,
+                                                                    float* nrm2, long long rows, int D) {
+    constexpr int V = Elem<T>::kVec;
+    const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const T* src = tokens + row * D;
+    float nn = 0.f;
+    for (int e = lane * V; e < D; e += 32 * V) {
+        float x[V];
+        load_vec<T>(src, nullptr, false, e, x);
+#pragma unroll
+        for (int q = 0; q < V; ++q) nn = fmaf(x[q], x[q], nn);
+        if constexpr (sizeof(T) == 4) store_parts<V>(split + row * 2 * D, split + row * 2 * D + D, e, x);
+    }
+    nn = warp_sum(nn);
+    if (lane == 0) nrm2[row] = nn;
 }
 
 struct BipartiteLaunch {
-    int n_stages;       // operand stages in shared memory
+    int n_stages;       // operand stages in shared memory (1 .. kMaxStages)
+    int ahead;          // tiles requested ahead of the one whose arrival is awaited (0 .. n_stages - 1)
     int stage_stride;   // bytes between stages (the geometry of the longest line)
-    int tmem_cols;      // power of two >= 32 covering the widest similarity matrix
+    int tmem_cols;      // power of two >= 32 covering the widest product
     int max_len, r;
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads) oim_bipartite_kernel(const ChainArgs a, const BipartiteLaunch cfg) {
+__global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainArgs a, const BipartiteLaunch cfg) {
     constexpr int V = Elem<T>::kVec;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[9];   // [0..7] stage consumed, [8] similarity matrix complete
+    // [0 .. 6] tile landed (one arrival per loader warp), [7 .. 13] tile consumed by the MMAs,
+    // [14] product complete
+    __shared__ __align__(8) unsigned long long s_bar[2 * kMaxStages + 1];
     __shared__ uint32_t s_tmem;
     __shared__ int s_item, s_ok, s_fail;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -149,17 +173,24 @@ __global__ void __launch_bounds__(kThreads) oim_bipartite_kernel(const ChainArgs
     // shared memory: operand stages, slack for the M = 128 over-read, then the per-line arrays
     const uint32_t stages_base = smem_u32(smem_raw);
     unsigned char* tail = smem_raw + (size_t)cfg.n_stages * cfg.stage_stride + kSlack;
-    float* s_nn = reinterpret_cast<float*>(tail);                         // [len][16] partial squared norms
-    float* s_rn = s_nn + (size_t)cfg.max_len * kPieces;                   // [len] 1 / |v| by tile row (A rows, then B rows)
-    unsigned* s_root = reinterpret_cast<unsigned*>(s_rn + cfg.max_len);   // [len] root | merged bit by position
-    float* s_score = reinterpret_cast<float*>(s_root + cfg.max_len);      // [na] best cosine of A cell i
-    int* s_dst = reinterpret_cast<int*>(s_score + (cfg.max_len + 1) / 2); // [na] position of its best B cell
-    int* s_sel = s_dst + (cfg.max_len + 1) / 2;                           // [m] (A position << 16) | B position
+    const __nv_bfloat16** s_hi = reinterpret_cast<const __nv_bfloat16**>(tail);   // [len] hi part of tile row
+    const __nv_bfloat16** s_lo = s_hi + cfg.max_len;                              // [len] lo part, or null (all zero)
+    float* s_rn = reinterpret_cast<float*>(s_lo + cfg.max_len);                   // [len] 1 / |v| by tile row (A rows, then B rows)
+    unsigned* s_root = reinterpret_cast<unsigned*>(s_rn + cfg.max_len);           // [len] root | merged bit by position
+    float* s_score = reinterpret_cast<float*>(s_root + cfg.max_len);              // [na] best cosine of A cell i
+    int* s_dst = reinterpret_cast<int*>(s_score + (cfg.max_len + 1) / 2);         // [na] position of its best B cell
+    int* s_sel = s_dst + (cfg.max_len + 1) / 2;                                   // [m] (A position << 16) | B position
+    float* s_part = reinterpret_cast<float*>(s_sel + cfg.r + 8);                  // partial squared norms of the new sums
+    float* s_S = reinterpret_cast<float*>(smem_raw);   // lo-row block of the product; the stages are idle when it is used
 
     const uint32_t bar0 = smem_u32(&s_bar[0]);
-    const uint32_t bar_acc = bar0 + 8 * 8;
+    const uint32_t bar_acc = bar0 + 8 * (2 * kMaxStages);
     if (tid == 0) {
-        for (int i = 0; i < 9; ++i) mbar_init(bar0 + 8 * i, 1);
+        for (int i = 0; i < kMaxStages; ++i) {
+            mbar_init(bar0 + 8 * i, kWarps);
+            mbar_init(bar0 + 8 * (kMaxStages + i), 1);
+        }
+        mbar_init(bar_acc, 1);
         mbar_fence_init();
         s_fail = 0;
     }
@@ -172,9 +203,10 @@ __global__ void __launch_bounds__(kThreads) oim_bipartite_kernel(const ChainArgs
     int step = 0;
     StepDesc st = a.steps[0];
     int step_end = a.n_steps > 1 ? a.steps[1].item_begin : a.total_items;
-    unsigned fills = 0;        // operand tiles written so far by this CTA (all items)
-    unsigned items_done = 0;   // similarity matrices completed so far by this CTA
+    unsigned fills = 0;        // operand tiles consumed so far by this CTA (all items)
+    unsigned items_done = 0;   // products completed so far by this CTA
     bool mma_pending = false;  // an item was abandoned with MMAs possibly in flight
+    const unsigned S = (unsigned)cfg.n_stages;
 
     for (;;) {
         __syncthreads();                       // the previous item's shared memory is no longer read
@@ -211,108 +243,148 @@ __global__ void __launch_bounds__(kThreads) oim_bipartite_kernel(const ChainArgs
         int32_t* size = a.size + img;
         const T* tokens = reinterpret_cast<const T*>(a.tokens) + img * D;
         float* acc = a.acc + img * D;
+        __nv_bfloat16* split = a.split + img * 2 * D;
+        float* nrm2 = a.nrm2 + img;
 
-        // ---- the line's cells; a lo part is needed only where some cell holds an fp32 sum
-        bool m_a = sizeof(T) == 4, m_b = sizeof(T) == 4;
+        // ---- the line's cells: where the parts of each row live, and its norm.  A lo part exists
+        // for fp32 input and for every cell that holds a sum.
+        bool m_a = false, m_b = false;
         for (int j = tid; j < len; j += kThreads) {
             const unsigned r = (unsigned)__ldcg(cell_in + base + j * stride);
             s_root[j] = r;
-            if (r & kMergedBit) { if (j & 1) m_b = true; else m_a = true; }
+            const int id = (int)(r & ~kMergedBit);
+            const bool parts = sizeof(T) == 4 || (r & kMergedBit) != 0;
+            const int row = (j & 1) ? g.na + (j >> 1) : (j >> 1);
+            const __nv_bfloat16* hi = parts ? split + (size_t)id * 2 * D
+                                            : reinterpret_cast<const __nv_bfloat16*>(tokens + (size_t)id * D);
+            s_hi[row] = hi;
+            s_lo[row] = parts ? hi + D : nullptr;
+            const float nn = __ldcg(nrm2 + id);
+            s_rn[row] = nn > 0.f ? 1.0f / sqrtf(nn) : 0.f;          // a zero vector has similarity 0 with everything
+            if (parts) { if (j & 1) m_b = true; else m_a = true; }
         }
         const bool lo_a = __syncthreads_or(m_a) != 0;
         const bool lo_b = __syncthreads_or(m_b) != 0;
 
-        // ---- similarity matrix: operand tiles of 128 channels, MMAs issued behind them
+        // ---- the product [A hi; A lo] x [B hi; B lo]^T over tiles of 64 channels
         const int nkc = (D + kKC - 1) / kKC;
-        const int total_q = len * kPieces;
-        const uint32_t idesc = make_idesc_bf16(128, g.rb, false, false);
-        bool alive = true;
-        for (int kc = 0; kc < nkc; ++kc) {
-            const int stage = (int)(fills % (unsigned)cfg.n_stages);
-            const unsigned use = fills / (unsigned)cfg.n_stages;
-            if (use >= 1 && !mbar_wait(bar0 + 8 * stage, (int)((use - 1) & 1), a.status)) s_fail = 1;
-            const uint32_t sb = stages_base + (uint32_t)stage * (uint32_t)cfg.stage_stride;
-            for (int q0 = tid; q0 < total_q; q0 += 4 * kThreads) {
-                float x[4][8];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int q = q0 + u * kThreads;
-                    if (q < total_q) {
-                        const int row = q >> 4, piece = q & 15;
-                        const int pos = row < g.na ? 2 * row : 2 * (row - g.na) + 1;
-                        const unsigned r = s_root[pos];
-                        const size_t o = (size_t)(r & ~kMergedBit) * D;
-                        load_piece<T>(tokens + o, acc + o, (r & kMergedBit) != 0, kc * kKC + piece * 8, D, x[u]);
+        const unsigned fill0 = fills;
+        // both halves of A inside the MMA's 128 rows, and room for the lo-row block in the idle stages
+        const bool stack_m = 2 * g.ra <= 128 && (size_t)g.ra * (g.rb + 1) * 4 <= (size_t)S * cfg.stage_stride;
+
+        if (warp < kWarps) {
+            // loaders: tile c of this line goes to stage (fill0 + c) % S once the MMAs that last read it are done
+            const int total_q = len * kPieces;
+            int issued = 0;
+            for (int kc = 0; kc < nkc; ++kc) {
+                while (issued < nkc && issued <= kc + cfg.ahead) {
+                    const unsigned f = fill0 + (unsigned)issued;
+                    const unsigned stage = f % S, use = f / S;
+                    if (use >= 1) {                                // lane 0 watches the barrier for its warp
+                        if (lane == 0 && !mbar_wait(bar0 + 8 * (kMaxStages + stage), (int)((use - 1) & 1), a.status)) s_fail = 1;
+                        __syncwarp();
                     }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int q = q0 + u * kThreads;
-                    if (q < total_q) {
-                        const int row = q >> 4, piece = q & 15;
-                        float nn = kc == 0 ? 0.f : s_nn[q];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) nn = fmaf(x[u][e], x[u][e], nn);
-                        s_nn[q] = nn;
-                        uint4 hi, lo;
-                        split8(x[u], hi, lo);
+                    const uint32_t sb = stages_base + stage * (uint32_t)cfg.stage_stride;
+                    for (int q = tid; q < total_q; q += kLoaders) {
+                        const int row = q >> 3, piece = q & 7;
+                        const int e = issued * kKC + piece * 8;
+                        const bool valid = e < D;
                         const bool is_a = row < g.na;
                         const int rr = is_a ? row : row - g.na;
-                        const uint32_t addr = sb + (is_a ? 0 : g.off_bhi) + piece * (is_a ? g.lbo_a : g.lbo_b) +
-                                              (rr >> 3) * 128 + (rr & 7) * 16;
-                        st_shared16(addr, hi);
-                        if (is_a ? lo_a : lo_b) st_shared16(addr + (is_a ? g.off_alo : g.off_blo - g.off_bhi), lo);
+                        const uint32_t dst = sb + (is_a ? 0 : g.off_b) + piece * (is_a ? g.lbo_a : g.lbo_b) +
+                                             (rr >> 3) * 128 + (rr & 7) * 16;
+                        const __nv_bfloat16* hi = s_hi[row];
+                        cp_async16(dst, valid ? hi + e : hi, valid);
+                        if (is_a ? lo_a : lo_b) {                  // the lo row sits ra (rb) rows below the hi row
+                            const __nv_bfloat16* lo = s_lo[row];
+                            const bool have = valid && lo != nullptr;
+                            cp_async16(dst + ((is_a ? g.ra : g.rb) >> 3) * 128, have ? lo + e : hi, have);
+                        }
                     }
+                    cp_async_commit();
+                    ++issued;
                 }
+                cp_async_wait_dyn(issued - kc - 1);        // this thread's share of tile kc has landed
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar0 + 8 * ((fill0 + (unsigned)kc) % S));
             }
-            fence_proxy_async();
-            __syncthreads();
-            if (s_fail) { alive = false; break; }
-            if (tid == 0) {
-                tc_fence_after();
+        } else {
+            // issuing warp: all lanes follow the barriers together (a lane that spun on the product
+            // barrier beside the issuing lane would take its issue slots)
+            const uint32_t idesc1 = make_idesc_bf16(128, lo_b ? 2 * g.rb : g.rb, false, false);
+            const uint32_t idesc2 = make_idesc_bf16(128, g.rb, false, false);
+            const bool second = lo_a && !stack_m;          // A lo x B hi as an instruction of its own
+            for (int kc = 0; kc < nkc; ++kc) {
+                const unsigned f = fill0 + (unsigned)kc;
+                const unsigned stage = f % S, use = f / S;
+                if (!mbar_wait(bar0 + 8 * stage, (int)(use & 1), a.status)) s_fail = 1;
+                __syncwarp();
+                if (lane == 0) {
+                    tc_fence_after();
+                    const uint32_t sb = stages_base + stage * (uint32_t)cfg.stage_stride;
+                    if (!s_fail) {
 #pragma unroll
-                for (int ks = 0; ks < kKC / 16; ++ks) {
-                    const uint64_t a_hi = make_desc(sb + ks * 2 * g.lbo_a, g.lbo_a, 128);
-                    const uint64_t b_hi = make_desc(sb + g.off_bhi + ks * 2 * g.lbo_b, g.lbo_b, 128);
-                    umma_bf16(tmem, a_hi, b_hi, idesc, (kc | ks) ? 1u : 0u);
-                    if (lo_a) umma_bf16(tmem, make_desc(sb + g.off_alo + ks * 2 * g.lbo_a, g.lbo_a, 128), b_hi, idesc, 1u);
-                    if (lo_b) umma_bf16(tmem, a_hi, make_desc(sb + g.off_blo + ks * 2 * g.lbo_b, g.lbo_b, 128), idesc, 1u);
+                        for (int ks = 0; ks < kKC / 16; ++ks) {
+                            const uint64_t b1 = make_desc(sb + g.off_b + ks * 2 * g.lbo_b, g.lbo_b, 128);
+                            umma_bf16(tmem, make_desc(sb + ks * 2 * g.lbo_a, g.lbo_a, 128), b1, idesc1, (kc | ks) ? 1u : 0u);
+                            if (second)
+                                umma_bf16(tmem, make_desc(sb + ks * 2 * g.lbo_a + (g.ra >> 3) * 128, g.lbo_a, 128), b1, idesc2,
+                                          1u);
+                        }
+                    }
+                    umma_commit(bar0 + 8 * (kMaxStages + stage));
                 }
-                umma_commit(bar0 + 8 * stage);
+                __syncwarp();
             }
-            ++fills;
+            if (lane == 0) umma_commit(bar_acc);
+            __syncwarp();
         }
-        if (!alive) { mma_pending = true; break; }
-        if (tid == 0) umma_commit(bar_acc);
-
-        // ---- norms (fixed summation order), while the last MMAs finish
-        for (int j = tid; j < len; j += kThreads) {
-            float nn = 0.f;
-#pragma unroll
-            for (int p = 0; p < kPieces; ++p) nn += s_nn[j * kPieces + p];
-            s_rn[j] = nn > 0.f ? 1.0f / sqrtf(nn) : 0.f;           // a zero vector has similarity 0 with everything
-        }
+        fills += (unsigned)nkc;
         if (!mbar_wait(bar_acc, (int)(items_done & 1), a.status)) s_fail = 1;
         __syncthreads();
         if (s_fail) { mma_pending = true; break; }
         ++items_done;
         tc_fence_after();
 
-        // ---- proposals: A row i (TMEM lane i) keeps the first maximum of its cosines
-        if (warp < 4 && warp * 32 < g.na) {
-            const int i = warp * 32 + lane;
-            const float rn_i = i < g.na ? s_rn[i] : 0.f;
-            float best = -INFINITY;
-            int best_j = 0;
+        // ---- with both halves of A in one MMA, the lo rows' block (A lo x B hi) goes through shared memory
+        const int ld_s = g.rb + 1;
+        if (lo_a && stack_m && warp < 4 && warp * 32 < 2 * g.ra && warp * 32 + 32 > g.ra) {
+            const int i = warp * 32 + lane - g.ra;
             for (int c0 = 0; c0 < g.rb; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
                 tmem_ld_wait_for(v);
+                if (i >= 0 && i < g.na) {
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj)
+                        if (c0 + jj < g.nb) s_S[i * ld_s + c0 + jj] = __uint_as_float(v[jj]);
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- proposals: A row i (TMEM lane i) keeps the first maximum of its cosines
+        if (warp < 4 && warp * 32 < g.na) {
+            const int i = warp * 32 + lane;
+            const float rn_i = i < g.na ? s_rn[i] : 0.f;
+            const bool add_s = lo_a && stack_m && i < g.na;
+            float best = -INFINITY;
+            int best_j = 0;
+            for (int c0 = 0; c0 < g.rb; c0 += 16) {
+                uint32_t v[16], w[16];
+                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                if (lo_b) tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(g.rb + c0), w);
+                tmem_ld_wait_for(v);
+                if (lo_b) tmem_ld_wait_for(w);
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) {
                     const int j = c0 + jj;
                     if (j < g.nb) {
-                        float c = __uint_as_float(v[jj]) * (rn_i * s_rn[g.na + j]);
+                        float d = __uint_as_float(v[jj]);                   // hi x hi
+                        if (lo_b) d += __uint_as_float(w[jj]);              // + hi x lo
+                        if (add_s) d += s_S[i * ld_s + j];                  // + lo x hi
+                        float c = d * (rn_i * s_rn[g.na + j]);
                         if (!(c == c)) c = -FLT_MAX;
                         if (c > best) { best = c; best_j = j; }
                     }
@@ -371,36 +443,44 @@ __global__ void __launch_bounds__(kThreads) oim_bipartite_kernel(const ChainArgs
             }
         }
 
-        // ---- merges: the warps are dealt out over (destination cell, slice of D).  The lowest rank
-        // that targets a destination adds every source of that destination, in rank order.
-        {
-            const int m = st.m;
-            const int nsl = m < kWarps ? kWarps / m : 1;
-            for (int idx = warp; idx < m * nsl; idx += kWarps) {
-                const int k = idx % m, sl = idx / m;
-                const int dst = s_sel[k] & 0xffff;
-                bool first = true;
-                for (int q = 0; q < k; ++q) first &= (s_sel[q] & 0xffff) != dst;
-                if (!first) continue;
-                const unsigned rd = s_root[dst];
-                const size_t od = (size_t)(rd & ~kMergedBit) * D;
-                for (int e = (sl * 32 + lane) * V; e < D; e += nsl * 32 * V) {
-                    float x[V], y[V];
-                    load_vec<T>(tokens + od, acc + od, rd & kMergedBit, e, x);
-                    for (int q = k; q < m; ++q) {
-                        if ((s_sel[q] & 0xffff) != dst) continue;
-                        const unsigned ra = s_root[s_sel[q] >> 16];
-                        const size_t oa = (size_t)(ra & ~kMergedBit) * D;
-                        load_vec<T>(tokens + oa, acc + oa, ra & kMergedBit, e, y);
+        // ---- merges: the loader warps are dealt out over (destination cell, slice of D).  The lowest
+        // rank that targets a destination adds every source of that destination, in rank order, and
+        // writes the fp32 sum, its bf16 parts and its share of the squared norm.
+        const int m = st.m;
+        const int nsl = m < kWarps ? kWarps / m : 1;
+        for (int idx = warp; idx < m * nsl && warp < kWarps; idx += kWarps) {
+            const int k = idx % m, sl = idx / m;
+            const int dst = s_sel[k] & 0xffff;
+            bool first = true;
+            for (int q = 0; q < k; ++q) first &= (s_sel[q] & 0xffff) != dst;
+            if (!first) continue;
+            const unsigned rd = s_root[dst];
+            const int id = (int)(rd & ~kMergedBit);
+            const size_t od = (size_t)id * D;
+            __nv_bfloat16* hi_row = split + (size_t)id * 2 * D;
+            float nn = 0.f;
+            for (int e = (sl * 32 + lane) * V; e < D; e += nsl * 32 * V) {
+                float x[V], y[V];
+                load_vec<T>(tokens + od, acc + od, rd & kMergedBit, e, x);
+                for (int q = k; q < m; ++q) {
+                    if ((s_sel[q] & 0xffff) != dst) continue;
+                    const unsigned ra = s_root[s_sel[q] >> 16];
+                    const size_t oa = (size_t)(ra & ~kMergedBit) * D;
+                    load_vec<T>(tokens + oa, acc + oa, ra & kMergedBit, e, y);
 #pragma unroll
-                        for (int i = 0; i < V; ++i) x[i] += y[i];
-                    }
-#pragma unroll
-                    for (int i = 0; i < V; i += 4)
-                        *reinterpret_cast<float4*>(acc + od + e + i) = make_float4(x[i], x[i + 1], x[i + 2], x[i + 3]);
+                    for (int i = 0; i < V; ++i) x[i] += y[i];
                 }
-                if (sl == 0 && lane == 0) {
-                    const int id = rd & ~kMergedBit;
+#pragma unroll
+                for (int i = 0; i < V; i += 4)
+                    *reinterpret_cast<float4*>(acc + od + e + i) = make_float4(x[i], x[i + 1], x[i + 2], x[i + 3]);
+                store_parts<V>(hi_row, hi_row + D, e, x);
+#pragma unroll
+                for (int i = 0; i < V; ++i) nn = fmaf(x[i], x[i], nn);
+            }
+            nn = warp_sum(nn);
+            if (lane == 0) {
+                s_part[k * nsl + sl] = nn;
+                if (sl == 0) {
                     int sz = __ldcg(size + id);
                     for (int q = k; q < m; ++q) {
                         if ((s_sel[q] & 0xffff) != dst) continue;
@@ -412,6 +492,16 @@ __global__ void __launch_bounds__(kThreads) oim_bipartite_kernel(const ChainArgs
                 }
             }
         }
+        __syncthreads();
+        for (int k = tid; k < m; k += kThreads) {          // norms of the new sums, slices added in order
+            const int dst = s_sel[k] & 0xffff;
+            bool first = true;
+            for (int q = 0; q < k; ++q) first &= (s_sel[q] & 0xffff) != dst;
+            if (!first) continue;
+            float nn = 0.f;
+            for (int sl = 0; sl < nsl; ++sl) nn += s_part[k * nsl + sl];
+            nrm2[s_root[dst] & ~kMergedBit] = nn;
+        }
 
         // ---- publish: every write of this line is ordered before the counter increment
         __syncthreads();
@@ -421,8 +511,9 @@ __global__ void __launch_bounds__(kThreads) oim_bipartite_kernel(const ChainArgs
         }
     }
 
-    // ---- exit: no MMA may be in flight when the accumulator columns are returned
-    if (mma_pending && tid == 0) {
+    // ---- exit: no copy and no MMA may be in flight when the CTA ends and its accumulator columns are returned
+    cp_async_wait<0>();
+    if (mma_pending && warp == kIssueWarp && lane == 0) {
         umma_commit(bar_acc);
         mbar_wait(bar_acc, (int)(items_done & 1), a.status);
     }
@@ -431,48 +522,73 @@ __global__ void __launch_bounds__(kThreads) oim_bipartite_kernel(const ChainArgs
     if (warp == 0) tmem_dealloc(tmem, cfg.tmem_cols);
 }
 
+size_t tail_bytes(int max_len, int r) {
+    return (size_t)max_len * (8 + 8 + 4 + 4) + (size_t)((max_len + 1) / 2) * 8 + (size_t)(r + 8) * 4 +
+           (size_t)(r + 8 + kWarps) * 4;
+}
+
 template <typename T>
 cudaError_t launch_typed(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
-    static int sms = 0, smem_cap = 0;
+    static int sms = 0, smem_cap = 0, regs_per_cta = 0;
     if (!sms) {
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&smem_cap, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        cudaFuncAttributes fa;
+        if (cudaFuncGetAttributes(&fa, oim_bipartite_kernel<T>) != cudaSuccess) return cudaGetLastError();
+        regs_per_cta = (kThreads / 32) * ((fa.numRegs * 32 + 255) / 256 * 256);   // registers are granted per warp, in units of 256
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
     BipartiteLaunch cfg;
     cfg.max_len = max_len;
     cfg.r = r;
     cfg.stage_stride = (line_geom(max_len).stage_bytes + 127) & ~127;
-    const size_t tail = (size_t)max_len * kPieces * 4 + (size_t)max_len * 8 + (size_t)((max_len + 1) / 2) * 8 +
-                        (size_t)(r + 8) * 4;
-    // two stages and two CTAs per SM where that fits, else as many stages (up to 4) as one CTA can hold
-    const size_t budget = (size_t)smem_cap - 1024;            // the static shared variables
-    const size_t fixed = kSlack + tail + 128;
-    int stages = 2;
-    if (2 * (2 * (size_t)cfg.stage_stride + fixed + 1024) > (size_t)smem_cap + 1024) {
-        stages = (int)((budget - fixed) / (size_t)cfg.stage_stride);
-        if (stages > 4) stages = 4;
-        if (stages < 1) return cudaErrorInvalidConfiguration;
-    }
-    cfg.n_stages = stages;
     int cols = 32;
-    while (cols < line_geom(max_len).rb) cols <<= 1;
+    while (cols < 2 * line_geom(max_len).rb) cols <<= 1;
     cfg.tmem_cols = cols;
+    const size_t fixed = kSlack + tail_bytes(max_len, r) + 128;
+    // CTAs per SM: the occupancy query of the runtime answers 1 for a kernel that allocates tensor
+    // memory, although such CTAs do share an SM; so the limits are counted here: registers, the
+    // 512 TMEM columns of an SM, and shared memory with at least three operand stages per CTA.
+    const size_t per_sm = (size_t)smem_cap + 1024;
+    int ctas = 65536 / regs_per_cta;
+    if (ctas > 512 / cols) ctas = 512 / cols;
+    if (ctas > 3) ctas = 3;
+    if (ctas < 1) ctas = 1;
+    int stages = 0;
+    for (; ctas >= 1; --ctas) {
+        const size_t budget = per_sm / ctas - 1024 /* reserved per CTA */ - 1024 /* static shared variables */;
+        stages = budget > fixed ? (int)((budget - fixed) / (size_t)cfg.stage_stride) : 0;
+        if (stages >= 3 || ctas == 1) break;
+    }
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 1) return cudaErrorInvalidConfiguration;
+    const int ahead = stages >= 3 ? stages - 2 : stages - 1;     // from three stages on, a refill never waits for the MMAs just issued
+    cfg.n_stages = stages;
+    cfg.ahead = ahead;
     const size_t smem = (size_t)stages * cfg.stage_stride + fixed;
     cudaError_t err = cudaFuncSetAttribute(oim_bipartite_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    int blocks_per_sm = 0;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, oim_bipartite_kernel<T>, kThreads, smem);
-    if (blocks_per_sm < 1) blocks_per_sm = 1;
-    if (blocks_per_sm * cols > 512) blocks_per_sm = 512 / cols;     // TMEM columns of an SM
-    int grid = blocks_per_sm * sms;
+    cudaFuncSetAttribute(oim_bipartite_kernel<T>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    int grid = ctas * sms;
     if (grid > a.total_items) grid = a.total_items;
     oim_bipartite_kernel<T><<<grid, kThreads, smem, stream>>>(a, cfg);
     return cudaGetLastError();
 }
 
 }  // namespace
+
+cudaError_t oim_bipartite_prepare(const ChainArgs& a, int dtype, cudaStream_t stream) {
+    const long long rows = (long long)a.B * a.HW;
+    const unsigned grid = (unsigned)((rows * 32 + 255) / 256);
+    if (dtype == LUVC_F32)
+        oim_bipartite_prepare_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(a.tokens), a.split, a.nrm2,
+                                                                      rows, a.D);
+    else
+        oim_bipartite_prepare_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(a.tokens), a.split, a.nrm2, rows, a.D);
+    return cudaGetLastError();
+}
 
 cudaError_t oim_bipartite_launch(const ChainArgs& a, int dtype, int max_len, int r, cudaStream_t stream) {
     if (max_len > kMaxLen) return cudaErrorInvalidValue;
