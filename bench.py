@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4])
     ap.add_argument("--impl", default="luvc", choices=["luvc", "reference"])
+    ap.add_argument("--oim-matching", default="adjacent", choices=["adjacent", "bipartite"],
+                    help="bipartite: time the full-line matching variant of OIM instead (device-timed numbers only: "
+                         "no end-to-end and no CPU-baseline leg)")
     ap.add_argument("--cpu-sample", type=int, default=0, help="units of the batch the CPU oracle is timed on (0 = auto)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -254,7 +257,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * secs / steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(spec), "note": "CPU oracle on a bounded sample per step"},
+        "config": {"workload": workload_name(spec) + ("" if args.oim_matching == "adjacent" else
+                                                      " [OIM variant: full-line bipartite matching]"), "note": "CPU oracle on a bounded sample per step"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": info["cores"], "kind": "oracle", "sample": info["sample"]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -320,7 +324,7 @@ def main():
 
     def step(i):
         x, y = xs[i % sets], ys[i % sets]
-        a = luvc.oim_merge(x, spec["target"])
+        a = luvc.oim_merge(x, spec["target"], matching=args.oim_matching)
         b = luvc.spu_prune(y, spec["keep"], spec["cutoff"])
         return a, b
 
@@ -407,12 +411,13 @@ def main():
     spu_bytes = spu_in_bytes + sb * sn * 4 + 2 * sb * spec["keep"] * sd * e + sb * spec["keep"] * 4
     spu_ms = phases["spu_transform"] + phases["spu_select"] + phases["spu_gather"]
     roofline = {
-        "kernel": "oim_chain_kernel (one launch runs the %d merge steps of a call)" % n_steps,
+        "kernel": "%s (one launch runs the %d merge steps of a call)" % (
+            "oim_chain_kernel" if args.oim_matching == "adjacent" else "oim_bipartite_kernel", n_steps),
         "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak if achieved else None, "peak_source": peak_src,
         "frac_of_8TBs": achieved / HBM_NOMINAL_GBS if achieved else None,
         "algorithmic_bytes_per_launch": iter_bytes, "avg_launch_ms": steps_ms, "merge_steps_per_launch": n_steps,
-        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(k),
+        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(k) if args.oim_matching == "adjacent" else None,
         "floor_bytes": floor_bytes,
         "spu": {"algorithmic_bytes": spu_bytes, "ms": spu_ms,
                 "achieved": spu_bytes / (spu_ms * 1e-3) / 1e9 if spu_ms > 0 else None,
@@ -420,7 +425,7 @@ def main():
     }
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and args.oim_matching == "adjacent":
         sample = args.cpu_sample or auto_cpu_sample(spec)
         info = cpu_oracle_pass(spec, sample, xs[0][:sample].float().cpu().numpy(),
                                ys[0][: max(1, sample)].float().cpu().numpy(), min_seconds=10.0)
@@ -431,11 +436,12 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32 arithmetic on bf16 I/O", "data": "synthetic",
-        "config": {"workload": workload_name(spec), "l2": "inputs rotate over %d distinct sets (%.0f MB) > L2" % (
+        "config": {"workload": workload_name(spec) + ("" if args.oim_matching == "adjacent" else
+                                                      " [OIM variant: full-line bipartite matching]"), "l2": "inputs rotate over %d distinct sets (%.0f MB) > L2" % (
             sets, sets * (oim_in_bytes + spu_in_bytes) / 1e6), "parallelism": "batch split, no collective" if world > 1 else "1 GPU"},
         "clocks": clocks,
         "e2e": {"value": whole_job_tokens_per_second(spec["tokens"], world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h} if args.oim_matching == "adjacent" else None,
         "gpu_launches": launches,
         "phases_ms": phases,
         "roofline": roofline,

@@ -81,7 +81,7 @@ __host__ __device__ inline LineGeom line_geom(int len) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, int parity, int* status) {
     for (int it = 0; it < kWaitLimit; ++it) {
         if (mbar_test_wait(bar, parity)) return true;
-        if (it > 4096) __nanosleep(64);
+        __nanosleep(it < 4096 ? 32 : 256);         // a spinning warp would take issue slots from the working ones
     }
     atomicCAS(status, 0, (int)LUVC_ERR_TIMEOUT);
     return false;
@@ -310,17 +310,16 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
                 if (lane == 0) mbar_arrive(bar0 + 8 * ((fill0 + (unsigned)kc) % S));
             }
         } else {
-            // issuing warp: all lanes follow the barriers together (a lane that spun on the product
-            // barrier beside the issuing lane would take its issue slots)
+            // issuing warp: lane 0 works, the others wait at the warp barriers (a lane that spun on the
+            // product barrier beside the issuing lane would take its issue slots)
             const uint32_t idesc1 = make_idesc_bf16(128, lo_b ? 2 * g.rb : g.rb, false, false);
             const uint32_t idesc2 = make_idesc_bf16(128, g.rb, false, false);
             const bool second = lo_a && !stack_m;          // A lo x B hi as an instruction of its own
             for (int kc = 0; kc < nkc; ++kc) {
                 const unsigned f = fill0 + (unsigned)kc;
                 const unsigned stage = f % S, use = f / S;
-                if (!mbar_wait(bar0 + 8 * stage, (int)(use & 1), a.status)) s_fail = 1;
-                __syncwarp();
                 if (lane == 0) {
+                    if (!mbar_wait(bar0 + 8 * stage, (int)(use & 1), a.status)) s_fail = 1;
                     tc_fence_after();
                     const uint32_t sb = stages_base + stage * (uint32_t)cfg.stage_stride;
                     if (!s_fail) {
@@ -341,7 +340,7 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
             __syncwarp();
         }
         fills += (unsigned)nkc;
-        if (!mbar_wait(bar_acc, (int)(items_done & 1), a.status)) s_fail = 1;
+        if (lane == 0 && !mbar_wait(bar_acc, (int)(items_done & 1), a.status)) s_fail = 1;   // one watcher per warp
         __syncthreads();
         if (s_fail) { mma_pending = true; break; }
         ++items_done;
