@@ -37,8 +37,6 @@
 namespace luvc {
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
@@ -127,8 +125,9 @@ __global__ void oim_setup_kernel(int32_t* cell, int32_t* size, int32_t* parent, 
 }
 
 // MINB: CTAs per SM the register budget is cut for (3: 80 registers, 4: 64 registers).
-template <typename T, int NCHUNK, int MINB>
-__global__ void __launch_bounds__(kThreads, MINB) oim_chain_kernel(const ChainArgs a) {
+template <typename T, int NCHUNK, int MINB, int THREADS>
+__global__ void __launch_bounds__(THREADS, MINB) oim_chain_kernel(const ChainArgs a) {
+    constexpr int kThreads = THREADS, kWarps = THREADS / 32;
     constexpr int V = Elem<T>::kVec;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_item;
@@ -469,33 +468,37 @@ size_t oim_workspace_bytes(int B, int H, int W, int D, int /*dtype*/, int matchi
     return bytes;
 }
 
-template <typename T, int NCHUNK, int MINB>
+template <typename T, int NCHUNK, int MINB, int THREADS = 256>
 static cudaError_t launch_chain_b(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
     static int sms = 0;      // per kernel instantiation
     int blocks_per_sm = 0;
     const size_t smem = (size_t)(3 * max_len + 2 * ((max_len + 1) / 2) + r + 8) * 4;
     if (smem > 48 * 1024)
-        cudaFuncSetAttribute(oim_chain_kernel<T, NCHUNK, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaFuncSetAttribute(oim_chain_kernel<T, NCHUNK, MINB, THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (!sms) {
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, oim_chain_kernel<T, NCHUNK, MINB>, kThreads, smem);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, oim_chain_kernel<T, NCHUNK, MINB, THREADS>, THREADS, smem);
     if (blocks_per_sm < 1) blocks_per_sm = 1;
     int grid = blocks_per_sm * sms;
     if (grid > a.total_items) grid = a.total_items;
-    oim_chain_kernel<T, NCHUNK, MINB><<<grid, kThreads, smem, stream>>>(a);
+    oim_chain_kernel<T, NCHUNK, MINB, THREADS><<<grid, THREADS, smem, stream>>>(a);
     return cudaGetLastError();
 }
 
 // Short lines leave a CTA mostly in its serial phases (ranking, merging, waiting for the image's
 // previous step): more resident CTAs overlap them.  Long lines are dominated by the streaming pass,
-// where the larger register budget wins.  The switch point is measured (36- vs 72-cell lines).
+// where the larger register budget wins; beyond about a hundred cells a line keeps sixteen warps
+// busy, and two CTAs of 512 threads finish each line sooner than three of 256 (a batch of few large
+// images has fewer lines per step than the GPU has CTA slots, so the time per line is what counts).
+// The switch points are measured (36-, 72- and 128-cell lines).
 template <typename T, int NCHUNK>
 static cudaError_t launch_chain(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
-    return max_len <= 48 ? launch_chain_b<T, NCHUNK, 4>(a, max_len, r, stream)
-                         : launch_chain_b<T, NCHUNK, 3>(a, max_len, r, stream);
+    if (max_len <= 48) return launch_chain_b<T, NCHUNK, 4>(a, max_len, r, stream);
+    if (max_len <= 96) return launch_chain_b<T, NCHUNK, 3>(a, max_len, r, stream);
+    return launch_chain_b<T, NCHUNK, 2, 512>(a, max_len, r, stream);
 }
 
 template <typename T>
@@ -526,7 +529,7 @@ static int oim_run_typed(const OimProblem& p) {
         ChainArgs a;
         a.tokens = p.tokens; a.acc = ws.acc; a.cell[0] = ws.cell_a; a.cell[1] = ws.cell_b;
         a.size = ws.size; a.parent = ws.parent; a.trace = p.trace; a.steps = ws.steps; a.done = ws.done;
-        a.next_item = ws.counters; a.status = p.status; a.split = ws.split; a.nrm2 = ws.nrm2;
+        a.next_item = ws.counters; a.status = p.status;
         a.B = p.B; a.HW = HW; a.D = p.D; a.n_steps = n_steps; a.total_items = (int)total_items;
         a.trace_stride = HW - target;
         const int chunk = 32 * Elem<T>::kVec;
@@ -534,9 +537,9 @@ static int oim_run_typed(const OimProblem& p) {
         const int max_len = p.H > p.W ? p.H : p.W;
         cudaError_t err;
         if (p.matching == LUVC_OIM_MATCH_BIPARTITE) {
-            err = oim_bipartite_prepare(a, p.dtype, p.stream);
+            err = oim_bipartite_prepare(a, ws.split, ws.nrm2, p.dtype, p.stream);
             count_launch();
-            if (err == cudaSuccess) err = oim_bipartite_launch(a, p.dtype, max_len, p.r, p.stream);
+            if (err == cudaSuccess) err = oim_bipartite_launch(a, ws.split, ws.nrm2, p.dtype, max_len, p.r, p.stream);
         } else
         switch (nchunk) {
             case 4: err = launch_chain<T, 4>(a, max_len, p.r, p.stream); break;

@@ -156,6 +156,8 @@ struct BipartiteLaunch {
     int stage_stride;   // bytes between stages (the geometry of the longest line)
     int tmem_cols;      // power of two >= 32 covering the widest product
     int max_len, r;
+    __nv_bfloat16* split;   // [B][HW][2][D] bf16 hi and lo parts of fp32 rows
+    float* nrm2;            // [B][HW] squared norm by root
 };
 
 template <typename T>
@@ -243,8 +245,8 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
         int32_t* size = a.size + img;
         const T* tokens = reinterpret_cast<const T*>(a.tokens) + img * D;
         float* acc = a.acc + img * D;
-        __nv_bfloat16* split = a.split + img * 2 * D;
-        float* nrm2 = a.nrm2 + img;
+        __nv_bfloat16* split = cfg.split + img * 2 * D;
+        float* nrm2 = cfg.nrm2 + img;
 
         // ---- the line's cells: where the parts of each row live, and its norm.  A lo part exists
         // for fp32 input and for every cell that holds a sum.
@@ -527,7 +529,7 @@ size_t tail_bytes(int max_len, int r) {
 }
 
 template <typename T>
-cudaError_t launch_typed(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
+cudaError_t launch_typed(const ChainArgs& a, __nv_bfloat16* split, float* nrm2, int max_len, int r, cudaStream_t stream) {
     static int sms = 0, smem_cap = 0, regs_per_cta = 0;
     if (!sms) {
         int dev = 0;
@@ -541,6 +543,8 @@ cudaError_t launch_typed(const ChainArgs& a, int max_len, int r, cudaStream_t st
     BipartiteLaunch cfg;
     cfg.max_len = max_len;
     cfg.r = r;
+    cfg.split = split;
+    cfg.nrm2 = nrm2;
     cfg.stage_stride = (line_geom(max_len).stage_bytes + 127) & ~127;
     int cols = 32;
     while (cols < 2 * line_geom(max_len).rb) cols <<= 1;
@@ -577,22 +581,23 @@ cudaError_t launch_typed(const ChainArgs& a, int max_len, int r, cudaStream_t st
 
 }  // namespace
 
-cudaError_t oim_bipartite_prepare(const ChainArgs& a, int dtype, cudaStream_t stream) {
+cudaError_t oim_bipartite_prepare(const ChainArgs& a, __nv_bfloat16* split, float* nrm2, int dtype, cudaStream_t stream) {
     const long long rows = (long long)a.B * a.HW;
     const unsigned grid = (unsigned)((rows * 32 + 255) / 256);
     if (dtype == LUVC_F32)
-        oim_bipartite_prepare_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(a.tokens), a.split, a.nrm2,
+        oim_bipartite_prepare_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(a.tokens), split, nrm2,
                                                                       rows, a.D);
     else
         oim_bipartite_prepare_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
-            static_cast<const __nv_bfloat16*>(a.tokens), a.split, a.nrm2, rows, a.D);
+            static_cast<const __nv_bfloat16*>(a.tokens), split, nrm2, rows, a.D);
     return cudaGetLastError();
 }
 
-cudaError_t oim_bipartite_launch(const ChainArgs& a, int dtype, int max_len, int r, cudaStream_t stream) {
+cudaError_t oim_bipartite_launch(const ChainArgs& a, __nv_bfloat16* split, float* nrm2, int dtype, int max_len, int r,
+                                 cudaStream_t stream) {
     if (max_len > kMaxLen) return cudaErrorInvalidValue;
-    return dtype == LUVC_F32 ? launch_typed<float>(a, max_len, r, stream)
-                             : launch_typed<__nv_bfloat16>(a, max_len, r, stream);
+    return dtype == LUVC_F32 ? launch_typed<float>(a, split, nrm2, max_len, r, stream)
+                             : launch_typed<__nv_bfloat16>(a, split, nrm2, max_len, r, stream);
 }
 
 }  // namespace luvc

@@ -63,8 +63,6 @@ struct ChainArgs {
     int32_t* size;        // [B][HW] by root
     int32_t* parent;      // [B][HW] by root: the root this one was merged into, or -1
     int32_t* trace;       // [B][HW - target] or null
-    __nv_bfloat16* split; // bipartite matching only: [B][HW][2][D] bf16 hi and lo parts of fp32 rows
-    float* nrm2;          // bipartite matching only: [B][HW] squared norm by root
     const StepDesc* steps;
     int* done;            // [n_steps][B] finished lines
     int* next_item;       // work counter
@@ -96,8 +94,12 @@ __device__ __forceinline__ bool wait_for_count(const int* ctr, int target, int* 
 
 // The chain of merge steps with the full-line bipartite matching (oim_bipartite.cu).
 // dtype: LUVC_BF16 or LUVC_F32; max_len: longest line of the schedule; r: merge number.
-// oim_bipartite_prepare fills nrm2 (and, for fp32 input, split) from the input tokens.
-cudaError_t oim_bipartite_prepare(const ChainArgs& a, int dtype, cudaStream_t stream);
-cudaError_t oim_bipartite_launch(const ChainArgs& a, int dtype, int max_len, int r, cudaStream_t stream);
+// It keeps, beside the chain's own scratch, split[B][HW][2][D] (bf16 hi and lo parts of every fp32
+// row) and nrm2[B][HW] (squared norm by root); oim_bipartite_prepare fills nrm2 (and, for fp32
+// input, split) from the input tokens.  They travel apart from ChainArgs, whose layout the
+// adjacent-pair kernel's register allocation is tuned to.
+cudaError_t oim_bipartite_prepare(const ChainArgs& a, __nv_bfloat16* split, float* nrm2, int dtype, cudaStream_t stream);
+cudaError_t oim_bipartite_launch(const ChainArgs& a, __nv_bfloat16* split, float* nrm2, int dtype, int max_len, int r,
+                                 cudaStream_t stream);
 
 }  // namespace luvc
