@@ -37,6 +37,11 @@
 namespace luvc {
 namespace {
 
+// Asks L2 for `bytes` (a multiple of 16) starting at the 16-byte aligned address p; nothing waits for it.
+__device__ __forceinline__ void prefetch_l2(const void* p, unsigned bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
@@ -53,13 +58,21 @@ __device__ __forceinline__ void pair_stats(const T* __restrict__ t0, const float
     if (has_next) {
         if constexpr (NCHUNK > 0) {
 #pragma unroll
+            float2 nn2 = make_float2(0.f, 0.f), dd2 = make_float2(0.f, 0.f);   // packed FMAs: even and odd elements apart
+#pragma unroll
             for (int c = 0; c < NCHUNK; ++c) {
                 float x[V], y[V];
                 load_vec<T>(t0, a0, m0, (c * 32 + lane) * V, x);
                 load_vec<T>(t1, a1, m1, (c * 32 + lane) * V, y);
 #pragma unroll
-                for (int q = 0; q < V; ++q) { nn = fmaf(x[q], x[q], nn); dd = fmaf(x[q], y[q], dd); }
+                for (int q = 0; q < V; q += 2) {
+                    const float2 xx = make_float2(x[q], x[q + 1]);
+                    nn2 = __ffma2_rn(xx, xx, nn2);
+                    dd2 = __ffma2_rn(xx, make_float2(y[q], y[q + 1]), dd2);
+                }
             }
+            nn += nn2.x + nn2.y;
+            dd += dd2.x + dd2.y;
         } else {
 #pragma unroll 2
             for (int e = lane * V; e < D; e += 32 * V) {
@@ -181,7 +194,16 @@ __global__ void __launch_bounds__(THREADS, MINB) oim_chain_kernel(const ChainArg
         const T* tokens = reinterpret_cast<const T*>(a.tokens) + img * D;
         float* acc = a.acc + img * D;
 
-        for (int j = tid; j < len; j += kThreads) s_root[j] = (unsigned)__ldcg(cell_in + base + j * stride);
+        // Every row of the line is asked for at once (one bulk prefetch into L2 per cell, no register
+        // held): the similarity pass below walks the cells a few at a time, and without this only its
+        // first loads would overlap the memory latency.
+        for (int j = tid; j < len; j += kThreads) {
+            const unsigned r = (unsigned)__ldcg(cell_in + base + j * stride);
+            s_root[j] = r;
+            const size_t o = (size_t)(r & ~kMergedBit) * D;
+            if (r & kMergedBit) prefetch_l2(acc + o, (unsigned)(D * sizeof(float)));
+            else prefetch_l2(tokens + o, (unsigned)(D * sizeof(T)));
+        }
         __syncthreads();
 
         // ---- similarity pass: one warp per cell, norm of v_j and dot with its successor
