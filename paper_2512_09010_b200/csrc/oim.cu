@@ -137,7 +137,7 @@ __global__ void oim_setup_kernel(int32_t* cell, int32_t* size, int32_t* parent, 
     }
 }
 
-// MINB: CTAs per SM the register budget is cut for (3: 80 registers, 4: 64 registers).
+// MINB: CTAs per SM the register budget is cut for.
 template <typename T, int NCHUNK, int MINB, int THREADS>
 __global__ void __launch_bounds__(THREADS, MINB) oim_chain_kernel(const ChainArgs a) {
     constexpr int kThreads = THREADS, kWarps = THREADS / 32;
@@ -511,15 +511,15 @@ static cudaError_t launch_chain_b(const ChainArgs& a, int max_len, int r, cudaSt
 }
 
 // Short lines leave a CTA mostly in its serial phases (ranking, merging, waiting for the image's
-// previous step): more resident CTAs overlap them.  Long lines are dominated by the streaming pass,
-// where the larger register budget wins; beyond about a hundred cells a line keeps sixteen warps
-// busy, and two CTAs of 512 threads finish each line sooner than three of 256 (a batch of few large
-// images has fewer lines per step than the GPU has CTA slots, so the time per line is what counts).
-// The switch points are measured (36-, 72- and 128-cell lines).
+// previous step): more resident CTAs overlap them.  Longer lines are dominated by the streaming
+// pass: three CTAs of ten warps per SM (64 registers) do best at 72 cells, and beyond about a
+// hundred cells a line keeps sixteen warps busy, so two CTAs of 512 threads finish each line sooner
+// (a batch of few large images has fewer lines per step than the GPU has CTA slots, so the time per
+// line is what counts).  The switch points are measured (36-, 72- and 128-cell lines).
 template <typename T, int NCHUNK>
 static cudaError_t launch_chain(const ChainArgs& a, int max_len, int r, cudaStream_t stream) {
     if (max_len <= 48) return launch_chain_b<T, NCHUNK, 4>(a, max_len, r, stream);
-    if (max_len <= 96) return launch_chain_b<T, NCHUNK, 3>(a, max_len, r, stream);
+    if (max_len <= 96) return launch_chain_b<T, NCHUNK, 3, 320>(a, max_len, r, stream);
     return launch_chain_b<T, NCHUNK, 2, 512>(a, max_len, r, stream);
 }
 
