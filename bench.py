@@ -35,7 +35,7 @@ HBM_FALLBACK_GBS = 6650.0     # used only if MEASURED_PEAKS.json is absent
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (null until a capture for that workload exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {2: 1.088e9 + 0.135e9}     # profiles/oim_chain_kernel_configs2.txt
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {2: 1.428e9 + 0.140e9}     # profiles/oim_chain_kernel_configs2.txt
 
 
 def parse_args():
