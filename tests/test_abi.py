@@ -86,6 +86,10 @@ def test_argument_errors_are_reported_before_any_device_work(luvc):
     assert L.luvc_spu_prune_ex(fake, 1, 8, 8, 2.0, 2, fake, fake, ctypes.byref(s)) == 5             # cutoff
     assert L.luvc_spu_prune_ex(fake, 1, 8, 4, 0.5, 2, fake, fake, ctypes.byref(s)) == 6             # 8-byte rows
     assert L.luvc_oim_workspace_bytes(1, 24, 24, 1024, 0) >= 576 * 1024 * 4
+    assert L.luvc_oim_workspace_bytes_ex(1, 24, 24, 1024, 0, 0) == L.luvc_oim_workspace_bytes(1, 24, 24, 1024, 0)
+    # the bipartite matching also keeps a bf16 hi + lo copy of every row and a norm per token
+    assert L.luvc_oim_workspace_bytes_ex(1, 24, 24, 1024, 0, 1) >= L.luvc_oim_workspace_bytes(1, 24, 24, 1024, 0) + 576 * 1024 * 4
+    assert L.luvc_oim_workspace_bytes_ex(1, 24, 24, 1024, 0, 7) == 0
     assert L.luvc_spu_workspace_bytes(1, 144, 4096, 0.0, 0) > 0
 
 

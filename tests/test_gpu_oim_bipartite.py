@@ -97,3 +97,18 @@ def test_large_configurations_sampled_replay_and_invariants(luvc, oracle_mod, co
     Hf, Wf, _ = luvc.oim_plan(c["H"], c["W"], c["target"])
     check_oim_invariants(xh, got[0], got[1], got[2], c["dtype"], (c["H"], c["W"]), (Hf, Wf), local=False)
     check_oim_against_oracle(oracle_mod, xh, *got, c["dtype"], target=c["target"], images=[0], matching="bipartite")
+
+
+def test_caller_workspace_needs_the_larger_size(luvc):
+    g = torch.Generator().manual_seed(27)
+    x = torch.randn((1, 6, 6, 16), generator=g).cuda()
+    small = luvc.lib.luvc_oim_workspace_bytes(1, 6, 6, 16, luvc.F32)
+    need = luvc.lib.luvc_oim_workspace_bytes_ex(1, 6, 6, 16, luvc.F32, 1)
+    assert need > small
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    a = luvc.oim_merge(x, 9, workspace=ws, matching="bipartite")
+    b = luvc.oim_merge(x, 9, matching="bipartite")
+    assert all(torch.equal(u, v) for u, v in zip(a, b))
+    with pytest.raises(luvc.LuvcError) as e:
+        luvc.oim_merge(x, 9, workspace=ws[:small], matching="bipartite")
+    assert luvc.STATUS_NAMES[e.value.status] == "LUVC_ERR_WORKSPACE"
