@@ -79,6 +79,8 @@ def test_argument_errors_are_reported_before_any_device_work(luvc):
     assert L.luvc_oim_merge_ex(fake, 1, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 2         # unknown matching
     o.matching = 1
     assert L.luvc_oim_merge_ex(fake, 1, 2, 258, 8, 258, fake, fake, fake, ctypes.byref(o)) == 2     # bipartite line > 256
+    o.dtype = 1
+    assert L.luvc_oim_merge_ex(fake, 1, 4, 4, 12, 4, fake, fake, fake, ctypes.byref(o)) == 6        # bipartite: D % 8 != 0
     s = luvc.SpuOpts()
     assert L.luvc_spu_prune_ex(None, 1, 8, 8, 0.5, 2, None, None, ctypes.byref(s)) == 1
     assert L.luvc_spu_prune_ex(fake, 1, 8, 8, 0.5, 9, fake, fake, ctypes.byref(s)) == 4             # keep > N

@@ -144,3 +144,15 @@ def test_value_enhancement_bias(luvc, oracle_mod):
         tok2 = tok.clone()
         luvc.oim_value_enhance(tok2, sizes, out=tok2)
         assert torch.equal(tok2, enhanced)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_results_repeat_bit_for_bit(luvc, dtype):
+    # no float atomics and a fixed summation order everywhere: the same call gives the same bits,
+    # whichever CTA happens to take which line
+    g = torch.Generator().manual_seed(34)
+    x = torch.randn((3, 40, 36, 200), generator=g).to(dtype).cuda()
+    first = luvc.oim_merge(x, 20 * 18, want_trace=True)
+    for _ in range(4):
+        again = luvc.oim_merge(x, 20 * 18, want_trace=True)
+        assert all(torch.equal(u, v) for u, v in zip(first, again))

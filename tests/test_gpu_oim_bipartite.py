@@ -112,3 +112,15 @@ def test_caller_workspace_needs_the_larger_size(luvc):
     with pytest.raises(luvc.LuvcError) as e:
         luvc.oim_merge(x, 9, workspace=ws[:small], matching="bipartite")
     assert luvc.STATUS_NAMES[e.value.status] == "LUVC_ERR_WORKSPACE"
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_results_repeat_bit_for_bit(luvc, dtype):
+    # no float atomics and a fixed summation order everywhere: the same call gives the same bits,
+    # whichever CTA happens to take which line
+    g = torch.Generator().manual_seed(33)
+    x = torch.randn((3, 40, 36, 200), generator=g).to(dtype).cuda()
+    first = luvc.oim_merge(x, 20 * 18, want_trace=True, matching="bipartite")
+    for _ in range(4):
+        again = luvc.oim_merge(x, 20 * 18, want_trace=True, matching="bipartite")
+        assert all(torch.equal(u, v) for u, v in zip(first, again))
