@@ -186,7 +186,11 @@ int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target
 
 /* Same operator on HOST buffers (pinned memory recommended): copies the tokens to
  * the device, runs, copies the three outputs back and synchronises the stream
- * before returning.  dtype is a luvc_dtype. */
+ * before returning.  dtype is a luvc_dtype.  The staging buffers belong to the
+ * library and are separate for luvc_oim_merge_host and luvc_spu_prune_host: one
+ * call of each may run at the same time from two host threads, each on its own
+ * luvc stream (the copies of one then overlap the other's work); two calls of the
+ * same entry point must not overlap. */
 int luvc_oim_merge_host(const void* tokens, int B, int H, int W, int D, int target_count, int dtype,
                         void* out_tokens, int32_t* out_sizes, int32_t* out_map);
 

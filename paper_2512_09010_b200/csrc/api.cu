@@ -42,7 +42,7 @@ thread_local cudaStream_t t_stream = nullptr;
 // Library-owned scratch: one growing buffer per purpose, shared by all threads.
 // Calls that use it from several host threads at once must use different streams'
 // work serially; the plain entry points take this lock only while (re)allocating.
-enum Slot { kOimWs = 0, kSpuWs, kIoIn, kIoOut, kStatus, kCascade, kSlots };
+enum Slot { kOimWs = 0, kSpuWs, kIoIn, kIoOut, kStatus, kCascade, kIoInSpu, kIoOutSpu, kSlots };
 struct Scratch { void* ptr = nullptr; size_t bytes = 0; };
 Scratch g_scratch[kSlots];
 std::mutex g_mutex;
@@ -386,8 +386,8 @@ int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, i
     if (keep < 1 || keep > N) return LUVC_ERR_KEEP;
     const size_t es = elem_size(dtype);
     const size_t in_bytes = (size_t)B * N * D * es, hid_bytes = align_up((size_t)B * keep * D * es);
-    unsigned char* din = static_cast<unsigned char*>(scratch(kIoIn, in_bytes));
-    unsigned char* dout = static_cast<unsigned char*>(scratch(kIoOut, hid_bytes + align_up((size_t)B * keep * 4)));
+    unsigned char* din = static_cast<unsigned char*>(scratch(kIoInSpu, in_bytes));
+    unsigned char* dout = static_cast<unsigned char*>(scratch(kIoOutSpu, hid_bytes + align_up((size_t)B * keep * 4)));
     if (!din || !dout) return LUVC_ERR_CUDA;
     cudaStream_t st = t_stream;
     if (cudaMemcpyAsync(din, hidden, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return LUVC_ERR_CUDA;

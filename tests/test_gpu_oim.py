@@ -128,6 +128,39 @@ def test_host_buffer_entry_point(luvc, oracle_mod):
     assert torch.equal(tok, ref[0].cpu()) and torch.equal(sizes, ref[1].cpu()) and torch.equal(mp, ref[2].cpu())
 
 
+def test_the_two_host_entry_points_may_run_at_the_same_time(luvc):
+    # separate staging buffers: an OIM host call and an SPU host call from two host threads, each on
+    # its own stream, must give what they give one after the other
+    import concurrent.futures
+    g = torch.Generator().manual_seed(18)
+    x = torch.randn((4, 24, 24, 256), generator=g).to(torch.bfloat16).pin_memory()
+    y = torch.randn((4, 512, 1024), generator=g).to(torch.bfloat16).pin_memory()
+
+    def outputs():
+        return (torch.empty((4, 144, 256), dtype=torch.bfloat16).pin_memory(), torch.empty((4, 144), dtype=torch.int32).pin_memory(),
+                torch.empty((4, 576), dtype=torch.int32).pin_memory(), torch.empty((4, 128), dtype=torch.int32).pin_memory(),
+                torch.empty((4, 128, 1024), dtype=torch.bfloat16).pin_memory())
+
+    ref = outputs()
+    luvc.oim_merge_host(x, 144, ref[0], ref[1], ref[2])
+    luvc.spu_prune_host(y, 128, 0.125, ref[3], ref[4])
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+
+    def on(stream, fn, *args):
+        torch.cuda.set_device(0)
+        with torch.cuda.stream(stream):
+            fn(*args)
+
+    with concurrent.futures.ThreadPoolExecutor(max_workers=2) as pool:
+        for _ in range(5):
+            got = outputs()
+            jobs = [pool.submit(on, streams[0], luvc.oim_merge_host, x, 144, got[0], got[1], got[2]),
+                    pool.submit(on, streams[1], luvc.spu_prune_host, y, 128, 0.125, got[3], got[4])]
+            for job in jobs:
+                job.result()
+            assert all(torch.equal(u, v) for u, v in zip(got, ref))
+
+
 def test_value_enhancement_bias(luvc, oracle_mod):
     # Eq. 2: V + log s.  log s as an optional output of the merge, and the row-wise add as its own call
     g = torch.Generator().manual_seed(11)
