@@ -176,8 +176,10 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
     const uint32_t stages_base = smem_u32(smem_raw);
     unsigned char* tail = smem_raw + (size_t)cfg.n_stages * cfg.stage_stride + kSlack;
     const __nv_bfloat16** s_hi = reinterpret_cast<const __nv_bfloat16**>(tail);   // [len] hi part of tile row
-    const __nv_bfloat16** s_lo = s_hi + cfg.max_len;                              // [len] lo part, or null (all zero)
-    float* s_rn = reinterpret_cast<float*>(s_lo + cfg.max_len);                   // [len] 1 / |v| by tile row (A rows, then B rows)
+    // [len] where the row's first piece goes inside a stage (| 1: the row has a lo part, behind its hi part;
+    // | 2: A row) and the byte distance between its pieces
+    uint2* s_where = reinterpret_cast<uint2*>(s_hi + cfg.max_len);
+    float* s_rn = reinterpret_cast<float*>(s_where + cfg.max_len);                   // [len] 1 / |v| by tile row (A rows, then B rows)
     unsigned* s_root = reinterpret_cast<unsigned*>(s_rn + cfg.max_len);           // [len] root | merged bit by position
     float* s_score = reinterpret_cast<float*>(s_root + cfg.max_len);              // [na] best cosine of A cell i
     int* s_dst = reinterpret_cast<int*>(s_score + (cfg.max_len + 1) / 2);         // [na] position of its best B cell
@@ -256,14 +258,15 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
             s_root[j] = r;
             const int id = (int)(r & ~kMergedBit);
             const bool parts = sizeof(T) == 4 || (r & kMergedBit) != 0;
-            const int row = (j & 1) ? g.na + (j >> 1) : (j >> 1);
-            const __nv_bfloat16* hi = parts ? split + (size_t)id * 2 * D
-                                            : reinterpret_cast<const __nv_bfloat16*>(tokens + (size_t)id * D);
-            s_hi[row] = hi;
-            s_lo[row] = parts ? hi + D : nullptr;
+            const bool is_a = !(j & 1);
+            const int rr = j >> 1, row = is_a ? rr : g.na + rr;
+            s_hi[row] = parts ? split + (size_t)id * 2 * D : reinterpret_cast<const __nv_bfloat16*>(tokens + (size_t)id * D);
+            s_where[row] = make_uint2((uint32_t)((is_a ? 0 : g.off_b) + (rr >> 3) * 128 + (rr & 7) * 16) | (parts ? 1u : 0u) |
+                                          (is_a ? 2u : 0u),
+                                      (uint32_t)(is_a ? g.lbo_a : g.lbo_b));
             const float nn = __ldcg(nrm2 + id);
             s_rn[row] = nn > 0.f ? 1.0f / sqrtf(nn) : 0.f;          // a zero vector has similarity 0 with everything
-            if (parts) { if (j & 1) m_b = true; else m_a = true; }
+            if (parts) { if (is_a) m_a = true; else m_b = true; }
         }
         const bool lo_a = __syncthreads_or(m_a) != 0;
         const bool lo_b = __syncthreads_or(m_b) != 0;
@@ -277,6 +280,8 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
         if (warp < kWarps) {
             // loaders: tile c of this line goes to stage (fill0 + c) % S once the MMAs that last read it are done
             const int total_q = len * kPieces;
+            const uint32_t lo_off_a = lo_a ? (uint32_t)(g.ra >> 3) * 128 : 0u;   // the lo row sits ra (rb) rows below the hi row;
+            const uint32_t lo_off_b = lo_b ? (uint32_t)(g.rb >> 3) * 128 : 0u;   // 0: that operand has no lo half in this line
             int issued = 0;
             for (int kc = 0; kc < nkc; ++kc) {
                 while (issued < nkc && issued <= kc + cfg.ahead) {
@@ -289,18 +294,16 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
                     const uint32_t sb = stages_base + stage * (uint32_t)cfg.stage_stride;
                     for (int q = tid; q < total_q; q += kLoaders) {
                         const int row = q >> 3, piece = q & 7;
-                        const int e = issued * kKC + piece * 8;
-                        const bool valid = e < D;
-                        const bool is_a = row < g.na;
-                        const int rr = is_a ? row : row - g.na;
-                        const uint32_t dst = sb + (is_a ? 0 : g.off_b) + piece * (is_a ? g.lbo_a : g.lbo_b) +
-                                             (rr >> 3) * 128 + (rr & 7) * 16;
+                        const bool valid = issued * kKC + piece * 8 < D;
+                        const uint2 w = s_where[row];
                         const __nv_bfloat16* hi = s_hi[row];
-                        cp_async16(dst, valid ? hi + e : hi, valid);
-                        if (is_a ? lo_a : lo_b) {                  // the lo row sits ra (rb) rows below the hi row
-                            const __nv_bfloat16* lo = s_lo[row];
-                            const bool have = valid && lo != nullptr;
-                            cp_async16(dst + ((is_a ? g.ra : g.rb) >> 3) * 128, have ? lo + e : hi, have);
+                        const __nv_bfloat16* src = hi + (issued * kKC + piece * 8);
+                        const uint32_t dst = sb + (w.x & ~15u) + piece * w.y;
+                        cp_async16(dst, valid ? src : hi, valid);
+                        const uint32_t lo_off = (w.x & 2u) ? lo_off_a : lo_off_b;
+                        if (lo_off) {
+                            const bool have = valid && (w.x & 1u);
+                            cp_async16(dst + lo_off, have ? src + D : hi, have);
                         }
                     }
                     cp_async_commit();
