@@ -185,6 +185,8 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
     int* s_dst = reinterpret_cast<int*>(s_score + (cfg.max_len + 1) / 2);         // [na] position of its best B cell
     int* s_sel = s_dst + (cfg.max_len + 1) / 2;                                   // [m] (A position << 16) | B position
     float* s_part = reinterpret_cast<float*>(s_sel + cfg.r + 8);                  // partial squared norms of the new sums
+    float* s_score2 = s_part + cfg.r + 8 + kWarps;                                // [na] candidate of the second warp of a quadrant
+    int* s_dst2 = reinterpret_cast<int*>(s_score2 + (cfg.max_len + 1) / 2);
     float* s_S = reinterpret_cast<float*>(smem_raw);   // lo-row block of the product; the stages are idle when it is used
 
     const uint32_t bar0 = smem_u32(&s_bar[0]);
@@ -353,11 +355,13 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
 
         // ---- with both halves of A in one MMA, the lo rows' block (A lo x B hi) goes through shared memory
         const int ld_s = g.rb + 1;
-        if (lo_a && stack_m && warp < 4 && warp * 32 < 2 * g.ra && warp * 32 + 32 > g.ra) {
-            const int i = warp * 32 + lane - g.ra;
-            for (int c0 = 0; c0 < g.rb; c0 += 16) {
+        // Two warps share each quadrant of TMEM lanes (warp & 3) and take alternate 16-column chunks (warp >> 2).
+        const int quad = warp & 3, half = (warp >> 2) & 1;
+        if (lo_a && stack_m && warp < kWarps && quad * 32 < 2 * g.ra && quad * 32 + 32 > g.ra) {
+            const int i = quad * 32 + lane - g.ra;
+            for (int c0 = half * 16; c0 < g.rb; c0 += 32) {
                 uint32_t v[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
                 tmem_ld_wait_for(v);
                 if (i >= 0 && i < g.na) {
 #pragma unroll
@@ -369,16 +373,16 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
         __syncthreads();
 
         // ---- proposals: A row i (TMEM lane i) keeps the first maximum of its cosines
-        if (warp < 4 && warp * 32 < g.na) {
-            const int i = warp * 32 + lane;
+        if (warp < kWarps && quad * 32 < g.na) {
+            const int i = quad * 32 + lane;
             const float rn_i = i < g.na ? s_rn[i] : 0.f;
             const bool add_s = lo_a && stack_m && i < g.na;
             float best = -INFINITY;
             int best_j = 0;
-            for (int c0 = 0; c0 < g.rb; c0 += 16) {
+            for (int c0 = half * 16; c0 < g.rb; c0 += 32) {
                 uint32_t v[16], w[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                if (lo_b) tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(g.rb + c0), w);
+                tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
+                if (lo_b) tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(g.rb + c0), w);
                 tmem_ld_wait_for(v);
                 if (lo_b) tmem_ld_wait_for(w);
 #pragma unroll
@@ -394,13 +398,22 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
                     }
                 }
             }
-            if (i < g.na) { s_score[i] = best; s_dst[i] = 2 * best_j + 1; }
+            if (i < g.na) {                     // this warp's candidate; warp 0 joins the two halves below
+                (half ? s_score2 : s_score)[i] = best;
+                (half ? s_dst2 : s_dst)[i] = 2 * best_j + 1;
+            }
         }
         tc_fence_before();
         __syncthreads();
 
         // ---- ranking: warp 0 takes the m best proposals (ties: the lowest A position)
         if (warp == 0) {
+            for (int c = lane; c < g.na; c += 32) {      // first maximum over both halves: the larger cosine, then the lower position
+                const float s2 = s_score2[c];
+                const int d2 = s_dst2[c];
+                if (s2 > s_score[c] || (s2 == s_score[c] && d2 < s_dst[c])) { s_score[c] = s2; s_dst[c] = d2; }
+            }
+            __syncwarp();
             for (int k = 0; k < st.m; ++k) {
                 float best = -INFINITY;
                 int best_c = 0x7fffffff;
@@ -528,7 +541,7 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
 
 size_t tail_bytes(int max_len, int r) {
     return (size_t)max_len * (8 + 8 + 4 + 4) + (size_t)((max_len + 1) / 2) * 8 + (size_t)(r + 8) * 4 +
-           (size_t)(r + 8 + kWarps) * 4;
+           (size_t)(r + 8 + kWarps) * 4 + (size_t)((max_len + 1) / 2) * 8;
 }
 
 template <typename T>
