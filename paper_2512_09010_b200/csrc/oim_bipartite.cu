@@ -13,11 +13,12 @@
 //   * eight loader warps gather the line's rows through the cell grid with cp.async, 16 bytes
 //     at a time, straight into K-major operand tiles of 64 channels, several tiles in flight;
 //     the lo rows of an operand sit below its hi rows in the same tile;
-//   * a ninth warp issues tcgen05.mma (fp32 accumulation in TMEM): [A hi; A lo] x [B hi; B lo]^T
-//     is one instruction per 16 channels when both halves of A fit the 128 rows of the MMA, two
-//     otherwise; parts that are zero for the whole line are left out;
-//   * the rows of the product are read back with tcgen05.ld, the hi/lo blocks added, scaled to
-//     cosines, and each A row keeps its first maximum.
+//   * a ninth warp issues tcgen05.mma (fp32 accumulation in TMEM), per 16 channels A hi x B hi^T and,
+//     into the same accumulator, A lo x B hi^T and A hi x B lo^T; a part that is zero for the whole
+//     line is left out.  (One instruction on stacked operands, [A hi; A lo] x [B hi; B lo]^T, was
+//     slower: its blocks have to be added after the read-back, across TMEM lanes.)
+//   * the rows of the product are read back with tcgen05.ld by the two warps of each lane quadrant,
+//     scaled to cosines, and each A row keeps its first maximum.
 // Loaders and the issuing warp meet only through mbarriers (tile landed / tile consumed).
 //
 // Ranking, the size-weighted merge and the compaction of the line follow; the data layout, the
@@ -154,7 +155,7 @@ struct BipartiteLaunch {
     int n_stages;       // operand stages in shared memory (1 .. kMaxStages)
     int ahead;          // tiles requested ahead of the one whose arrival is awaited (0 .. n_stages - 1)
     int stage_stride;   // bytes between stages (the geometry of the longest line)
-    int tmem_cols;      // power of two >= 32 covering the widest product
+    int tmem_cols;      // power of two >= 32 covering the widest similarity matrix
     int max_len, r;
     __nv_bfloat16* split;   // [B][HW][2][D] bf16 hi and lo parts of fp32 rows
     float* nrm2;            // [B][HW] squared norm by root
@@ -187,7 +188,6 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
     float* s_part = reinterpret_cast<float*>(s_sel + cfg.r + 8);                  // partial squared norms of the new sums
     float* s_score2 = s_part + cfg.r + 8 + kWarps;                                // [na] candidate of the second warp of a quadrant
     int* s_dst2 = reinterpret_cast<int*>(s_score2 + (cfg.max_len + 1) / 2);
-    float* s_S = reinterpret_cast<float*>(smem_raw);   // lo-row block of the product; the stages are idle when it is used
 
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     const uint32_t bar_acc = bar0 + 8 * (2 * kMaxStages);
@@ -273,11 +273,9 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
         const bool lo_a = __syncthreads_or(m_a) != 0;
         const bool lo_b = __syncthreads_or(m_b) != 0;
 
-        // ---- the product [A hi; A lo] x [B hi; B lo]^T over tiles of 64 channels
+        // ---- the similarity matrix A B^T (hi and lo parts) over tiles of 64 channels
         const int nkc = (D + kKC - 1) / kKC;
         const unsigned fill0 = fills;
-        // both halves of A inside the MMA's 128 rows, and room for the lo-row block in the idle stages
-        const bool stack_m = 2 * g.ra <= 128 && (size_t)g.ra * (g.rb + 1) * 4 <= (size_t)S * cfg.stage_stride;
 
         if (warp < kWarps) {
             // loaders: tile c of this line goes to stage (fill0 + c) % S once the MMAs that last read it are done
@@ -319,9 +317,8 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
         } else {
             // issuing warp: lane 0 works, the others wait at the warp barriers (a lane that spun on the
             // product barrier beside the issuing lane would take its issue slots)
-            const uint32_t idesc1 = make_idesc_bf16(128, lo_b ? 2 * g.rb : g.rb, false, false);
-            const uint32_t idesc2 = make_idesc_bf16(128, g.rb, false, false);
-            const bool second = lo_a && !stack_m;          // A lo x B hi as an instruction of its own
+            // hi x hi, then lo x hi and hi x lo where the line has lo parts: all into the same columns
+            const uint32_t idesc = make_idesc_bf16(128, g.rb, false, false);
             for (int kc = 0; kc < nkc; ++kc) {
                 const unsigned f = fill0 + (unsigned)kc;
                 const unsigned stage = f % S, use = f / S;
@@ -332,11 +329,14 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
                     if (!s_fail) {
 #pragma unroll
                         for (int ks = 0; ks < kKC / 16; ++ks) {
-                            const uint64_t b1 = make_desc(sb + g.off_b + ks * 2 * g.lbo_b, g.lbo_b, 128);
-                            umma_bf16(tmem, make_desc(sb + ks * 2 * g.lbo_a, g.lbo_a, 128), b1, idesc1, (kc | ks) ? 1u : 0u);
-                            if (second)
-                                umma_bf16(tmem, make_desc(sb + ks * 2 * g.lbo_a + (g.ra >> 3) * 128, g.lbo_a, 128), b1, idesc2,
-                                          1u);
+                            const uint64_t a_hi = make_desc(sb + ks * 2 * g.lbo_a, g.lbo_a, 128);
+                            const uint64_t b_hi = make_desc(sb + g.off_b + ks * 2 * g.lbo_b, g.lbo_b, 128);
+                            umma_bf16(tmem, a_hi, b_hi, idesc, (kc | ks) ? 1u : 0u);
+                            if (lo_a)
+                                umma_bf16(tmem, make_desc(sb + ks * 2 * g.lbo_a + (g.ra >> 3) * 128, g.lbo_a, 128), b_hi, idesc, 1u);
+                            if (lo_b)
+                                umma_bf16(tmem, a_hi, make_desc(sb + g.off_b + ks * 2 * g.lbo_b + (g.rb >> 3) * 128, g.lbo_b, 128),
+                                          idesc, 1u);
                         }
                     }
                     umma_commit(bar0 + 8 * (kMaxStages + stage));
@@ -353,46 +353,24 @@ __global__ void __launch_bounds__(kThreads, 3) oim_bipartite_kernel(const ChainA
         ++items_done;
         tc_fence_after();
 
-        // ---- with both halves of A in one MMA, the lo rows' block (A lo x B hi) goes through shared memory
-        const int ld_s = g.rb + 1;
         // Two warps share each quadrant of TMEM lanes (warp & 3) and take alternate 16-column chunks (warp >> 2).
         const int quad = warp & 3, half = (warp >> 2) & 1;
-        if (lo_a && stack_m && warp < kWarps && quad * 32 < 2 * g.ra && quad * 32 + 32 > g.ra) {
-            const int i = quad * 32 + lane - g.ra;
-            for (int c0 = half * 16; c0 < g.rb; c0 += 32) {
-                uint32_t v[16];
-                tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
-                tmem_ld_wait_for(v);
-                if (i >= 0 && i < g.na) {
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj)
-                        if (c0 + jj < g.nb) s_S[i * ld_s + c0 + jj] = __uint_as_float(v[jj]);
-                }
-            }
-        }
-        __syncthreads();
 
         // ---- proposals: A row i (TMEM lane i) keeps the first maximum of its cosines
         if (warp < kWarps && quad * 32 < g.na) {
             const int i = quad * 32 + lane;
             const float rn_i = i < g.na ? s_rn[i] : 0.f;
-            const bool add_s = lo_a && stack_m && i < g.na;
             float best = -INFINITY;
             int best_j = 0;
             for (int c0 = half * 16; c0 < g.rb; c0 += 32) {
-                uint32_t v[16], w[16];
+                uint32_t v[16];
                 tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
-                if (lo_b) tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(g.rb + c0), w);
                 tmem_ld_wait_for(v);
-                if (lo_b) tmem_ld_wait_for(w);
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) {
                     const int j = c0 + jj;
                     if (j < g.nb) {
-                        float d = __uint_as_float(v[jj]);                   // hi x hi
-                        if (lo_b) d += __uint_as_float(w[jj]);              // + hi x lo
-                        if (add_s) d += s_S[i * ld_s + j];                  // + lo x hi
-                        float c = d * (rn_i * s_rn[g.na + j]);
+                        float c = __uint_as_float(v[jj]) * (rn_i * s_rn[g.na + j]);
                         if (!(c == c)) c = -FLT_MAX;
                         if (c > best) { best = c; best_j = j; }
                     }
@@ -563,7 +541,7 @@ cudaError_t launch_typed(const ChainArgs& a, __nv_bfloat16* split, float* nrm2, 
     cfg.nrm2 = nrm2;
     cfg.stage_stride = (line_geom(max_len).stage_bytes + 127) & ~127;
     int cols = 32;
-    while (cols < 2 * line_geom(max_len).rb) cols <<= 1;
+    while (cols < line_geom(max_len).rb) cols <<= 1;
     cfg.tmem_cols = cols;
     const size_t fixed = kSlack + tail_bytes(max_len, r) + 128;
     // CTAs per SM: the occupancy query of the runtime answers 1 for a kernel that allocates tensor
