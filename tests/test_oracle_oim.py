@@ -231,6 +231,41 @@ def test_replay_accepts_own_trace_and_flags_a_wrong_one(oracle_mod):
     assert flagged["stats"][0, 2] > 0
 
 
+def _line_of_unit_vectors(angles):
+    """One row of 2-D unit vectors at the given angles: the cosine of two cells is cos(angle difference)."""
+    a = np.asarray(angles, dtype=np.float64)
+    return np.stack([np.cos(a), np.sin(a)], axis=-1).astype(np.float32)[None, None]      # [1, 1, len, 2]
+
+
+def test_replay_selection_rule_on_a_line_with_known_margins(oracle_mod):
+    # Section 3.2's matching on one line of seven cells.  Even cells and their best neighbour:
+    #   cell 0 -> right, cos 0.1 = 0.99500;  cell 2 -> right, cos 0.3 = 0.95534 (left: cos 0.4)
+    #   cell 4 -> right, cos 0.5 = 0.87758 (left: cos 0.7);  cell 6 -> left, cos 1.0 = 0.54030
+    x = _line_of_unit_vectors([0.0, 0.1, 0.5, 0.8, 1.5, 2.0, 3.0])
+    own = oracle_mod.oim(x, out_hw=(1, 6))
+    assert own["trace"][0].tolist() == [0 * 2 + 1]
+    np.testing.assert_allclose(own["stats"][0, 0], 0.9950041652780258 - 0.955336489125606, atol=1e-6)
+    # a trace that merges cell 2 instead of cell 0: the chosen score is 0.03967 below the best unchosen one
+    swapped = np.array([[2 * 2 + 1]], np.int32)
+    margin = 0.9950041652780258 - 0.955336489125606
+    strict = oracle_mod.oim(x, out_hw=(1, 6), trace=swapped, tol=margin - 1e-3)
+    assert strict["stats"][0, 2] > 0
+    lenient = oracle_mod.oim(x, out_hw=(1, 6), trace=swapped, tol=margin + 1e-3)
+    assert lenient["stats"][0, 2] == 0 and lenient["stats"][0, 3] > 0          # accepted, but noted as a deviation
+    assert lenient["map"][0].tolist() == [0, 1, 2, 2, 3, 4, 5]                  # and the replay applied the trace's merge
+    # two merges per line: {0, 4} instead of {0, 2}; the margin is cos 0.3 - cos 0.5 = 0.07775
+    own2 = oracle_mod.oim(x, out_hw=(1, 5))
+    assert sorted(own2["trace"][0].tolist()) == [1, 5]
+    swapped2 = np.array([[0 * 2 + 1, 4 * 2 + 1]], np.int32)
+    margin2 = 0.955336489125606 - 0.8775825618903728
+    assert oracle_mod.oim(x, out_hw=(1, 5), trace=swapped2, tol=margin2 - 1e-3)["stats"][0, 2] > 0
+    assert oracle_mod.oim(x, out_hw=(1, 5), trace=swapped2, tol=margin2 + 1e-3)["stats"][0, 2] == 0
+    # the same swap along the other axis (a single column)
+    xt = np.ascontiguousarray(x.transpose(0, 2, 1, 3))
+    assert oracle_mod.oim(xt, out_hw=(6, 1), trace=swapped, tol=margin - 1e-3)["stats"][0, 2] > 0
+    assert oracle_mod.oim(xt, out_hw=(6, 1), trace=swapped, tol=margin + 1e-3)["stats"][0, 2] == 0
+
+
 def test_config0_shapes_and_near_ties(oracle_mod):
     x = gi.oim_input(0).numpy()
     r = oracle_mod.oim(x, target=144)
@@ -248,3 +283,10 @@ def test_value_enhancement_is_the_log_of_the_size(oracle_mod):
     np.testing.assert_allclose(e[0, 0], v[0, 0])                      # log 1 = 0
     np.testing.assert_allclose(e[0, 1] - v[0, 1], np.log(4.0))
     np.testing.assert_allclose(np.exp(e - v)[0, :, 0], s[0])          # the bias exponentiates back to the size
+    # hand values of Eq. 2's bias: ln 2, ln 3, ln 4 typed in
+    v = np.zeros((1, 4, 1))
+    e = oracle_mod.oim_value_enhance(v, np.array([[1, 2, 3, 4]]))
+    np.testing.assert_allclose(e[0, :, 0], [0.0, 0.6931471805599453, 1.0986122886681098, 1.3862943611198906],
+                               rtol=0, atol=1e-15)
+    e = oracle_mod.oim_value_enhance(np.array([[[-0.25, 7.0]]]), np.array([[4]]))
+    np.testing.assert_allclose(e[0, 0], [1.1362943611198906, 8.386294361119891], rtol=0, atol=1e-15)

@@ -154,3 +154,32 @@ def test_replay_accepts_own_trace_and_flags_a_wrong_one(oracle_mod):
     malformed = run["trace"].copy()
     malformed[0][0] = (1 << 16) | 1                                # an odd source
     assert oracle_mod.oim(x, target=9, trace=malformed, matching="bipartite")["stats"][0, 2] > 0
+
+
+def test_replay_selection_rule_on_a_line_with_known_margins(oracle_mod):
+    # one line of 2-D unit vectors at angles 0, 0.1, 0.5, 0.8, 1.5, 2.0, 3.0: an even cell's proposal
+    # over ALL odd cells.  cell 0 -> cell 1 (cos 0.1);  cell 2 -> cell 3 (cos 0.3; cell 1: cos 0.4);
+    # cell 4 -> cell 5 (cos 0.5; cell 3: cos 0.7);  cell 6 -> cell 5 (cos 1.0)
+    a = np.array([0.0, 0.1, 0.5, 0.8, 1.5, 2.0, 3.0])
+    x = np.stack([np.cos(a), np.sin(a)], axis=-1).astype(np.float32)[None, None]
+    own = oracle_mod.oim(x, out_hw=(1, 6), matching="bipartite")
+    assert own["trace"][0].tolist() == [(0 << 16) | 1]
+    margin = 0.9950041652780258 - 0.955336489125606           # cos 0.1 - cos 0.3
+    np.testing.assert_allclose(own["stats"][0, 0], margin, atol=1e-6)
+    swapped = np.array([[(2 << 16) | 3]], np.int32)            # merges cell 2 although cell 0 scores higher
+    strict = oracle_mod.oim(x, out_hw=(1, 6), trace=swapped, tol=margin - 1e-3, matching="bipartite")
+    assert strict["stats"][0, 2] > 0
+    lenient = oracle_mod.oim(x, out_hw=(1, 6), trace=swapped, tol=margin + 1e-3, matching="bipartite")
+    assert lenient["stats"][0, 2] == 0 and lenient["stats"][0, 3] > 0
+    assert lenient["map"][0].tolist() == [0, 1, 2, 2, 3, 4, 5]
+    # two merges: {0, 4} instead of {0, 2}, margin cos 0.3 - cos 0.5
+    swapped2 = np.array([[(0 << 16) | 1, (4 << 16) | 5]], np.int32)
+    margin2 = 0.955336489125606 - 0.8775825618903728
+    assert oracle_mod.oim(x, out_hw=(1, 5), trace=swapped2, tol=margin2 - 1e-3, matching="bipartite")["stats"][0, 2] > 0
+    assert oracle_mod.oim(x, out_hw=(1, 5), trace=swapped2, tol=margin2 + 1e-3, matching="bipartite")["stats"][0, 2] == 0
+    # a proposal that is not the cell's best one: cell 2 into cell 1 (cos 0.4) instead of cell 3 (cos 0.3)?
+    # cos 0.4 = 0.92106 < cos 0.3: 0.03428 below the best, so it is a violation below that and accepted above
+    worse = np.array([[(0 << 16) | 1, (2 << 16) | 1]], np.int32)
+    gap = 0.955336489125606 - 0.9210609940028851
+    assert oracle_mod.oim(x, out_hw=(1, 5), trace=worse, tol=gap - 1e-3, matching="bipartite")["stats"][0, 2] > 0
+    assert oracle_mod.oim(x, out_hw=(1, 5), trace=worse, tol=gap + 1e-3, matching="bipartite")["stats"][0, 2] == 0
