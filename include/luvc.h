@@ -25,10 +25,16 @@
  *     (D % 8 == 0 for bf16, D % 4 == 0 for fp32), else LUVC_ERR_ALIGN.
  *   - Device calls are asynchronous on the calling thread's luvc stream (see
  *     luvc_set_stream) and do not synchronise the host.
- *   - The plain entry points use a library-owned scratch buffer that grows with
- *     cudaMalloc on demand (a host-synchronous call the first time a larger
- *     problem is seen) and is released by luvc_shutdown().  The _ex entry points
- *     use only the caller's workspace when one is given.
+ *   - The plain entry points use library-owned scratch buffers, one set per
+ *     device (keyed by the ordinal of the device that is current at the call),
+ *     grown with cudaMalloc on demand (a host-synchronous call the first time a
+ *     larger problem is seen) and released by luvc_shutdown().  All calls on a
+ *     device share that one set: two calls whose GPU work overlaps (two streams,
+ *     or two host threads) race on it and give undefined results - keep them on
+ *     one stream, order them with events, or give each its own workspace through
+ *     the _ex forms.  An _ex call that is given a workspace uses only that
+ *     workspace; given a device_status word as well it touches no library-owned
+ *     memory at all.
  */
 #ifndef LUVC_H_
 #define LUVC_H_
@@ -75,13 +81,21 @@ int luvc_set_stream(void* cuda_stream);
 
 /* Device-side conditions (a bounded wait inside a kernel that gave up) are written
  * to a status word in device memory instead of trapping.  This call synchronises
- * the given stream, returns that word as a luvc_status (LUVC_OK if nothing was
- * reported) and clears it.  While the word is set, later operator calls stop early;
- * their outputs are then undefined. */
+ * the given stream, returns the current device's library-owned word as a
+ * luvc_status (LUVC_OK if nothing was reported) and clears it.  While a word is
+ * set, operator calls that use it stop early and leave their outputs untouched or
+ * partly written (undefined, but every access stays inside the caller's buffers).
+ * Calls that were given their own word (device_status of the option structs) report
+ * there instead; luvc_read_status reads and clears such a word. */
 int luvc_check_status(void* cuda_stream);
+int luvc_read_status(int32_t* device_status, void* cuda_stream);
 
-/* Frees the library-owned scratch buffers of the current device.  Synchronises
- * the device first.  Safe to call more than once. */
+/* Bytes a caller-owned status block must have (device memory, 16-byte aligned, zeroed
+ * by the caller before its first use; the library only ever writes its first word). */
+#define LUVC_STATUS_BYTES 16
+
+/* Frees the library-owned scratch buffers of the current device (and its status
+ * word).  Synchronises the device first.  Safe to call more than once. */
 int luvc_shutdown(void);
 
 /* Number of kernels this library has launched since it was loaded (all threads). */
@@ -149,10 +163,16 @@ typedef struct {
                                 (position of the merged cell in its line) * 2 + direction
                                 (0 = into the previous cell of the line, 1 = into the next),
                                 ordered by step, line, rank of the candidate */
+    size_t trace_bytes;      /* size of the trace buffer; with trace != NULL it must be at least
+                                B * (H*W - out_h*out_w) * 4, else LUVC_ERR_WORKSPACE (nothing is queued) */
     float* out_log_sizes;    /* optional device [B, target_count] fp32: log(s), the bias that the
                                 value enhancement of Eq. 2 adds to the values (V + log s) */
     int matching;            /* LUVC_OIM_MATCH_ADJACENT (0) or LUVC_OIM_MATCH_BIPARTITE: which cells
                                 of a line are compared (see luvc_oim_matching) */
+    int32_t* device_status;  /* optional device block of LUVC_STATUS_BYTES (see luvc_read_status);
+                                NULL = the library-owned word of the current device */
+    int merge_per_step_h;    /* cells removed per COLUMN per height step (0 = merge_per_step) */
+    int merge_per_step_w;    /* cells removed per ROW per width step (0 = merge_per_step) */
 } luvc_oim_opts;
 
 /*
@@ -222,6 +242,8 @@ typedef struct {
     int no_window;           /* 0: Hamming-windowed pass band (Eq. 5); 1: flat pass band
                                 (the paper's "without HW" ablation) */
     float* out_scores;       /* optional device [B, N] fp32: the energies E of Eq. 8 */
+    int32_t* device_status;  /* optional device block of LUVC_STATUS_BYTES (see luvc_read_status);
+                                NULL = the library-owned word of the current device */
 } luvc_spu_opts;
 
 /*

@@ -48,8 +48,9 @@ def lib() -> ctypes.CDLL:
             c_int, c_dbl = ctypes.c_int, ctypes.c_double
             P = ctypes.c_void_p
             L.oracle_oim_final_dims.argtypes = [c_int, c_int, c_int, P, P]
-            L.oracle_oim_schedule.argtypes = [c_int] * 6 + [P, P, c_int]
-            L.oracle_oim_batch.argtypes = [P] + [c_int] * 9 + [P, P, P, P, c_dbl, P, P, c_int]
+            L.oracle_oim_schedule.argtypes = [c_int] * 7 + [P, P, c_int]
+            L.oracle_oim_anyres_plan.argtypes = [c_int] * 4 + [P, P, P, P]
+            L.oracle_oim_batch.argtypes = [P] + [c_int] * 10 + [P, P, P, P, c_dbl, P, P, c_int]
             L.oracle_dft_naive.argtypes = [P, c_int, P, P]
             L.oracle_dft_naive.restype = None
             L.oracle_fft.argtypes = [P, P, c_int, c_int, P, P]
@@ -87,12 +88,31 @@ def oim_final_dims(H: int, W: int, target: int):
     return hf.value, wf.value
 
 
+def _per_axis(r):
+    """r is one merge number for both axes, or a pair (r_h, r_w): cells removed per column in a
+    height step, per row in a width step."""
+    if isinstance(r, (tuple, list)):
+        return int(r[0]), int(r[1])
+    return int(r), int(r)
+
+
+def oim_anyres_plan(H: int, W: int, ops: int, r: int = 2):
+    """Per-axis merge numbers and final grid for an image whose sides differ (appendix, the variant
+    that adjusts the merges to the aspect ratio): ((r_h, r_w), (Hf, Wf))."""
+    v = [ctypes.c_int(0) for _ in range(4)]
+    rc = lib().oracle_oim_anyres_plan(H, W, ops, r, *[ctypes.byref(c) for c in v])
+    if rc:
+        raise ValueError("%d operations with merge number %d leave nothing of a %dx%d grid" % (ops, r, H, W))
+    return (v[0].value, v[1].value), (v[2].value, v[3].value)
+
+
 def oim_schedule(H, W, Hf, Wf, r=2, height_first=False):
     """List of (axis, m) steps; axis 0 shrinks the width, axis 1 the height."""
     cap = 2 * (H + W) + 4
     axes = np.zeros(cap, np.int32)
     ms = np.zeros(cap, np.int32)
-    n = lib().oracle_oim_schedule(H, W, Hf, Wf, r, int(height_first), _ptr(axes), _ptr(ms), cap)
+    r_h, r_w = _per_axis(r)
+    n = lib().oracle_oim_schedule(H, W, Hf, Wf, r_w, r_h, int(height_first), _ptr(axes), _ptr(ms), cap)
     if n < 0:
         raise ValueError("grid %dx%d cannot be reduced to %dx%d" % (H, W, Hf, Wf))
     return [(int(axes[i]), int(ms[i])) for i in range(n)]
@@ -104,7 +124,8 @@ def oim(tokens, target=None, out_hw=None, r=2, height_first=False, trace=None, t
 
     ``matching``: "adjacent" compares every even cell of a line with its one or two
     neighbours; "bipartite" compares it with every odd cell of the line (the reading
-    behind the O(n_v^1.5 k) cost stated in Section 3.2).
+    behind the O(n_v^1.5 k) cost stated in Section 3.2).  ``r``: the merge number, or a pair
+    (r_h, r_w) for the per-axis numbers of the appendix's aspect-ratio variant.
 
     Returns a dict: tokens [B,T,D] float64, sizes [B,T] int32, map [B,H*W] int32,
     trace [B,H*W-T] int32, stats [B,4] = (min selection margin, min direction
@@ -123,7 +144,8 @@ def oim(tokens, target=None, out_hw=None, r=2, height_first=False, trace=None, t
     if trace is not None:
         tin = np.ascontiguousarray(np.asarray(trace, dtype=np.int32)).reshape(B, H * W - T)
     nt = nthreads or hardware_threads()
-    rc = lib().oracle_oim_batch(_ptr(x), B, H, W, D, Hf, Wf, r, int(height_first),
+    r_h, r_w = _per_axis(r)
+    rc = lib().oracle_oim_batch(_ptr(x), B, H, W, D, Hf, Wf, r_w, r_h, int(height_first),
                                 {"adjacent": 0, "bipartite": 1}[matching], _ptr(out_tokens),
                                 _ptr(out_sizes), _ptr(out_map), _ptr(tin), float(tol), _ptr(trace_out),
                                 _ptr(stats), nt)

@@ -463,16 +463,18 @@ int oracle_oim_final_dims(int H, int W, int target, int* Hf, int* Wf) {
 // (the other order when height_first), each removing m cells per line, until
 // the grid is Hf x Wf.  axes[i] is 0 (width) or 1 (height).  Returns the number
 // of steps, or -1 if the target cannot be reached.
-int oracle_oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first,
+// r_w cells leave every row in a width step, r_h cells every column in a height step
+// (the appendix uses 2 for both; its anyres variant lets the two differ with the image's shape).
+int oracle_oim_schedule(int H, int W, int Hf, int Wf, int r_w, int r_h, int height_first,
                         int32_t* axes, int32_t* ms, int cap) {
-    if (Hf < 1 || Wf < 1 || Hf > H || Wf > W || r < 1) return -1;
+    if (Hf < 1 || Wf < 1 || Hf > H || Wf > W || r_w < 1 || r_h < 1) return -1;
     int h = H, w = W, n = 0;
     while (h != Hf || w != Wf) {
         bool progressed = false;
         for (int turn = 0; turn < 2; ++turn) {
             const int axis = height_first ? 1 - turn : turn;
             const int len = axis == 0 ? w : h, lf = axis == 0 ? Wf : Hf;
-            const int m = merges_this_step(len, lf, r);
+            const int m = merges_this_step(len, lf, axis == 0 ? r_w : r_h);
             if (m <= 0) continue;
             if (axes && n < cap) { axes[n] = axis; ms[n] = m; }
             ++n;
@@ -484,6 +486,23 @@ int oracle_oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first,
     return n;
 }
 
+// Merge numbers for an image whose sides differ (appendix, the variant for encoders that keep the
+// image's aspect ratio: "the merging operations along the spatial dimensions are dynamically
+// adjusted based on the aspect ratio").  The reading taken: `ops` operations, each one width step
+// and one height step; the shorter side loses r cells per step and the longer side
+// round(r * long / short), so that both sides shrink by about the same fraction and the grid
+// keeps its shape.  Returns 0 and the per-axis numbers and final grid, 1 if a side would vanish.
+int oracle_oim_anyres_plan(int H, int W, int ops, int r, int* r_h, int* r_w, int* Hf, int* Wf) {
+    if (H < 1 || W < 1 || ops < 0 || r < 1) return 1;
+    int rh = r, rw = r;
+    if (W > H) rw = (int)std::floor((double)r * (double)W / (double)H + 0.5);
+    if (H > W) rh = (int)std::floor((double)r * (double)H / (double)W + 0.5);
+    const long long hf = (long long)H - (long long)ops * rh, wf = (long long)W - (long long)ops * rw;
+    if (hf < 1 || wf < 1) return 1;
+    *r_h = rh; *r_w = rw; *Hf = (int)hf; *Wf = (int)wf;
+    return 0;
+}
+
 // OIM on one image.  tokens: [H*W][D] (exact input values as float).
 // out_tokens: [Hf*Wf][D] double; out_sizes: [Hf*Wf]; out_map: [H*W] (final
 // row-major cell of every source token).  trace_in == NULL: the oracle decides.
@@ -492,11 +511,11 @@ int oracle_oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first,
 // the full-line bipartite reading) are checked against `tol` and applied.  trace_out (may be
 // NULL) gets the applied decisions.  stats[0..3] = minimum selection margin,
 // minimum direction margin, violations, deviations.
-int oracle_oim_image(const float* tokens, int H, int W, int D, int Hf, int Wf, int r, int height_first, int matching,
+int oracle_oim_image(const float* tokens, int H, int W, int D, int Hf, int Wf, int r_w, int r_h, int height_first, int matching,
                      double* out_tokens, int32_t* out_sizes, int32_t* out_map,
                      const int32_t* trace_in, double tol, int32_t* trace_out, double* stats) {
     std::vector<int32_t> axes(2 * (size_t)(H + W) + 4), ms(axes.size());
-    const int nsteps = oracle_oim_schedule(H, W, Hf, Wf, r, height_first, axes.data(), ms.data(), (int)axes.size());
+    const int nsteps = oracle_oim_schedule(H, W, Hf, Wf, r_w, r_h, height_first, axes.data(), ms.data(), (int)axes.size());
     if (nsteps < 0) return 1;
     std::vector<Cell> grid((size_t)H * W);
     for (int i = 0; i < H * W; ++i) {
@@ -526,14 +545,14 @@ int oracle_oim_image(const float* tokens, int H, int W, int D, int Hf, int Wf, i
 }
 
 // A batch of images on `nthreads` host threads (images are independent).
-int oracle_oim_batch(const float* tokens, int B, int H, int W, int D, int Hf, int Wf, int r, int height_first, int matching,
+int oracle_oim_batch(const float* tokens, int B, int H, int W, int D, int Hf, int Wf, int r_w, int r_h, int height_first, int matching,
                      double* out_tokens, int32_t* out_sizes, int32_t* out_map,
                      const int32_t* trace_in, double tol, int32_t* trace_out, double* stats, int nthreads) {
     const size_t ntrace = (size_t)H * W - (size_t)Hf * Wf;
     std::vector<int> rc((size_t)B, 0);
     auto work = [&](int t) {
         for (int b = t; b < B; b += nthreads)
-            rc[b] = oracle_oim_image(tokens + (size_t)b * H * W * D, H, W, D, Hf, Wf, r, height_first, matching,
+            rc[b] = oracle_oim_image(tokens + (size_t)b * H * W * D, H, W, D, Hf, Wf, r_w, r_h, height_first, matching,
                                      out_tokens + (size_t)b * Hf * Wf * D, out_sizes + (size_t)b * Hf * Wf,
                                      out_map + (size_t)b * H * W,
                                      trace_in ? trace_in + (size_t)b * ntrace : nullptr, tol,

@@ -208,6 +208,52 @@ def test_plan_maximises_total_similarity_on_tiny_grids(oracle_mod, H, W, Hf, Wf)
         assert np.array_equal(r["sizes"][0].reshape(Hf, Wf), sizes)
 
 
+def _anyres_golden():
+    plans, scheds = [], []
+    for line in open(os.path.join(GOLDEN, "oim_anyres_schedules.txt")):
+        f = line.split()
+        if not f or f[0].startswith("#"):
+            continue
+        if f[0] == "P":
+            plans.append(tuple(int(v) for v in f[1:]))
+        else:
+            scheds.append((tuple(int(v) for v in f[1:7]), [tuple(int(v) for v in st.split(":")) for st in f[7:]]))
+    return plans, scheds
+
+
+def test_per_axis_merge_numbers_follow_the_hand_counted_schedules(oracle_mod):
+    plans, scheds = _anyres_golden()
+    assert len(plans) >= 3 and len(scheds) >= 3
+    for H, W, ops, r, r_h, r_w, Hf, Wf, steps in plans:
+        assert oracle_mod.oim_anyres_plan(H, W, ops, r) == ((r_h, r_w), (Hf, Wf))
+        assert len(oracle_mod.oim_schedule(H, W, Hf, Wf, r=(r_h, r_w))) == steps
+    for (H, W, Hf, Wf, r_h, r_w), steps in scheds:
+        assert oracle_mod.oim_schedule(H, W, Hf, Wf, r=(r_h, r_w)) == steps
+    with pytest.raises(ValueError):
+        oracle_mod.oim_anyres_plan(8, 40, 4, 2)          # the long side would lose 4 x 10 = 40 cells, all it has
+
+
+def test_per_axis_merge_numbers_keep_the_invariants(oracle_mod):
+    # a 6 x 14 grid with 1 cell per column step and 3 per row step: every line loses exactly its
+    # axis' number, sizes add up, merged tokens are the means of their sources
+    x = _rand_grid(2, 6, 14, 7, seed=31)
+    r = oracle_mod.oim(x, out_hw=(4, 8), r=(1, 3))
+    assert r["sizes"].sum(axis=1).tolist() == [84, 84]
+    per_line = [(0, 3), (1, 1), (0, 3), (1, 1)]
+    assert oracle_mod.oim_schedule(6, 14, 4, 8, r=(1, 3)) == per_line
+    assert r["trace"].shape[1] == 6 * 3 + 11 * 1 + 5 * 3 + 8 * 1
+    for b in range(2):
+        flat = x[b].reshape(84, 7).astype(np.float64)
+        for c in range(32):
+            src = np.nonzero(r["map"][b] == c)[0]
+            assert len(src) == r["sizes"][b, c]
+            np.testing.assert_allclose(r["tokens"][b, c], flat[src].mean(axis=0), rtol=1e-12, atol=1e-12)
+    # the same merge number on both axes, given as a pair, is the plain call
+    a = oracle_mod.oim(x, out_hw=(4, 8), r=(2, 2))
+    b_ = oracle_mod.oim(x, out_hw=(4, 8), r=2)
+    np.testing.assert_array_equal(a["map"], b_["map"])
+
+
 # ------------------------------------------------------------------ replay
 
 
