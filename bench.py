@@ -33,9 +33,25 @@ L2_BYTES = 126 * 1024 * 1024
 HBM_NOMINAL_GBS = 8000.0      # the figure the metric's "% of 8 TB/s" divides by
 HBM_FALLBACK_GBS = 6650.0     # used only if MEASURED_PEAKS.json is absent
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (null until a capture for that workload exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {2: 1.428e9 + 0.140e9}     # profiles/oim_chain_kernel_configs2.txt
+
+
+def ncu_traffic():
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
+    profiles/ (profiles/ncu_traffic.json: kernel -> workload -> bytes, with the source version of the
+    kernel the counters were taken on; an entry is ignored once that source has changed)."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if not os.path.exists(path):
+        return {}
+    import hashlib
+
+    table = json.load(open(path))
+    out = {}
+    for kernel, entry in table.items():
+        src = os.path.join(ROOT, entry["source"])
+        digest = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] if os.path.exists(src) else None
+        if digest == entry.get("source_sha256_16"):
+            out[kernel] = {int(k): float(v) for k, v in entry["bytes_per_launch"].items()}
+    return out
 
 
 def parse_args():
@@ -50,6 +66,8 @@ def parse_args():
                          "no end-to-end and no CPU-baseline leg)")
     ap.add_argument("--cpu-sample", type=int, default=0, help="units of the batch the CPU oracle is timed on (0 = auto)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="skip the per_config object (configs[2]-[4] with the cutoff x keep sweep of configs[4])")
     return ap.parse_args()
 
 
@@ -96,6 +114,20 @@ def oim_iter_bytes(luvc, B, H, W, D, target, e=2):
             total += B * (h * w + nh * nw) * (D * e + 4)
             h, w = nh, nw
     return total, n_steps
+
+
+def floor_bytes_oim(B, H, W, D, T, e=2):
+    """What must move if the whole chain stayed on chip: the input once, the three outputs once."""
+    return B * H * W * D * e + B * T * (D * e + 4) + B * H * W * 4
+
+
+def spu_bytes(sb, sn, sd, keep, e=2):
+    """Algorithmic bytes of one prune: the transform reads the sequence once and writes the scores, the
+    select reads them and writes the indices, the gather reads and writes the kept rows."""
+    transform = sb * sn * sd * e + sb * sn * 4
+    select = sb * sn * 4 + sb * keep * 4
+    gather = 2 * sb * keep * sd * e
+    return transform, select, gather
 
 
 def make_inputs(spec, device, sets):
@@ -290,6 +322,125 @@ def whole_job_tokens_per_second(tokens_per_rank, world, ms_per_step):
 # ----------------------------------------------------------------------------- the GPU arm
 
 
+def load_peak():
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        return float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return HBM_FALLBACK_GBS, "fallback"
+
+
+def rate(nbytes, ms, peak):
+    """GB/s and its fractions of the measured copy rate and of the nominal 8 TB/s."""
+    if not ms or ms <= 0:
+        return {"bytes": nbytes, "ms": ms, "achieved": None, "frac": None, "frac_of_8TBs": None}
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"bytes": nbytes, "ms": ms, "achieved": gbs, "frac": gbs / peak, "frac_of_8TBs": gbs / HBM_NOMINAL_GBS}
+
+
+def timed_steps(torch, step, steps, warmup, barrier):
+    """`warmup` untimed steps, then `steps` steps between two events on the current stream."""
+    for i in range(warmup):
+        step(i)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(steps):
+        step(i)
+    ev1.record()
+    barrier()
+    return ev0.elapsed_time(ev1)
+
+
+def phase_times(luvc, step, reps):
+    """The library's own events around its phases, one step at a time, averaged."""
+    luvc.profile_enable(True)
+    phases = {name: 0.0 for name in luvc.PHASES}
+    for i in range(reps):
+        step(i)
+        got = luvc.profile_read()
+        for name in phases:
+            phases[name] += got[name] / reps
+    luvc.profile_enable(False)
+    return phases
+
+
+def oim_roofline(luvc, spec, phases, peak, peak_src, traffic, matching):
+    B, H, W, D = spec["oim"]
+    iter_bytes, n_steps = oim_iter_bytes(luvc, B, H, W, D, spec["target"], 2)
+    steps_ms = phases["oim_steps"]
+    r = rate(iter_bytes, steps_ms, peak)
+    kernel = "oim_chain_kernel" if matching == "adjacent" else "oim_bipartite_kernel"
+    t = traffic.get(kernel, {}).get(spec["id"])
+    out = {
+        "kernel": "%s (one launch runs the %d merge steps of a call)" % (kernel, n_steps),
+        "bound": "hbm", "achieved": r["achieved"], "peak": peak, "unit": "GB/s", "frac": r["frac"],
+        "peak_source": peak_src, "frac_of_8TBs": r["frac_of_8TBs"],
+        "algorithmic_bytes_per_launch": iter_bytes, "avg_launch_ms": steps_ms, "merge_steps_per_launch": n_steps,
+        "algorithmic_bytes_note": "per step: read the grid, write the compacted grid (tokens + sizes), summed over the "
+                                  "schedule; this kernel keeps tokens in place, so part of those reads is served by L2 "
+                                  "and the compaction write is not performed: see `dram` and `floor`",
+        "traffic": t,
+        "dram": rate(t, steps_ms, peak) if t else None,
+        "floor": rate(floor_bytes_oim(B, H, W, D, spec["target"]), steps_ms, peak),
+    }
+    return out
+
+
+def spu_roofline(spec, keep, phases, peak):
+    sb, sn, sd = spec["spu"]
+    tb, selb, gb = spu_bytes(sb, sn, sd, keep)
+    total_ms = phases["spu_transform"] + phases["spu_select"] + phases["spu_gather"]
+    out = rate(tb + selb + gb, total_ms, peak)
+    out.update({"bound": "hbm", "unit": "GB/s", "peak": peak,
+                "transform": rate(tb, phases["spu_transform"], peak),
+                "select": rate(selb, phases["spu_select"], peak),
+                "gather": rate(gb, phases["spu_gather"], peak)})
+    return out
+
+
+def per_config_report(torch, luvc, device, peak, peak_src, traffic, barrier, have):
+    """configs[2], [3], [4] each timed on this machine: ms per step, the OIM chain's and the SPU's own
+    roofline objects, and for configs[4] the whole cutoff x keep sweep of the prune."""
+    import luvc_inputs as gi
+
+    report = {}
+    for k in (2, 3, 4):
+        spec = workload_spec(k)
+        if k in have:
+            xs, ys, sets = have[k]
+        else:
+            sets = 2
+            xs, ys = make_inputs(spec, device, sets)
+
+        def step(i, spec=spec, xs=xs, ys=ys, sets=sets):
+            luvc.oim_merge(xs[i % sets], spec["target"])
+            luvc.spu_prune(ys[i % sets], spec["keep"], spec["cutoff"])
+
+        ms = timed_steps(torch, step, 10, 3, barrier) / 10
+        ph = phase_times(luvc, step, 10)
+        entry = {"workload": workload_name(spec), "ms_per_step": ms, "tokens_per_s": spec["tokens"] / (ms * 1e-3),
+                 "phases_ms": ph, "oim": oim_roofline(luvc, spec, ph, peak, peak_src, traffic, "adjacent"),
+                 "spu": spu_roofline(spec, spec["keep"], ph, peak)}
+        c = gi.CONFIGS[k]
+        sweep = []
+        cutoffs = c.get("cutoffs", (0.0,))
+        for cutoff in cutoffs:
+            for keep in c["keep"]:
+                def prune(i, ys=ys, sets=sets, keep=keep, cutoff=cutoff):
+                    luvc.spu_prune(ys[i % sets], keep, cutoff)
+
+                timed_steps(torch, prune, 2, 3, barrier)
+                ph2 = phase_times(luvc, prune, 6)
+                row = spu_roofline(spec, keep, ph2, peak)
+                row.update({"cutoff": cutoff if cutoff > 0 else 0.125, "keep": keep})
+                sweep.append(row)
+        entry["spu_sweep"] = sweep
+        report["configs[%d]" % k] = entry
+        del xs, ys
+        torch.cuda.empty_cache()
+    return report
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -356,15 +507,7 @@ def main():
     value = whole_job_tokens_per_second(spec["tokens"], world, ms_per_step)
 
     # ---- per-phase pass: the library's own events around its phases, one step at a time
-    luvc.profile_enable(True)
-    phases = {name: 0.0 for name in luvc.PHASES}
-    reps = min(args.steps, 20)
-    for i in range(reps):
-        step(i)
-        got = luvc.profile_read()
-        for name in phases:
-            phases[name] += got[name] / reps
-    luvc.profile_enable(False)
+    phases = phase_times(luvc, step, min(args.steps, 20))
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region
     x_host = xs[0].cpu().pin_memory()
@@ -396,50 +539,37 @@ def main():
         for job in jobs:
             job.result()
 
-    for _ in range(3):
-        e2e_step()
-    barrier()
-    e2e_reps = max(3, min(args.steps, 20))
-    ev0.record()
-    for _ in range(e2e_reps):
-        e2e_step()
-    ev1.record()
-    barrier()
+    e2e_ms = None
+    if args.oim_matching == "adjacent":
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e2e_reps = max(3, min(args.steps, 20))
+        ev0.record()
+        for _ in range(e2e_reps):
+            e2e_step()
+        ev1.record()
+        barrier()
+        e2e_ms = max_over_ranks(ev0.elapsed_time(ev1) / e2e_reps, world, device)
     pool.shutdown()
-    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1) / e2e_reps, world, device)
     h2d = x_host.numel() * 2 + y_host.numel() * 2
     d2h = sum(t_.numel() * t_.element_size() for t_ in (o_tok, o_sz, o_map, o_idx, o_hid))
+    del x_host, y_host
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    else:
-        peak, peak_src = HBM_FALLBACK_GBS, "fallback"
-    iter_bytes, n_steps = oim_iter_bytes(luvc, B, H, W, D, spec["target"], e)
-    floor_bytes = B * H * W * D * e + B * T * (D * e + 4) + B * H * W * 4
-    steps_ms = phases["oim_steps"]
-    achieved = iter_bytes / (steps_ms * 1e-3) / 1e9 if steps_ms > 0 else None
-    spu_bytes = spu_in_bytes + sb * sn * 4 + 2 * sb * spec["keep"] * sd * e + sb * spec["keep"] * 4
-    spu_ms = phases["spu_transform"] + phases["spu_select"] + phases["spu_gather"]
-    roofline = {
-        "kernel": "%s (one launch runs the %d merge steps of a call)" % (
-            "oim_chain_kernel" if args.oim_matching == "adjacent" else "oim_bipartite_kernel", n_steps),
-        "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-        "frac": achieved / peak if achieved else None, "peak_source": peak_src,
-        "frac_of_8TBs": achieved / HBM_NOMINAL_GBS if achieved else None,
-        "algorithmic_bytes_per_launch": iter_bytes, "avg_launch_ms": steps_ms, "merge_steps_per_launch": n_steps,
-        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(k) if args.oim_matching == "adjacent" else None,
-        "floor_bytes": floor_bytes,
-        "spu": {"algorithmic_bytes": spu_bytes, "ms": spu_ms,
-                "achieved": spu_bytes / (spu_ms * 1e-3) / 1e9 if spu_ms > 0 else None,
-                "frac": spu_bytes / (spu_ms * 1e-3) / 1e9 / peak if spu_ms > 0 else None},
-    }
+    # ---- roofline of the dominant kernel (the OIM chain), with the SPU's beside it
+    peak, peak_src = load_peak()
+    traffic = ncu_traffic()
+    roofline = oim_roofline(luvc, spec, phases, peak, peak_src, traffic, args.oim_matching)
+    roofline["spu"] = spu_roofline(spec, spec["keep"], phases, peak)
+
+    per_config = None
+    if not args.no_per_config and world == 1 and args.oim_matching == "adjacent":
+        per_config = per_config_report(torch, luvc, device, peak, peak_src, traffic, barrier, {k: (xs, ys, sets)})
 
     cpu = None
     if not args.no_cpu_baseline and args.oim_matching == "adjacent":
@@ -447,7 +577,8 @@ def main():
         info = cpu_oracle_pass(spec, sample, xs[0][:sample].float().cpu().numpy(),
                                ys[0][: max(1, sample)].float().cpu().numpy(), min_seconds=10.0)
         cpu = {"value": info["tokens"] / info["seconds"], "unit": UNIT, "cores": info["cores"], "kind": "oracle",
-               "sample": info["sample"], "seconds": info["seconds"]}
+               "sample": info["sample"], "seconds": info["seconds"],
+               "configs0_single_thread_seconds": config0_single_thread_seconds()}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -458,15 +589,34 @@ def main():
             sets, sets * (oim_in_bytes + spu_in_bytes) / 1e6), "parallelism": "batch split, no collective" if world > 1 else "1 GPU"},
         "clocks": clocks,
         "e2e": {"value": whole_job_tokens_per_second(spec["tokens"], world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h} if args.oim_matching == "adjacent" else None,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h} if e2e_ms else None,
         "gpu_launches": launches,
         "phases_ms": phases,
         "roofline": roofline,
+        "per_config": per_config,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def config0_single_thread_seconds():
+    """The oracle on configs[0] (one fp32 image, then its 144 projected tokens) on ONE host thread."""
+    import torch
+
+    import luvc_inputs as gi
+    import oracle
+
+    x = gi.oim_input(0).float().numpy()
+    t0 = time.perf_counter()
+    r = oracle.oim(x, target=gi.CONFIGS[0]["target"], nthreads=1)
+    y = gi.spu_input_from_tokens(0, torch.from_numpy(r["tokens"]).float()).float().numpy()
+    t1 = time.perf_counter()
+    e = oracle.spu_scores(y[0], oracle.spu_sigma(y.shape[1], 0.0), nthreads=1)
+    oracle.spu_select(e, gi.CONFIGS[0]["keep"][0])
+    t2 = time.perf_counter()
+    return {"oim": t1 - t0, "spu": t2 - t1}
 
 
 if __name__ == "__main__":

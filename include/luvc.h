@@ -94,6 +94,15 @@ int luvc_read_status(int32_t* device_status, void* cuda_stream);
  * by the caller before its first use; the library only ever writes its first word). */
 #define LUVC_STATUS_BYTES 16
 
+/* Test hook for the give-up path of the bounded device-side waits (no counterpart in the paper).
+ * Writes two knobs into a status block (device_status, or the current device's library-owned
+ * block when NULL): `probes` > 0 replaces the probe limit of the OIM chain's waits, and
+ * `hold_back` > 0 starts the first image's count of finished lines of the first merge step that
+ * far below zero, so that no wait on it can ever be satisfied and each gives up after `probes`
+ * probes (microseconds).  The call that follows then ends with LUVC_ERR_TIMEOUT in the block.
+ * 0, 0 restores normal operation.  Synchronises the stream. */
+int luvc_debug_wait_probes(int probes, int hold_back, int32_t* device_status, void* cuda_stream);
+
 /* Frees the library-owned scratch buffers of the current device (and its status
  * word).  Synchronises the device first.  Safe to call more than once. */
 int luvc_shutdown(void);
@@ -126,6 +135,17 @@ int luvc_profile_read(float* ms, int count);
  * (0 = the paper's merge number 2).  LUVC_ERR_TARGET if no such pair exists. */
 int luvc_oim_plan(int H, int W, int target_count, int merge_per_step,
                   int* out_h, int* out_w, int* n_steps);
+
+/* Host-only planning for grids whose sides differ (appendix "Iterative Strategy and Pseudocode of
+ * OIM": for an encoder that keeps the image's aspect ratio the merges along the two spatial axes
+ * follow that ratio; the paper gives no formula, this is the library's reading).  n_ops operations
+ * of one width step and one height step each; the shorter side loses merge_per_step (0 = 2) cells
+ * per step, the longer side round(merge_per_step * long / short), so the grid keeps its shape.
+ * Returns the per-axis numbers (for luvc_oim_opts.merge_per_step_h / _w), the final grid
+ * (for out_h / out_w; target_count = out_h * out_w) and the number of steps.
+ * LUVC_ERR_TARGET if a side would shrink below one cell. */
+int luvc_oim_plan_anyres(int H, int W, int n_ops, int merge_per_step, int* merge_h, int* merge_w,
+                         int* out_h, int* out_w, int* n_steps);
 
 /* Bytes of workspace luvc_oim_merge_ex needs for this problem with the adjacent matching;
  * the _ex form takes the luvc_oim_matching (the bipartite matching also keeps a bf16
@@ -306,7 +326,14 @@ int luvc_spu_cascade(const void* hidden, int B, int N, int D, int n_stages, cons
  * memory budget.  This call never calls cudaMalloc, cudaFree or any routine that
  * allocates, and needs no caller workspace.  Its workspace is an array of
  * LUVC_SPU_STATIC_MAX_BYTES (+256) bytes that is part of the library's device
- * image: every GPU that loads the library holds it from load until exit.
+ * image: every GPU that loads that image holds it until the process exits.
+ * With CUDA's lazy module loading (the default of current toolkits) the image, and
+ * with it the array, is loaded by the first call on a device, and each kernel's
+ * code by its first launch: those first uses can reserve device memory and can
+ * synchronise.  So make ONE warm-up call per device (and per kind of problem: element
+ * type, and a sequence length of the same factor class) at start-up, before the
+ * device's memory is handed to another allocator - or run with
+ * CUDA_MODULE_LOADING=EAGER; from then on no call reserves anything.
  *
  * Arguments and results are those of luvc_spu_prune_ex with default options
  * (Hamming-windowed pass band, no score export): hidden [B,N,D], out_idx [B,keep],
@@ -324,12 +351,19 @@ int luvc_spu_cascade(const void* hidden, int B, int N, int D, int n_stages, cons
  * call clears the part that must start at zero, but two calls whose GPU work
  * overlaps (different streams, or several host threads) race on it - run them on
  * one stream or order them with events.  A bounded device-side wait that gives up
- * is recorded inside the array, not in the word luvc_check_status reads; the
- * outputs of such a call are undefined.  With luvc_profile_enable(1) the first
+ * is recorded inside the array, not in the word luvc_check_status reads:
+ * luvc_spu_static_status reads it; the outputs of such a call are undefined.
+ * With luvc_profile_enable(1) the first
  * call creates CUDA events; leave profiling off where that matters.
  */
 int luvc_spu_prune_static(const void* hidden, int B, int N, int D, float cutoff, int keep, int dtype,
                           void* cuda_stream, int32_t* out_idx, void* out_hidden);
+
+/* Synchronises the stream and returns, as a luvc_status, what the most recent
+ * luvc_spu_prune_static call on the current device recorded inside the array (LUVC_OK, or
+ * LUVC_ERR_TIMEOUT when a bounded wait gave up); the next call clears it.  Allocates nothing.
+ * (No counterpart in the paper.) */
+int luvc_spu_static_status(void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -26,10 +26,11 @@ STATUS_NAMES = {
 # every symbol include/luvc.h declares
 EXPORTS = (
     "luvc_version", "luvc_status_string", "luvc_set_stream", "luvc_shutdown", "luvc_kernel_launches",
-    "luvc_profile_enable", "luvc_profile_read", "luvc_check_status",
-    "luvc_oim_plan", "luvc_oim_workspace_bytes", "luvc_oim_workspace_bytes_ex", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
+    "luvc_profile_enable", "luvc_profile_read", "luvc_check_status", "luvc_read_status", "luvc_debug_wait_probes",
+    "luvc_oim_plan", "luvc_oim_plan_anyres", "luvc_oim_workspace_bytes", "luvc_oim_workspace_bytes_ex", "luvc_oim_merge", "luvc_oim_merge_f32", "luvc_oim_merge_ex",
     "luvc_oim_merge_host", "luvc_oim_value_enhance", "luvc_spu_sigma", "luvc_spu_workspace_bytes", "luvc_spu_prune",
-    "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host", "luvc_spu_prune_static", "luvc_spu_cascade",
+    "luvc_spu_prune_f32", "luvc_spu_prune_ex", "luvc_spu_prune_host", "luvc_spu_prune_static", "luvc_spu_static_status",
+    "luvc_spu_cascade",
 )
 
 
@@ -45,7 +46,8 @@ class OimOpts(ctypes.Structure):
         ("dtype", ctypes.c_int), ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("out_h", ctypes.c_int), ("out_w", ctypes.c_int),
         ("merge_per_step", ctypes.c_int), ("height_first", ctypes.c_int), ("trace", ctypes.c_void_p),
-        ("out_log_sizes", ctypes.c_void_p), ("matching", ctypes.c_int),
+        ("trace_bytes", ctypes.c_size_t), ("out_log_sizes", ctypes.c_void_p), ("matching", ctypes.c_int),
+        ("device_status", ctypes.c_void_p), ("merge_per_step_h", ctypes.c_int), ("merge_per_step_w", ctypes.c_int),
     ]
 
 
@@ -53,6 +55,7 @@ class SpuOpts(ctypes.Structure):
     _fields_ = [
         ("dtype", ctypes.c_int), ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("no_window", ctypes.c_int), ("out_scores", ctypes.c_void_p),
+        ("device_status", ctypes.c_void_p),
     ]
 
 
@@ -72,6 +75,10 @@ def _load() -> ctypes.CDLL:
     L.luvc_set_stream.argtypes = [p]
     L.luvc_kernel_launches.restype = ctypes.c_longlong
     L.luvc_check_status.argtypes = [p]
+    L.luvc_read_status.argtypes = [p, p]
+    L.luvc_debug_wait_probes.argtypes = [i, i, p, p]
+    L.luvc_spu_static_status.argtypes = [p]
+    L.luvc_oim_plan_anyres.argtypes = [i, i, i, i] + [ctypes.POINTER(i)] * 5
     L.luvc_profile_enable.argtypes = [i]
     L.luvc_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), i]
     L.luvc_oim_plan.argtypes = [i, i, i, i, ctypes.POINTER(i), ctypes.POINTER(i), ctypes.POINTER(i)]
@@ -155,16 +162,30 @@ def oim_plan(H: int, W: int, target_count: int, merge_per_step: int = 0):
     return h.value, w.value, n.value
 
 
+def oim_plan_anyres(H: int, W: int, n_ops: int, merge_per_step: int = 0):
+    """((merge_h, merge_w), (out_h, out_w), n_steps) for a grid whose sides differ (host only)."""
+    v = [ctypes.c_int() for _ in range(5)]
+    _check(lib.luvc_oim_plan_anyres(H, W, n_ops, merge_per_step, *[ctypes.byref(c) for c in v]), "luvc_oim_plan_anyres")
+    return (v[0].value, v[1].value), (v[2].value, v[3].value), v[4].value
+
+
+def read_status(block: torch.Tensor) -> int:
+    """luvc_read_status on a caller-owned status block (int32 tensor of >= 4 words on the device)."""
+    return int(lib.luvc_read_status(block.data_ptr(), _stream_ptr(block.device)))
+
+
 def spu_sigma(N: int, cutoff: float = 0.0) -> int:
     return lib.luvc_spu_sigma(N, float(cutoff))
 
 
 def oim_merge(tokens: torch.Tensor, target_count: int, *, out_hw=None, merge_per_step: int = 0,
               height_first: bool = False, want_trace: bool = False, workspace: torch.Tensor | None = None,
-              want_log_sizes: bool = False, matching: str = "adjacent"):
+              want_log_sizes: bool = False, matching: str = "adjacent", merge_per_step_hw=None,
+              device_status: torch.Tensor | None = None):
     """luvc_oim_merge_ex on a CUDA tensor [B,H,W,D]; returns (out_tokens [B,T,D], out_sizes [B,T] int32,
     out_map [B,H*W] int32) and, with want_trace, the per-merge decision log [B,H*W-T] int32.
-    matching: "adjacent" or "bipartite" (luvc_oim_matching)."""
+    matching: "adjacent" or "bipartite" (luvc_oim_matching); merge_per_step_hw: (per column in a height
+    step, per row in a width step); device_status: a caller-owned status block (see read_status)."""
     if not tokens.is_cuda:
         raise ValueError("tokens must live on a CUDA device; host buffers go through oim_merge_host")
     tokens = tokens.contiguous()
@@ -187,6 +208,10 @@ def oim_merge(tokens: torch.Tensor, target_count: int, *, out_hw=None, merge_per
         o.height_first = int(bool(height_first))
         o.matching = {"adjacent": 0, "bipartite": 1}[matching]
         o.trace = trace.data_ptr() if (trace is not None and trace.numel()) else None
+        o.trace_bytes = trace.numel() * 4 if trace is not None else 0
+        if merge_per_step_hw is not None:
+            o.merge_per_step_h, o.merge_per_step_w = int(merge_per_step_hw[0]), int(merge_per_step_hw[1])
+        o.device_status = device_status.data_ptr() if device_status is not None else None
         log_sizes = torch.empty((B, max(T, 0)), dtype=torch.float32, device=dev) if want_log_sizes else None
         o.out_log_sizes = log_sizes.data_ptr() if log_sizes is not None else None
         _check(lib.luvc_oim_merge_ex(tokens.data_ptr(), B, H, W, D, T, out_tokens.data_ptr(), out_sizes.data_ptr(),
@@ -231,7 +256,8 @@ def oim_merge_plain(tokens: torch.Tensor, target_count: int):
 
 
 def spu_prune(hidden: torch.Tensor, keep: int, cutoff: float = 0.0, *, no_window: bool = False,
-              want_scores: bool = False, workspace: torch.Tensor | None = None):
+              want_scores: bool = False, workspace: torch.Tensor | None = None,
+              device_status: torch.Tensor | None = None):
     """luvc_spu_prune_ex on a CUDA tensor [B,N,D]; returns (out_idx [B,keep] int32, out_hidden [B,keep,D])
     and, with want_scores, the energies E [B,N] float32."""
     if not hidden.is_cuda:
@@ -251,6 +277,7 @@ def spu_prune(hidden: torch.Tensor, keep: int, cutoff: float = 0.0, *, no_window
             o.workspace, o.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
         o.no_window = int(bool(no_window))
         o.out_scores = scores.data_ptr() if scores is not None else None
+        o.device_status = device_status.data_ptr() if device_status is not None else None
         _check(lib.luvc_spu_prune_ex(hidden.data_ptr(), B, N, D, float(cutoff), k, out_idx.data_ptr(),
                                      out_hidden.data_ptr(), ctypes.byref(o)), "luvc_spu_prune_ex")
     if want_scores:

@@ -39,17 +39,26 @@ namespace {
 
 thread_local cudaStream_t t_stream = nullptr;
 
-// Library-owned scratch: one growing buffer per purpose, shared by all threads.
-// Calls that use it from several host threads at once must use different streams'
-// work serially; the plain entry points take this lock only while (re)allocating.
+// Library-owned scratch: one growing buffer per purpose and per device (keyed by the ordinal of the
+// device that is current at the call), shared by all threads and streams of the process.  Calls
+// whose GPU work overlaps race on it (documented in luvc.h); the lock only covers (re)allocation.
 enum Slot { kOimWs = 0, kSpuWs, kIoIn, kIoOut, kStatus, kCascade, kIoInSpu, kIoOutSpu, kSlots };
+constexpr int kMaxDevices = 64;
 struct Scratch { void* ptr = nullptr; size_t bytes = 0; };
-Scratch g_scratch[kSlots];
+Scratch g_scratch[kMaxDevices][kSlots];
 std::mutex g_mutex;
 
+int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
 void* scratch(Slot s, size_t bytes) {
+    const int dev = current_device();
+    if (dev < 0) return nullptr;
     std::lock_guard<std::mutex> lock(g_mutex);
-    Scratch& sc = g_scratch[s];
+    Scratch& sc = g_scratch[dev][s];
     if (sc.bytes >= bytes && sc.ptr) return sc.ptr;
     if (sc.ptr) { cudaDeviceSynchronize(); cudaFree(sc.ptr); sc.ptr = nullptr; sc.bytes = 0; }
     void* p = nullptr;
@@ -58,19 +67,34 @@ void* scratch(Slot s, size_t bytes) {
     return p;
 }
 
-// The device status word: 256 bytes allocated once and zeroed, never freed before luvc_shutdown.
+// The current device's status block: 256 bytes allocated once and zeroed, kept until luvc_shutdown.
 int* status_word() {
+    const int dev = current_device();
+    if (dev < 0) return nullptr;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
-        if (g_scratch[kStatus].ptr) return static_cast<int*>(g_scratch[kStatus].ptr);
+        if (g_scratch[dev][kStatus].ptr) return static_cast<int*>(g_scratch[dev][kStatus].ptr);
     }
     void* p = scratch(kStatus, 256);
     if (p && cudaMemset(p, 0, 256) != cudaSuccess) return nullptr;
     return static_cast<int*>(p);
 }
 
+// Reads (after synchronising the stream) and clears the first word of a status block.
+int read_status_block(int* block, cudaStream_t stream) {
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return LUVC_ERR_CUDA;
+    int host = 0;
+    if (cudaMemcpy(&host, block, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return LUVC_ERR_CUDA;
+    if (host != 0 && cudaMemset(block, 0, sizeof(int)) != cudaSuccess) return LUVC_ERR_CUDA;
+    return host;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 size_t elem_size(int dtype) { return dtype == LUVC_F32 ? 4 : 2; }
+
+// Merge numbers per axis: the axis' own field, else the common one, else the appendix's 2.
+int oim_r_w(const luvc_oim_opts& o) { return o.merge_per_step_w ? o.merge_per_step_w : (o.merge_per_step ? o.merge_per_step : 2); }
+int oim_r_h(const luvc_oim_opts& o) { return o.merge_per_step_h ? o.merge_per_step_h : (o.merge_per_step ? o.merge_per_step : 2); }
 
 int check_oim(const void* tokens, int B, int H, int W, int D, int target, const void* out_tokens,
               const void* out_sizes, const void* out_map, const luvc_oim_opts& o, int* Hf, int* Wf) {
@@ -82,7 +106,8 @@ int check_oim(const void* tokens, int B, int H, int W, int D, int target, const 
     if (!aligned16(tokens) || !aligned16(out_tokens) || (reinterpret_cast<uintptr_t>(out_sizes) & 3u) ||
         (reinterpret_cast<uintptr_t>(out_map) & 3u))
         return LUVC_ERR_ALIGN;
-    if (o.merge_per_step < 0) return LUVC_ERR_TARGET;
+    if (o.merge_per_step < 0 || o.merge_per_step_h < 0 || o.merge_per_step_w < 0) return LUVC_ERR_TARGET;
+    if (o.device_status && (reinterpret_cast<uintptr_t>(o.device_status) & 15u)) return LUVC_ERR_ALIGN;
     if (o.matching != LUVC_OIM_MATCH_ADJACENT && o.matching != LUVC_OIM_MATCH_BIPARTITE) return LUVC_ERR_SHAPE;
     if (o.matching == LUVC_OIM_MATCH_BIPARTITE && (H > 256 || W > 256)) return LUVC_ERR_SHAPE;
     if (o.matching == LUVC_OIM_MATCH_BIPARTITE && D % 8 != 0) return LUVC_ERR_ALIGN;
@@ -94,8 +119,12 @@ int check_oim(const void* tokens, int B, int H, int W, int D, int target, const 
         return LUVC_ERR_TARGET;
     }
     int n = 0;
-    if (!oim_schedule(H, W, *Hf, *Wf, o.merge_per_step ? o.merge_per_step : 2, o.height_first, nullptr, 0, &n))
-        return LUVC_ERR_TARGET;
+    if (!oim_schedule(H, W, *Hf, *Wf, oim_r_w(o), oim_r_h(o), o.height_first, nullptr, 0, &n)) return LUVC_ERR_TARGET;
+    if (o.trace) {
+        if (reinterpret_cast<uintptr_t>(o.trace) & 3u) return LUVC_ERR_ALIGN;
+        const size_t need = (size_t)B * ((size_t)H * W - (size_t)*Hf * *Wf) * sizeof(int32_t);
+        if (o.trace_bytes < need) return LUVC_ERR_WORKSPACE;
+    }
     return LUVC_OK;
 }
 
@@ -146,9 +175,11 @@ int luvc_set_stream(void* cuda_stream) {
 }
 
 int luvc_shutdown(void) {
+    const int dev = current_device();
+    if (dev < 0) return LUVC_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_mutex);
     cudaDeviceSynchronize();
-    for (auto& sc : g_scratch) {
+    for (auto& sc : g_scratch[dev]) {
         if (sc.ptr) cudaFree(sc.ptr);
         sc.ptr = nullptr; sc.bytes = 0;
     }
@@ -156,13 +187,25 @@ int luvc_shutdown(void) {
 }
 
 int luvc_check_status(void* cuda_stream) {
-    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return LUVC_ERR_CUDA;
     int* word = status_word();
     if (!word) return LUVC_ERR_CUDA;
-    int host = 0;
-    if (cudaMemcpy(&host, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return LUVC_ERR_CUDA;
-    if (host != 0 && cudaMemset(word, 0, sizeof(int)) != cudaSuccess) return LUVC_ERR_CUDA;
-    return host;
+    return read_status_block(word, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int luvc_read_status(int32_t* device_status, void* cuda_stream) {
+    if (!device_status) return LUVC_ERR_NULL;
+    return read_status_block(device_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int luvc_debug_wait_probes(int probes, int hold_back, int32_t* device_status, void* cuda_stream) {
+    if (probes < 0 || hold_back < 0) return LUVC_ERR_SHAPE;
+    int* block = device_status ? device_status : status_word();
+    if (!block) return LUVC_ERR_CUDA;
+    const int knobs[2] = {probes, hold_back};
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(block + kStatusProbeLimit, knobs, sizeof(knobs), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return LUVC_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;   // `knobs` lives on this stack
 }
 
 long long luvc_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
@@ -192,8 +235,27 @@ int luvc_oim_plan(int H, int W, int target_count, int merge_per_step, int* out_h
     if (H < 1 || W < 1) return LUVC_ERR_SHAPE;
     int hf, wf, n;
     if (merge_per_step < 0 || !oim_final_dims(H, W, target_count, &hf, &wf)) return LUVC_ERR_TARGET;
-    if (!oim_schedule(H, W, hf, wf, merge_per_step ? merge_per_step : 2, 0, nullptr, 0, &n)) return LUVC_ERR_TARGET;
+    const int r = merge_per_step ? merge_per_step : 2;
+    if (!oim_schedule(H, W, hf, wf, r, r, 0, nullptr, 0, &n)) return LUVC_ERR_TARGET;
     *out_h = hf; *out_w = wf; *n_steps = n;
+    return LUVC_OK;
+}
+
+int luvc_oim_plan_anyres(int H, int W, int n_ops, int merge_per_step, int* merge_h, int* merge_w, int* out_h,
+                         int* out_w, int* n_steps) {
+    if (!merge_h || !merge_w || !out_h || !out_w || !n_steps) return LUVC_ERR_NULL;
+    if (H < 1 || W < 1) return LUVC_ERR_SHAPE;
+    if (n_ops < 0 || merge_per_step < 0) return LUVC_ERR_TARGET;
+    const long long r = merge_per_step ? merge_per_step : 2;
+    // the longer side's number is r * long / short rounded to the nearest integer (halves up), in integers
+    const long long lo = H < W ? H : W, hi = H < W ? W : H;
+    const long long r_long = (2 * r * hi + lo) / (2 * lo);
+    const long long rh = H > W ? r_long : r, rw = W > H ? r_long : r;
+    const long long hf = H - n_ops * rh, wf = W - n_ops * rw;
+    if (hf < 1 || wf < 1 || rh > 0x7fffffffll || rw > 0x7fffffffll) return LUVC_ERR_TARGET;
+    int n = 0;
+    if (!oim_schedule(H, W, (int)hf, (int)wf, (int)rw, (int)rh, 0, nullptr, 0, &n)) return LUVC_ERR_TARGET;
+    *merge_h = (int)rh; *merge_w = (int)rw; *out_h = (int)hf; *out_w = (int)wf; *n_steps = n;
     return LUVC_OK;
 }
 
@@ -224,14 +286,14 @@ int luvc_oim_merge_ex(const void* tokens, int B, int H, int W, int D, int target
     }
     OimProblem p;
     p.tokens = tokens; p.B = B; p.H = H; p.W = W; p.D = D; p.Hf = Hf; p.Wf = Wf;
-    p.r = opts->merge_per_step ? opts->merge_per_step : 2;
+    p.r_w = oim_r_w(*opts); p.r_h = oim_r_h(*opts);
     p.height_first = opts->height_first ? 1 : 0;
     p.dtype = opts->dtype;
     p.out_tokens = out_tokens; p.out_sizes = out_sizes; p.out_map = out_map; p.trace = opts->trace;
     p.out_log_sizes = opts->out_log_sizes;
     p.matching = opts->matching;
     p.workspace = ws; p.stream = static_cast<cudaStream_t>(opts->stream);
-    p.status = status_word();
+    p.status = opts->device_status ? opts->device_status : status_word();
     if (!p.status) return LUVC_ERR_CUDA;
     return oim_run(p);
 }
@@ -254,7 +316,15 @@ int luvc_oim_merge_host(const void* tokens, int B, int H, int W, int D, int targ
                         void* out_tokens, int32_t* out_sizes, int32_t* out_map) {
     if (!tokens || !out_tokens || !out_sizes || !out_map) return LUVC_ERR_NULL;
     if (dtype != LUVC_BF16 && dtype != LUVC_F32) return LUVC_ERR_DTYPE;
-    if (B < 1 || H < 1 || W < 1 || D < 1 || target_count < 1) return LUVC_ERR_SHAPE;
+    {   // every argument rule of the device form, before anything is allocated or copied (host
+        // pointers need no alignment, so an aligned stand-in goes through the pointer checks)
+        luvc_oim_opts probe = {};
+        probe.dtype = dtype;
+        int hf = 0, wf = 0;
+        void* const aligned = reinterpret_cast<void*>(uintptr_t{256});
+        const int rc = check_oim(aligned, B, H, W, D, target_count, aligned, aligned, aligned, probe, &hf, &wf);
+        if (rc) return rc;
+    }
     const size_t es = elem_size(dtype), hw = (size_t)H * W;
     const size_t in_bytes = (size_t)B * hw * D * es;
     const size_t tok_bytes = align_up((size_t)B * target_count * D * es);
@@ -307,6 +377,7 @@ int luvc_spu_prune_ex(const void* hidden, int B, int N, int D, float cutoff, int
     int sigma = 0;
     const int rc = check_spu(hidden, B, N, D, cutoff, keep, out_idx, out_hidden, opts->dtype, &sigma);
     if (rc) return rc;
+    if (opts->device_status && (reinterpret_cast<uintptr_t>(opts->device_status) & 15u)) return LUVC_ERR_ALIGN;
     const size_t need = spu_workspace_bytes(B, N, D, sigma, opts->dtype);
     void* ws = opts->workspace;
     if (ws) {
@@ -320,7 +391,7 @@ int luvc_spu_prune_ex(const void* hidden, int B, int N, int D, float cutoff, int
     p.no_window = opts->no_window ? 1 : 0;
     p.out_idx = out_idx; p.out_hidden = out_hidden; p.out_scores = opts->out_scores;
     p.workspace = ws; p.stream = static_cast<cudaStream_t>(opts->stream);
-    p.status = status_word();
+    p.status = opts->device_status ? opts->device_status : status_word();
     if (!p.status) return LUVC_ERR_CUDA;
     return spu_run(p);
 }
@@ -382,8 +453,12 @@ int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, i
                         int32_t* out_idx, void* out_hidden) {
     if (!hidden || !out_idx || !out_hidden) return LUVC_ERR_NULL;
     if (dtype != LUVC_BF16 && dtype != LUVC_F32) return LUVC_ERR_DTYPE;
-    if (B < 1 || N < 1 || D < 1) return LUVC_ERR_SHAPE;
-    if (keep < 1 || keep > N) return LUVC_ERR_KEEP;
+    {   // the device form's argument rules first: nothing is allocated or copied for a bad request
+        int sigma = 0;
+        void* const aligned = reinterpret_cast<void*>(uintptr_t{256});
+        const int rc = check_spu(aligned, B, N, D, cutoff, keep, aligned, aligned, dtype, &sigma);
+        if (rc) return rc;
+    }
     const size_t es = elem_size(dtype);
     const size_t in_bytes = (size_t)B * N * D * es, hid_bytes = align_up((size_t)B * keep * D * es);
     unsigned char* din = static_cast<unsigned char*>(scratch(kIoInSpu, in_bytes));

@@ -30,11 +30,12 @@ struct OimStep {
 // Final grid for a target count; false if none fits.
 bool oim_final_dims(int H, int W, int target, int* Hf, int* Wf);
 // Step list from H x W to Hf x Wf; returns false if unreachable.  `steps` may be null (count only).
-bool oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first, OimStep* steps, int cap, int* n_steps);
+// r_w cells leave every row in a width step, r_h cells every column in a height step.
+bool oim_schedule(int H, int W, int Hf, int Wf, int r_w, int r_h, int height_first, OimStep* steps, int cap, int* n_steps);
 
 struct OimProblem {
     const void* tokens;
-    int B, H, W, D, Hf, Wf, r, height_first, dtype;
+    int B, H, W, D, Hf, Wf, r_w, r_h, height_first, dtype;
     int matching;   // luvc_oim_matching
     void* out_tokens;
     int32_t* out_sizes;
@@ -42,9 +43,13 @@ struct OimProblem {
     int32_t* trace;
     float* out_log_sizes;
     void* workspace;
-    int* status;   // device status word shared by all calls (0 = ok, else a luvc_status)
+    int* status;   // device status block: [0] 0 = ok, else a luvc_status; [1], [2] test knobs (see kStatusWords)
     cudaStream_t stream;
 };
+// Words of a status block.  [1] and [2] are zero in normal use; the wait-expiry test sets them:
+// [1] > 0 replaces the probe limit of the chain's waits, [2] is subtracted from the first image's
+// count of finished lines of the first step, so that the waits on it can never be satisfied.
+enum { kStatusWord = 0, kStatusProbeLimit = 1, kStatusHoldBack = 2, kStatusWords = 4 };
 size_t oim_workspace_bytes(int B, int H, int W, int D, int dtype, int matching = 0);
 int oim_run(const OimProblem& p);
 int oim_value_enhance(const void* values, const int32_t* sizes, long long rows, int D, int dtype, void* out,

@@ -106,23 +106,27 @@ __device__ __forceinline__ void pair_stats(const T* __restrict__ t0, const float
 
 // Set-up: identity grid, unit sizes, no parents, zeroed counters, and the step table
 // (the same rule the host uses to validate the request).
-__global__ void oim_setup_kernel(int32_t* cell, int32_t* size, int32_t* parent, int HW, long long total,
-                                 StepDesc* steps, int* done, int* next_item, int B, int H, int W, int Hf, int Wf,
-                                 int r, int height_first, int n_steps) {
+__global__ void oim_setup_kernel(int32_t* cell, int32_t* cell_b, int32_t* size, int32_t* parent, int32_t* cellpos,
+                                 int HW, long long total, StepDesc* steps, int* done, int* next_item,
+                                 const int* status, int B, int H, int W, int Hf, int Wf, int r_w, int r_h,
+                                 int height_first, int n_steps) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < total) {
         cell[i] = (int32_t)(i % HW);
+        cell_b[i] = (int32_t)(i % HW);     // never read before a step writes it; valid all the same
         size[i] = 1;
         parent[i] = -1;
+        cellpos[i] = 0;
     }
-    if (i < (long long)n_steps * B) done[i] = 0;
+    // the first counter starts below zero only when a test holds it back (its waits then run out)
+    if (i < (long long)n_steps * B) done[i] = i == 0 ? -status[kStatusHoldBack] : 0;
     if (i == 0) {
         *next_item = 0;
         int h = H, w = W, n = 0, item = 0, toff = 0;
         while ((h != Hf || w != Wf) && n < n_steps) {
             for (int turn = 0; turn < 2 && n < n_steps; ++turn) {
                 const int axis = height_first ? 1 - turn : turn;
-                const int len = axis == 0 ? w : h, goal = axis == 0 ? Wf : Hf;
+                const int len = axis == 0 ? w : h, goal = axis == 0 ? Wf : Hf, r = axis == 0 ? r_w : r_h;
                 int m = len - goal < r ? len - goal : r;
                 if (m > (len + 1) / 2) m = (len + 1) / 2;
                 if (len < 2 || m <= 0) continue;
@@ -147,6 +151,11 @@ __global__ void __launch_bounds__(THREADS, MINB) oim_chain_kernel(const ChainArg
     __shared__ int s_ok;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int D = a.D, B = a.B;
+    // a status word that is already set (this call's own failure elsewhere, or an earlier call's
+    // that nobody has read yet) stops the chain before it touches anything
+    if (tid == 0) s_ok = load_acquire(a.status) == 0 ? 1 : 0;
+    __syncthreads();
+    if (!s_ok) return;
     int step = 0;
     StepDesc st = a.steps[0];
     int step_end = a.n_steps > 1 ? a.steps[1].item_begin : a.total_items;
@@ -347,14 +356,16 @@ template <typename T>
 __global__ void __launch_bounds__(256) oim_emit_kernel(const void* tokens_v, const float* acc, const int32_t* cell,
                                                        const int32_t* size, int32_t* cellpos, void* out_v,
                                                        int32_t* out_sizes, float* out_log_sizes, int HW, int target,
-                                                       int D, long long total_cells) {
+                                                       int D, long long total_cells, const int* status) {
     constexpr int V = Elem<T>::kVec;
     const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (gw >= total_cells) return;
+    if (__ldcg(status) != 0) return;       // the chain gave up: its grids are unfinished, nothing is emitted
     const int b = (int)(gw / target), c = (int)(gw % target);
     const size_t img = (size_t)b * HW;
     const int root = (int)((unsigned)cell[img + c] & ~kMergedBit);
+    if (root >= HW) return;                // cannot happen after a finished chain; keeps every index in range
     const int s = size[img + root];
     const T* tok = reinterpret_cast<const T*>(tokens_v) + (img + root) * D;
     const float* arow = acc + (img + root) * D;
@@ -391,14 +402,15 @@ __global__ void __launch_bounds__(256) oim_emit_kernel(const void* tokens_v, con
 
 // Every source token follows its chain of merges to the root that survived.
 __global__ void oim_map_kernel(const int32_t* parent, const int32_t* cellpos, int32_t* out_map, int HW,
-                               long long total) {
+                               long long total, const int* status) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total) return;
+    if (__ldcg(status) != 0) return;
     const size_t img = (size_t)(i / HW) * HW;
     int r = (int)(i % HW);
     for (int hop = 0; hop < HW; ++hop) {   // a chain is shorter than the number of tokens
         const int p = parent[img + r];
-        if (p < 0) break;
+        if (p < 0 || p >= HW) break;
         r = p;
     }
     out_map[i] = cellpos[img + r];
@@ -460,14 +472,15 @@ bool oim_final_dims(int H, int W, int target, int* Hf, int* Wf) {
     return true;
 }
 
-bool oim_schedule(int H, int W, int Hf, int Wf, int r, int height_first, OimStep* steps, int cap, int* n_steps) {
-    if (Hf < 1 || Wf < 1 || Hf > H || Wf > W || r < 1) return false;
+bool oim_schedule(int H, int W, int Hf, int Wf, int r_w, int r_h, int height_first, OimStep* steps, int cap,
+                  int* n_steps) {
+    if (Hf < 1 || Wf < 1 || Hf > H || Wf > W || r_w < 1 || r_h < 1) return false;
     int h = H, w = W, n = 0;
     while (h != Hf || w != Wf) {
         bool moved = false;
         for (int turn = 0; turn < 2; ++turn) {
             const int axis = height_first ? 1 - turn : turn;
-            const int len = axis == 0 ? w : h, goal = axis == 0 ? Wf : Hf;
+            const int len = axis == 0 ? w : h, goal = axis == 0 ? Wf : Hf, r = axis == 0 ? r_w : r_h;
             int m = len - goal < r ? len - goal : r;
             if (m > (len + 1) / 2) m = (len + 1) / 2;   // only even-position cells can be merged away
             if (len < 2 || m <= 0) continue;
@@ -531,7 +544,7 @@ static int oim_run_typed(const OimProblem& p) {
     const int cap = (int)max_steps(p.H, p.W);
     OimStep* steps = new OimStep[cap];
     int n_steps = 0;
-    if (!oim_schedule(p.H, p.W, p.Hf, p.Wf, p.r, p.height_first, steps, cap, &n_steps) || n_steps > cap) {
+    if (!oim_schedule(p.H, p.W, p.Hf, p.Wf, p.r_w, p.r_h, p.height_first, steps, cap, &n_steps) || n_steps > cap) {
         delete[] steps;
         return LUVC_ERR_TARGET;
     }
@@ -543,8 +556,8 @@ static int oim_run_typed(const OimProblem& p) {
     phase_begin(LUVC_PHASE_OIM_TOTAL, p.stream);
     long long setup_threads = n > (long long)n_steps * p.B ? n : (long long)n_steps * p.B;
     oim_setup_kernel<<<(unsigned)((setup_threads + 255) / 256), 256, 0, p.stream>>>(
-        ws.cell_a, ws.size, ws.parent, HW, n, ws.steps, ws.done, ws.counters, p.B, p.H, p.W, p.Hf, p.Wf, p.r,
-        p.height_first, n_steps);
+        ws.cell_a, ws.cell_b, ws.size, ws.parent, ws.cellpos, HW, n, ws.steps, ws.done, ws.counters, p.status, p.B, p.H,
+        p.W, p.Hf, p.Wf, p.r_w, p.r_h, p.height_first, n_steps);
     count_launch();
     phase_begin(LUVC_PHASE_OIM_STEPS, p.stream);
     if (n_steps > 0) {
@@ -557,17 +570,18 @@ static int oim_run_typed(const OimProblem& p) {
         const int chunk = 32 * Elem<T>::kVec;
         const int nchunk = p.D % chunk == 0 ? p.D / chunk : 0;
         const int max_len = p.H > p.W ? p.H : p.W;
+        const int r_max = p.r_w > p.r_h ? p.r_w : p.r_h;
         cudaError_t err;
         if (p.matching == LUVC_OIM_MATCH_BIPARTITE) {
             err = oim_bipartite_prepare(a, ws.split, ws.nrm2, p.dtype, p.stream);
             count_launch();
-            if (err == cudaSuccess) err = oim_bipartite_launch(a, ws.split, ws.nrm2, p.dtype, max_len, p.r, p.stream);
+            if (err == cudaSuccess) err = oim_bipartite_launch(a, ws.split, ws.nrm2, p.dtype, max_len, r_max, p.stream);
         } else
         switch (nchunk) {
-            case 4: err = launch_chain<T, 4>(a, max_len, p.r, p.stream); break;
-            case 5: err = launch_chain<T, 5>(a, max_len, p.r, p.stream); break;
-            case 8: err = launch_chain<T, 8>(a, max_len, p.r, p.stream); break;
-            default: err = launch_chain<T, 0>(a, max_len, p.r, p.stream); break;
+            case 4: err = launch_chain<T, 4>(a, max_len, r_max, p.stream); break;
+            case 5: err = launch_chain<T, 5>(a, max_len, r_max, p.stream); break;
+            case 8: err = launch_chain<T, 8>(a, max_len, r_max, p.stream); break;
+            default: err = launch_chain<T, 0>(a, max_len, r_max, p.stream); break;
         }
         count_launch();
         if (err != cudaSuccess) return LUVC_ERR_CUDA;
@@ -577,9 +591,9 @@ static int oim_run_typed(const OimProblem& p) {
     const long long cells = (long long)p.B * target;
     oim_emit_kernel<T><<<(unsigned)((cells * 32 + 255) / 256), 256, 0, p.stream>>>(
         p.tokens, ws.acc, final_cell, ws.size, ws.cellpos, p.out_tokens, p.out_sizes, p.out_log_sizes, HW, target, p.D,
-        cells);
+        cells, p.status);
     count_launch();
-    oim_map_kernel<<<(unsigned)((n + 255) / 256), 256, 0, p.stream>>>(ws.parent, ws.cellpos, p.out_map, HW, n);
+    oim_map_kernel<<<(unsigned)((n + 255) / 256), 256, 0, p.stream>>>(ws.parent, ws.cellpos, p.out_map, HW, n, p.status);
     count_launch();
     phase_end(LUVC_PHASE_OIM_TOTAL, p.stream);
     return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;

@@ -79,9 +79,13 @@ __device__ __forceinline__ int load_acquire(const int* p) {
 }
 
 // Thread 0 of a CTA waits until *ctr reaches `target`.  Gives up after kSpinLimit probes (or as soon
-// as another CTA has reported a failure) and records LUVC_ERR_TIMEOUT in the status word.
+// as another CTA has reported a failure) and records LUVC_ERR_TIMEOUT in the status word.  The
+// second word of the status block, when positive, replaces the probe limit (test knob).
 __device__ __forceinline__ bool wait_for_count(const int* ctr, int target, int* status) {
-    for (int it = 0; it < kSpinLimit; ++it) {
+    if (load_acquire(ctr) >= target) return true;                   // the usual case: nothing else is read
+    const int knob = load_acquire(status + kStatusProbeLimit);      // 0 unless a test shortened the wait
+    const int limit = knob > 0 ? knob : kSpinLimit;
+    for (int it = 0; it < limit; ++it) {
         if (load_acquire(ctr) >= target) return true;
         if (load_acquire(status) != 0) return false;
         __nanosleep(it < 64 ? 32 : 256);

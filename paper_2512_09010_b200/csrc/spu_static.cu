@@ -5,8 +5,9 @@
 // loop in which an allocation's implicit device synchronisation is not acceptable, or code running
 // under a memory budget it has promised not to exceed.  The other SPU entry points either grow a
 // library-owned buffer with cudaMalloc or ask the caller for a workspace.  This one does neither:
-// its workspace is the fixed array below, which is part of the loaded module, so every device
-// that loads the library holds these bytes from load until exit.
+// its workspace is the fixed array below, which is part of the library's device image, so every
+// device that loads that image holds these bytes until the process exits (with lazy module
+// loading the image arrives with the first call on a device: see the warm-up note in luvc.h).
 //
 // The array's name is only a handle on the host side; the device address is looked up once per
 // device with cudaGetSymbolAddress (with that device current) and handed to the kernels.
@@ -77,4 +78,14 @@ extern "C" int luvc_spu_prune_static(const void* hidden, int B, int N, int D, fl
     p.status = reinterpret_cast<int*>(base);
     p.stream = stream;
     return spu_run(p);
+}
+
+extern "C" int luvc_spu_static_status(void* cuda_stream) {
+    unsigned char* base = nullptr;
+    const int rc = scratch_base(&base);
+    if (rc != LUVC_OK) return rc;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return LUVC_ERR_CUDA;
+    int host = 0;
+    if (cudaMemcpy(&host, base, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return LUVC_ERR_CUDA;
+    return host;
 }

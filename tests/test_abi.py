@@ -112,3 +112,48 @@ def test_argument_errors_of_the_added_entry_points(luvc):
     # the allocation-free prune checks its size limit before it touches the device
     assert L.luvc_spu_prune_static(fake, 8, 16384, 4096, 0.0, 4, 0, None, fake, fake) == 8
     assert L.luvc_spu_prune_static(fake, 1, 16, 8, 0.0, 17, 0, None, fake, fake) == 4
+
+
+def test_trace_size_status_alignment_and_host_forms_are_checked_first(luvc):
+    L = luvc.lib
+    fake = ctypes.c_void_p(4096)
+    o = luvc.OimOpts()
+    o.trace = 4096
+    o.trace_bytes = 2 * (16 - 4) * 4 - 1                 # B * (H*W - target) * 4 is needed
+    assert L.luvc_oim_merge_ex(fake, 2, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 8      # short trace buffer
+    o.trace_bytes = 0
+    assert L.luvc_oim_merge_ex(fake, 2, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 8
+    o = luvc.OimOpts()
+    o.device_status = 4100                                # not 16-byte aligned
+    assert L.luvc_oim_merge_ex(fake, 1, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 6
+    s = luvc.SpuOpts()
+    s.device_status = 4100
+    assert L.luvc_spu_prune_ex(fake, 1, 8, 8, 0.5, 2, fake, fake, ctypes.byref(s)) == 6
+    o = luvc.OimOpts()
+    o.merge_per_step_w = -1
+    assert L.luvc_oim_merge_ex(fake, 1, 4, 4, 8, 4, fake, fake, fake, ctypes.byref(o)) == 3
+    # host-buffer forms: every argument rule answers before anything is allocated or copied
+    assert L.luvc_oim_merge_host(fake, 1, 4, 4, 8, 7, 0, fake, fake, fake) == 3                    # 7 has no grid in 4 x 4
+    assert L.luvc_oim_merge_host(fake, 1, 4, 4, 8, 17, 0, fake, fake, fake) == 3                   # more than H*W
+    assert L.luvc_oim_merge_host(fake, 1, 4, 4, 12, 4, 0, fake, fake, fake) == 6
+    assert L.luvc_spu_prune_host(fake, 1, 8, 8, 2.0, 2, 0, fake, fake) == 5
+    assert L.luvc_spu_prune_host(fake, 1, 8, 8, 0.5, 9, 0, fake, fake) == 4
+    assert L.luvc_read_status(None, None) == 1
+    assert L.luvc_debug_wait_probes(-1, 0, None, None) == 2
+
+
+def test_aspect_ratio_plan_matches_the_hand_counted_schedules(luvc):
+    golden = os.path.join(ROOT, "tests", "golden", "oim_anyres_schedules.txt")
+    seen = 0
+    for line in open(golden):
+        f = line.split()
+        if not f or f[0] != "P":
+            continue
+        H, W, ops, r, r_h, r_w, Hf, Wf, steps = map(int, f[1:])
+        assert luvc.oim_plan_anyres(H, W, ops, r) == ((r_h, r_w), (Hf, Wf), steps)
+        seen += 1
+    assert seen >= 3
+    assert luvc.oim_plan_anyres(30, 40, 1) == ((2, 3), (28, 37), 2)          # merge number 0 = the appendix's 2
+    with pytest.raises(luvc.LuvcError) as e:
+        luvc.oim_plan_anyres(8, 40, 4, 2)
+    assert e.value.status == 3

@@ -105,16 +105,33 @@ def test_small_configurations_full(luvc, oracle_mod, config):
 
 
 @pytest.mark.parametrize("config", [2, 3, 4])
-def test_large_configurations_sampled_replay_and_invariants(luvc, oracle_mod, config):
-    # full size as benchmarked; the oracle replays a sample of the images, the invariants cover all
+def test_large_configurations_full_replay_and_invariants(luvc, oracle_mod, config):
+    # full size as benchmarked: the oracle replays EVERY image's decisions in double precision (a few
+    # seconds per configuration on the host cores) and the invariants are checked on top
     c = gi.CONFIGS[config]
     x = gi.oim_input(config, device="cuda")
     got = _run(luvc, x, target_count=c["target"])
     xh = x.float().cpu().numpy()
     Hf, Wf, _ = luvc.oim_plan(c["H"], c["W"], c["target"])
     check_oim_invariants(xh, got[0], got[1], got[2], c["dtype"], (c["H"], c["W"]), (Hf, Wf))
-    sample = sorted({0, c["B"] - 1})
-    check_oim_against_oracle(oracle_mod, xh, *got, c["dtype"], target=c["target"], images=sample)
+    check_oim_against_oracle(oracle_mod, xh, *got, c["dtype"], target=c["target"])
+
+
+def test_per_axis_merge_numbers_on_non_square_grids(luvc, oracle_mod):
+    # the appendix' aspect-ratio variant: the longer side loses more cells per step
+    g = torch.Generator().manual_seed(41)
+    for (H, W, ops), dtype in (((12, 24, 2), torch.float32), ((30, 20, 3), torch.bfloat16), ((9, 31, 1), torch.float32)):
+        (r_h, r_w), (Hf, Wf), n_steps = luvc.oim_plan_anyres(H, W, ops)
+        assert ((r_h, r_w), (Hf, Wf)) == oracle_mod.oim_anyres_plan(H, W, ops, 2)
+        x = torch.randn((2, H, W, 48), generator=g).to(dtype)
+        got = _run(luvc, x.cuda(), target_count=Hf * Wf, out_hw=(Hf, Wf), merge_per_step_hw=(r_h, r_w))
+        xh = x.float().numpy()
+        check_oim_against_oracle(oracle_mod, xh, *got, _name(x), out_hw=(Hf, Wf), r=(r_h, r_w))
+        check_oim_invariants(xh, got[0], got[1], got[2], _name(x), (H, W), (Hf, Wf))
+    # one axis' number alone; the other keeps the common one
+    x = torch.randn((1, 8, 20, 32), generator=g)
+    got = _run(luvc, x.cuda(), target_count=4 * 8, out_hw=(4, 8), merge_per_step_hw=(0, 5))
+    check_oim_against_oracle(oracle_mod, x.numpy(), *got, "f32", out_hw=(4, 8), r=(2, 5))
 
 
 def test_host_buffer_entry_point(luvc, oracle_mod):

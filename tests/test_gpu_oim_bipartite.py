@@ -96,7 +96,10 @@ def test_large_configurations_sampled_replay_and_invariants(luvc, oracle_mod, co
     xh = x.float().cpu().numpy()
     Hf, Wf, _ = luvc.oim_plan(c["H"], c["W"], c["target"])
     check_oim_invariants(xh, got[0], got[1], got[2], c["dtype"], (c["H"], c["W"]), (Hf, Wf), local=False)
-    check_oim_against_oracle(oracle_mod, xh, *got, c["dtype"], target=c["target"], images=[0], matching="bipartite")
+    # the oracle's full-line similarity matrices are slow at these sizes (a minute per 128 x 128 image and pass):
+    # a sample of the images is replayed, spread over the batch
+    sample = {2: [0, 3, 5, 7], 3: [0, 5, 10, 15, 16, 21, 26, 31], 4: [0, 3]}[config]
+    check_oim_against_oracle(oracle_mod, xh, *got, c["dtype"], target=c["target"], images=sample, matching="bipartite")
 
 
 def test_caller_workspace_needs_the_larger_size(luvc):

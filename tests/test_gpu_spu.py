@@ -136,27 +136,38 @@ def test_cascade_of_prunes(luvc, oracle_mod):
         x = luvc.spu_prune(x.cuda(), keep, 0.0)[1].cpu()
 
 
-def test_stress_configuration_sampled(luvc, oracle_mod):
-    # 8 x 16384 x 4096 as benchmarked; the oracle evaluates a sample of tokens from the definition
+def test_stress_configuration_whole_sequences_and_the_full_sweep(luvc, oracle_mod):
+    # 8 x 16384 x 4096 as benchmarked.  For each cutoff the oracle's FFT path scores ONE WHOLE sequence
+    # (a few seconds on the host cores): all 16384 scores are compared, and for each of the three keep
+    # counts the kept set of that sequence is judged against the ORACLE's scores.  The other sequences
+    # get the properties that hold at any size.
     c = gi.CONFIGS[4]
+    N = c["spu_N"]
     x = gi.spu_stress_input(device="cuda")
+    for (cutoff, b_ref) in zip(c["cutoffs"], (0, 3, 7)):
+        sigma = oracle_mod.spu_sigma(N, cutoff)
+        ref = oracle_mod.spu_scores(x[b_ref].float().cpu().numpy(), sigma)
+        for keep in c["keep"]:
+            idx, hid, scores = luvc.spu_prune(x, keep, cutoff, want_scores=True)
+            torch.cuda.synchronize()
+            idx_h, sc_h = idx.cpu().numpy(), scores.cpu().numpy()
+            assert_scores_close(sc_h[b_ref], ref, "sequence %d, cutoff %g" % (b_ref, cutoff))
+            if check_spu_selection(ref, idx_h[b_ref], keep):
+                np.testing.assert_array_equal(idx_h[b_ref], oracle_mod.spu_select(ref, keep))
+            for b in range(c["spu_B"]):
+                assert len(idx_h[b]) == keep and np.all(np.diff(idx_h[b]) > 0)
+                kept = np.zeros(N, bool)
+                kept[idx_h[b]] = True
+                assert sc_h[b][kept].min() >= sc_h[b][~kept].max()
+                assert torch.equal(hid[b], x[b][idx[b].long()])
+    # and a few tokens of other sequences straight from the definition (circular convolution with the filter's kernel)
     rng = np.random.default_rng(0)
-    for cutoff, keep in ((0.05, 1638), (0.125, 4096), (0.25, 8192)):
-        idx, hid, scores = luvc.spu_prune(x, keep, cutoff, want_scores=True)
-        torch.cuda.synchronize()
-        sigma = oracle_mod.spu_sigma(c["spu_N"], cutoff)
-        idx_h, sc_h = idx.cpu().numpy(), scores.cpu().numpy()
-        for b in (0, 7):
-            tokens = np.sort(rng.choice(c["spu_N"], size=6, replace=False))
-            ref = oracle_mod.spu_scores_at(x[b].float().cpu().numpy(), sigma, tokens)
-            assert_scores_close(sc_h[b][tokens], ref, "sampled scores, sequence %d" % b)
-        for b in range(c["spu_B"]):
-            # selection is consistent with the scores the kernel produced, exact in count and order
-            kept = np.zeros(c["spu_N"], bool)
-            kept[idx_h[b]] = True
-            assert len(idx_h[b]) == keep and np.all(np.diff(idx_h[b]) > 0)
-            assert sc_h[b][kept].min() >= sc_h[b][~kept].max()
-            assert torch.equal(hid[b], x[b][idx[b].long()])
+    idx, hid, scores = luvc.spu_prune(x, c["keep"][0], c["cutoffs"][0], want_scores=True)
+    sigma = oracle_mod.spu_sigma(N, c["cutoffs"][0])
+    for b in (2, 5):
+        tokens = np.sort(rng.choice(N, size=6, replace=False))
+        ref_at = oracle_mod.spu_scores_at(x[b].float().cpu().numpy(), sigma, tokens)
+        assert_scores_close(scores[b].cpu().numpy()[tokens], ref_at, "sampled scores, sequence %d" % b)
 
 
 def test_cascade_entry_point(luvc, oracle_mod):

@@ -31,7 +31,35 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point(luvc, dtype):
         assert torch.equal(idx, ref_idx)
         assert torch.equal(hid, ref_hid)
         assert torch.equal(hid, torch.stack([x[b][idx[b].long()] for b in range(B)]))
+        assert luvc.lib.luvc_spu_static_status(torch.cuda.current_stream().cuda_stream) == 0
     assert luvc.check_status() == 0
+
+
+def test_a_warmed_up_call_reserves_no_device_memory(luvc):
+    # outputs made beforehand, the C entry point called directly: after one warm-up call (which loads the
+    # library's device image and the kernels' code) a second call must leave the device's free memory as it was
+    import ctypes
+    g = torch.Generator().manual_seed(2513)
+    B, N, D, keep = 2, 192, 136, 40
+    x = torch.randn((B, N, D), generator=g).to(torch.bfloat16).cuda()
+    out_idx = torch.empty((B, keep), dtype=torch.int32, device="cuda")
+    out_hid = torch.empty((B, keep, D), dtype=torch.bfloat16, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        return luvc.lib.luvc_spu_prune_static(x.data_ptr(), B, N, D, ctypes.c_float(0.25), keep, luvc.BF16, stream,
+                                              out_idx.data_ptr(), out_hid.data_ptr())
+
+    assert call() == 0                                   # warm-up
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    assert call() == 0
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert luvc.lib.luvc_spu_static_status(stream) == 0
+    ref_idx, ref_hid = luvc.spu_prune(x, keep, 0.25)
+    assert torch.equal(out_idx, ref_idx) and torch.equal(out_hid, ref_hid)
 
 
 def test_sizes_beyond_the_fixed_array_are_refused(luvc):
