@@ -121,7 +121,6 @@ __global__ void oim_setup_kernel(int32_t* cell, int32_t* cell_b, int32_t* size, 
     // the first counter starts below zero only when a test holds it back (its waits then run out)
     if (i < (long long)n_steps * B) done[i] = i == 0 ? -status[kStatusHoldBack] : 0;
     if (i == 0) {
-        *next_item = 0;
         int h = H, w = W, n = 0, item = 0, toff = 0;
         while ((h != Hf || w != Wf) && n < n_steps) {
             for (int turn = 0; turn < 2 && n < n_steps; ++turn) {
@@ -138,6 +137,10 @@ __global__ void oim_setup_kernel(int32_t* cell, int32_t* cell_b, int32_t* size, 
                 if (axis == 0) w -= m; else h -= m;
             }
         }
+        // A status word that is already set (an earlier call's failure that nobody has read yet) stops
+        // this call before it starts: the work counter begins past the last item, so the chain's CTAs
+        // find nothing to claim (and the emit and map kernels look at the word themselves).
+        *next_item = status[kStatusWord] != 0 ? item : 0;
     }
 }
 
@@ -151,11 +154,6 @@ __global__ void __launch_bounds__(THREADS, MINB) oim_chain_kernel(const ChainArg
     __shared__ int s_ok;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int D = a.D, B = a.B;
-    // a status word that is already set (this call's own failure elsewhere, or an earlier call's
-    // that nobody has read yet) stops the chain before it touches anything
-    if (tid == 0) s_ok = load_acquire(a.status) == 0 ? 1 : 0;
-    __syncthreads();
-    if (!s_ok) return;
     int step = 0;
     StepDesc st = a.steps[0];
     int step_end = a.n_steps > 1 ? a.steps[1].item_begin : a.total_items;
