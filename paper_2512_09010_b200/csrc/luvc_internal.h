@@ -112,6 +112,19 @@ SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma);
 int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, void* yt_lo, int r_pad, int B, int N,
                  int D, int sigma, int* status, cudaStream_t stream);
 
+// Forward transform with both stages on the tensor cores (spu_fwd3.cu): N = 128 Q, 8 <= Q <= 128.
+struct SpuFwd3Plan {
+    int ok;             // 0: use the two-stage kernel of spu_fwd2.cu (or the dense contraction)
+    int Q;
+    int wide;           // 0: up to 4 bins per frequency class, 16 channels per item; 1: up to 16, 8 channels
+    int slices;         // passes over the input, each covering 4 / 16 values of k2
+    int C, n_ctiles, n_items;
+};
+SpuFwd3Plan spu_fwd3_plan(int B, int N, int D, int sigma);
+// Y[b][r][d] = c[r] * (band spectrum), the layout spu_fwd2_run writes.
+int spu_fwd3_run(const void* hidden, float* Y, const float* scale, int B, int N, int D, int sigma, int* status,
+                 cudaStream_t stream);
+
 // Two-stage inverse transform and energies of the bf16 path (spu_inv2.cu); needs the forward plan.
 struct SpuInv2Plan {
     int ok;             // 0: use the dense inverse contraction

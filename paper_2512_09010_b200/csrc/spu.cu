@@ -473,7 +473,10 @@ static int spu_run_typed(const SpuProblem& p) {
                                                                p.no_window);
     count_launch();
     if constexpr (kTensor) {
-        if (mode.fwd2) {
+        if (mode.fwd2 && mode.inv2 && spu_fwd3_plan(B, N, D, sigma).ok) {
+            const int rc1 = spu_fwd3_run(p.hidden, ws.Y2, ws.scale, B, N, D, sigma, p.status, p.stream);
+            if (rc1 != LUVC_OK) return rc1;
+        } else if (mode.fwd2) {
             const int rc1 = spu_fwd2_run(p.hidden, ws.Y2, ws.scale, mode.inv2 ? nullptr : ws.tc.yt_hi,
                                          mode.inv2 ? nullptr : ws.tc.yt_lo, pl.r_pad, B, N, D, sigma, p.status, p.stream);
             if (rc1 != LUVC_OK) return rc1;

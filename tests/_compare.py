@@ -97,7 +97,21 @@ def check_spu_selection(scores_ref, gpu_idx, keep):
 
 
 def assert_scores_close(gpu_scores, ref, what="scores"):
-    scale = np.abs(ref).max() if ref.size else 1.0
-    err = np.abs(gpu_scores.astype(np.float64) - ref)
-    bound = 1e-4 * np.abs(ref) + 1e-6 * scale
-    assert np.all(err <= bound), "%s: worst relative error %.3g" % (what, float((err / (np.abs(ref) + 1e-30)).max()))
+    """Energies of Eq. 8 against the oracle's.  A score is the norm of a filtered signal (Eq. 7) that,
+    next to a strong token, is a sum of large ringing terms of both signs: arithmetic that carries
+    16-17 significant bits per operand (fp32 accumulation of bf16-pair products, 2^-17 = 7.6e-6)
+    is exact relative to those TERMS, not to their sum, which can be a hundred times smaller in a
+    null of the ringing.  So the bound is 1e-4 of the score itself plus 1e-5 of the largest score
+    within 32 tokens (circular); half of all scores must still agree to 1e-5 of themselves."""
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(gpu_scores, dtype=np.float64)
+    n = ref.shape[0]
+    local = ref.copy()
+    for shift in range(1, min(32, n - 1) + 1):
+        local = np.maximum(local, np.maximum(np.roll(ref, shift), np.roll(ref, -shift)))
+    err = np.abs(got - ref)
+    bound = 1e-4 * np.abs(ref) + 1e-5 * local
+    worst = float((err / (np.abs(ref) + 1e-30)).max()) if n else 0.0
+    assert np.all(err <= bound), "%s: worst relative error %.3g" % (what, worst)
+    if n >= 16:
+        assert np.median(err / (np.abs(ref) + 1e-30)) <= 1e-5, "%s: median relative error too large" % what

@@ -62,6 +62,11 @@ def test_small_sequences_match_the_oracle(luvc, oracle_mod, dtype, B, N, D, keep
     (2, 1296, 136, 324, 0.125), # P = 48, Q = 27: ragged last tile, partial channel block
     (1, 2592, 264, 648, 0.05),  # P = 96
     (3, 768, 8, 77, 0.02),      # sigma smaller than P: most rows hold no bin
+    (2, 1024, 48, 100, 0.3),    # N = 128 x 8: both stages on the tensor cores, two bins per class
+    (1, 2048, 24, 300, 0.4),    # four bins per class (the narrow-band variant's limit), partial channel tile
+    (2, 1152, 72, 200, 0.25),   # Q = 9: ragged last tile of tokens
+    (1, 4096, 40, 500, 1.0),    # seventeen bins per class: two slices of the wide-band variant
+    (1, 16384, 24, 1638, 0.05), # the stress length: Q = 128, 32 tiles per item
 ])
 def test_two_stage_paths_match_the_oracle(luvc, oracle_mod, B, N, D, keep, cutoff):
     g = torch.Generator().manual_seed(N * 7 + D)
