@@ -305,7 +305,11 @@ int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, i
  * keeps, cutoffs  HOST arrays of n_stages entries; 1 <= keeps[t] <= keeps[t-1] <= N
  * out_idx     [B, keeps[n_stages-1]] int32  surviving tokens as indices into the ORIGINAL sequence, ascending
  * out_hidden  [B, keeps[n_stages-1], D]     their rows, bit-exact copies
- * Intermediate survivors live in library-owned scratch (grown with cudaMalloc on demand).
+ * A later stage reads its rows straight out of `hidden`, through the list of survivors composed so far
+ * (gather on load): the survivors' rows are written once, by the last stage.  Only a stage whose
+ * sequence is long enough for the two-stage transform kernels (which walk dense memory) has its rows
+ * copied into library-owned scratch first.  Index lists and the transform workspace live in
+ * library-owned scratch (grown with cudaMalloc on demand; see the note on overlapping calls above).
  * Dropping the last survivors altogether, as the paper does at the final layer, needs no kernel.
  */
 int luvc_spu_cascade(const void* hidden, int B, int N, int D, int n_stages, const int* keeps, const float* cutoffs,

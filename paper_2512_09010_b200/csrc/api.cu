@@ -425,28 +425,64 @@ int luvc_spu_cascade(const void* hidden, int B, int N, int D, int n_stages, cons
     luvc_spu_opts o = {};
     o.dtype = dtype; o.stream = cuda_stream;
     if (n_stages == 1) return luvc_spu_prune_ex(hidden, B, N, D, cutoffs ? cutoffs[0] : 0.f, keeps[0], out_idx, out_hidden, &o);
-    // scratch: two buffers of survivors' rows (ping-pong) and three index arrays (stage, total so far, new total)
+    {   // pointer and row-size rules of a single prune (the stages run through the internal entry point)
+        int sg = 0;
+        const int rc = check_spu(hidden, B, N, D, cutoffs ? cutoffs[0] : 0.f, keeps[0], out_idx, out_hidden, dtype, &sg);
+        if (rc) return rc;
+    }
+    // Stage t > 0 reads the survivors' rows straight out of `hidden` through the index list composed so far
+    // (gather on load) whenever a sequence of that length runs the dense contractions anyway; only a stage
+    // long enough for the two-stage kernels, which walk dense memory, gets its rows copied out first.  The
+    // survivors' rows are written once, by the last stage.
     const size_t es = elem_size(dtype);
-    const size_t rows = align_up((size_t)B * keeps[0] * D * es), idxb = align_up((size_t)B * keeps[0] * 4);
-    unsigned char* sc = static_cast<unsigned char*>(scratch(kCascade, 2 * rows + 3 * idxb));
-    if (!sc) return LUVC_ERR_CUDA;
-    void* buf[2] = {sc, sc + rows};
-    int32_t* idx_stage = reinterpret_cast<int32_t*>(sc + 2 * rows);
-    int32_t* idx_tot[2] = {reinterpret_cast<int32_t*>(sc + 2 * rows + idxb), reinterpret_cast<int32_t*>(sc + 2 * rows + 2 * idxb)};
-    const void* in = hidden;
+    int sigmas[64];
+    if (n_stages > 64) return LUVC_ERR_SHAPE;
+    size_t ws_need = 0, rows_need = 0;
     int n_in = N;
     for (int t = 0; t < n_stages; ++t) {
-        const bool last = t == n_stages - 1;
-        void* out_rows = last ? out_hidden : buf[t & 1];
-        int rc = luvc_spu_prune_ex(in, B, n_in, D, cutoffs ? cutoffs[t] : 0.f, keeps[t], idx_stage, out_rows, &o);
-        if (rc) return rc;
-        int32_t* tot = last ? out_idx : idx_tot[t & 1];
-        rc = spu_compose_indices(t == 0 ? nullptr : idx_tot[(t - 1) & 1], idx_stage, tot, B, t == 0 ? 0 : keeps[t - 1], keeps[t], st);
-        if (rc) return rc;
-        in = out_rows;
+        sigmas[t] = luvc_spu_sigma(n_in, cutoffs ? cutoffs[t] : 0.f);
+        if (sigmas[t] < 0) return LUVC_ERR_CUTOFF;
+        const bool fuse = t > 0 && spu_dense_is_natural(B, n_in, D, sigmas[t], dtype);
+        const size_t need = spu_workspace_bytes(B, n_in, D, sigmas[t], dtype, fuse);
+        ws_need = need > ws_need ? need : ws_need;
+        if (t > 0 && !fuse) rows_need = align_up((size_t)B * n_in * D * es) > rows_need ? align_up((size_t)B * n_in * D * es) : rows_need;
         n_in = keeps[t];
     }
-    return LUVC_OK;
+    const size_t idxb = align_up((size_t)B * keeps[0] * 4);
+    unsigned char* sc = static_cast<unsigned char*>(scratch(kCascade, rows_need + 3 * idxb));
+    void* ws = scratch(kSpuWs, ws_need);
+    int* status = status_word();
+    if (!sc || !ws || !status) return LUVC_ERR_CUDA;
+    void* rows_buf = sc;
+    int32_t* idx_stage = reinterpret_cast<int32_t*>(sc + rows_need);
+    int32_t* idx_tot[2] = {reinterpret_cast<int32_t*>(sc + rows_need + idxb), reinterpret_cast<int32_t*>(sc + rows_need + 2 * idxb)};
+    const int32_t* cur = nullptr;      // survivors so far as rows of `hidden` (null: all N, in order)
+    n_in = N;
+    for (int t = 0; t < n_stages; ++t) {
+        const bool last = t == n_stages - 1;
+        const bool fuse = t > 0 && spu_dense_is_natural(B, n_in, D, sigmas[t], dtype);
+        SpuProblem p;
+        p.B = B; p.N = n_in; p.D = D; p.sigma = sigmas[t]; p.keep = keeps[t]; p.dtype = dtype; p.no_window = 0;
+        p.out_idx = idx_stage; p.out_hidden = nullptr; p.out_scores = nullptr;
+        p.workspace = ws; p.status = status; p.stream = st;
+        if (t == 0) {
+            p.hidden = hidden;
+        } else if (fuse) {
+            p.hidden = hidden; p.row_index = cur; p.src_rows = N;
+        } else {
+            int rc = spu_gather_rows(hidden, cur, rows_buf, B, N, n_in, D, dtype, st);
+            if (rc) return rc;
+            p.hidden = rows_buf;
+        }
+        int rc = spu_run(p);
+        if (rc) return rc;
+        int32_t* tot = last ? out_idx : idx_tot[t & 1];
+        rc = spu_compose_indices(cur, idx_stage, tot, B, t == 0 ? 0 : keeps[t - 1], keeps[t], st);
+        if (rc) return rc;
+        cur = tot;
+        n_in = keeps[t];
+    }
+    return spu_gather_rows(hidden, out_idx, out_hidden, B, N, keeps[n_stages - 1], D, dtype, st);
 }
 
 int luvc_spu_prune_host(const void* hidden, int B, int N, int D, float cutoff, int keep, int dtype,

@@ -60,15 +60,26 @@ int oim_value_enhance(const void* values, const int32_t* sizes, long long rows, 
 struct SpuProblem {
     const void* hidden;
     int B, N, D, sigma, keep, dtype, no_window;
+    // Gather on load (the cascade): when row_index is given, token n of sequence b is row
+    // row_index[b][n] of sequence b of `hidden`, which then holds src_rows rows per sequence.
+    const int32_t* row_index = nullptr;
+    int src_rows = 0;
     int32_t* out_idx;
-    void* out_hidden;
+    void* out_hidden;   // may be null: no rows are gathered (the caller does it later)
     float* out_scores;
     void* workspace;
     int* status;   // device status word (see OimProblem)
     cudaStream_t stream;
 };
-size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype);
+// `indexed`: the problem reads its rows through a row index (only the dense contractions can).
+size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype, bool indexed = false);
 int spu_run(const SpuProblem& p);
+// True when a sequence of N tokens would run the dense band contractions anyway (no two-stage plan),
+// i.e. when reading it through a row index costs nothing extra.
+bool spu_dense_is_natural(int B, int N, int D, int sigma, int dtype);
+// out[b][j][:] = hidden[b][idx[b][j]][:] (hidden holds n_src rows per sequence)
+int spu_gather_rows(const void* hidden, const int32_t* idx, void* out, int B, int n_src, int keep, int D, int dtype,
+                    cudaStream_t stream);
 // out[b][j] = prev[b][cur[b][j]] (prev == nullptr: out = cur)
 int spu_compose_indices(const int32_t* prev, const int32_t* cur, int32_t* out, int B, int n_prev, int keep,
                         cudaStream_t stream);
@@ -95,8 +106,10 @@ SpuTcPlan spu_tc_plan(int B, int N, int D, int sigma);
 // of the plan.  `scale` must hold r_pad entries (zero beyond 2 sigma + 1); `tw2` is the table of
 // cos / sin of 2 pi j / L (used when the plan is coarse).
 // With `have_yt` the spectrum (yt_hi / yt_lo) is already in place and only the inverse pass runs.
+// row_index / src_rows: see SpuProblem (null: the rows are those of `hidden` in order).
 int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float2* tw2, const float* scale,
-               int B, int N, int D, int sigma, int* status, cudaStream_t stream, bool have_yt);
+               int B, int N, int D, int sigma, int* status, cudaStream_t stream, bool have_yt,
+               const int32_t* row_index = nullptr, int src_rows = 0);
 
 // Two-stage forward transform of the bf16 path (spu_fwd2.cu): N = P * Q, P a multiple of 16.
 struct SpuFwd2Plan {

@@ -74,14 +74,16 @@ __global__ void __launch_bounds__(kGemmThreads) spu_contract_kernel(const void* 
                                                                     float* __restrict__ out,
                                                                     const float2* __restrict__ tw,
                                                                     const float* __restrict__ scale,
-                                                                    int N, int D, int sigma) {
+                                                                    int N, int D, int sigma,
+                                                                    const int32_t* __restrict__ rows, int src_rows) {
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int R = 2 * sigma + 1;
     const int M = FWD ? R : N, K = FWD ? N : R;
     const int b = blockIdx.z, m0 = blockIdx.y * BM, d0 = blockIdx.x * BN;
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    const T* xin = reinterpret_cast<const T*>(bm_v) + (size_t)b * N * D;          // FWD operand
+    const T* xin = reinterpret_cast<const T*>(bm_v) + (size_t)b * (rows ? src_rows : N) * D;   // FWD operand
+    const int32_t* rowb = rows ? rows + (size_t)b * N : nullptr;                  // gather on load: token -> row
     const float* yin = reinterpret_cast<const float*>(bm_v) + (size_t)b * R * D;  // !FWD operand
 
     float acc[4][4];
@@ -106,7 +108,8 @@ __global__ void __launch_bounds__(kGemmThreads) spu_contract_kernel(const void* 
             const int ni = idx % BN, ki = idx / BN;
             const int red = k0 + ki, d = d0 + ni;
             float v = 0.f;
-            if (red < K && d < D) v = FWD ? to_f32<T>(xin[(size_t)red * D + d]) : yin[(size_t)red * D + d];
+            if (red < K && d < D)
+                v = FWD ? to_f32<T>(xin[(size_t)(rowb ? __ldg(rowb + red) : red) * D + d]) : yin[(size_t)red * D + d];
             Bs[ki][ni] = v;
         }
         __syncthreads();
@@ -393,11 +396,12 @@ struct Bf16Mode {
     int coarse, L;      // the inverse is evaluated on L uniform points of the period (L = N: the tokens)
     int n_parts;        // partial energy sums per point
 };
-Bf16Mode bf16_mode(int B, int N, int D, int sigma) {
+Bf16Mode bf16_mode(int B, int N, int D, int sigma, bool dense) {
     const SpuTcPlan tc = spu_tc_plan(B, N, D, sigma);
     const SpuInv2Plan iv = spu_inv2_plan(B, N, D, sigma);
     Bf16Mode m;
-    m.fwd2 = spu_fwd2_plan(B, N, D, sigma).ok != 0;
+    m.fwd2 = !dense && spu_fwd2_plan(B, N, D, sigma).ok != 0;   // `dense`: rows come through an index, which only
+                                                                // the dense contractions can follow
     m.inv2 = m.fwd2 && iv.ok != 0;
     m.coarse = m.inv2 ? iv.coarse : tc.coarse;
     m.L = m.inv2 ? iv.L : tc.L;
@@ -411,7 +415,7 @@ size_t coarse_gpart_elems(int B, int L, int sigma) {
 
 // Both paths share the twiddle table, the row constants and the scores; the rest differs.
 // With ws == nullptr only the size is computed.
-Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path, size_t* total) {
+Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path, bool dense, size_t* total) {
     unsigned char* p = static_cast<unsigned char*>(ws);
     unsigned char* const p0 = p;
     const int R = 2 * sigma + 1, tiles = (D + BN - 1) / BN;
@@ -425,7 +429,7 @@ Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path, size
         w.Y = reinterpret_cast<float*>(take((size_t)B * R * D * 4));
         w.part = reinterpret_cast<float*>(take((size_t)B * tiles * N * 4));
     } else {
-        const Bf16Mode m = bf16_mode(B, N, D, sigma);
+        const Bf16Mode m = bf16_mode(B, N, D, sigma, dense);
         if (m.coarse) {
             w.S = reinterpret_cast<float*>(take((size_t)B * m.L * 4));
             w.gpart = reinterpret_cast<float2*>(take(coarse_gpart_elems(B, m.L, sigma) * sizeof(float2)));
@@ -452,10 +456,14 @@ Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path, size
 
 }  // namespace
 
-size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype) {
+size_t spu_workspace_bytes(int B, int N, int D, int sigma, int dtype, bool indexed) {
     size_t total = 0;
-    carve(nullptr, B, N, D, sigma, dtype != LUVC_F32, &total);
+    carve(nullptr, B, N, D, sigma, dtype != LUVC_F32, indexed, &total);
     return total;
+}
+
+bool spu_dense_is_natural(int B, int N, int D, int sigma, int dtype) {
+    return dtype == LUVC_F32 || !spu_fwd2_plan(B, N, D, sigma).ok;
 }
 
 template <typename T>
@@ -463,9 +471,10 @@ static int spu_run_typed(const SpuProblem& p) {
     constexpr bool kTensor = sizeof(T) == 2;     // bf16 tokens go through the tensor cores
     const int N = p.N, D = p.D, B = p.B, sigma = p.sigma, R = 2 * sigma + 1;
     const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
-    Workspace ws = carve(p.workspace, B, N, D, sigma, kTensor, nullptr);
+    const bool indexed = p.row_index != nullptr;
+    Workspace ws = carve(p.workspace, B, N, D, sigma, kTensor, indexed, nullptr);
     float* E = p.out_scores ? p.out_scores : ws.E;
-    const Bf16Mode mode = kTensor ? bf16_mode(B, N, D, sigma) : Bf16Mode{};
+    const Bf16Mode mode = kTensor ? bf16_mode(B, N, D, sigma, indexed) : Bf16Mode{};
     const int tab = max(max(N, pl.r_pad), pl.L);
     const long long bn = (long long)B * N;
     phase_begin(LUVC_PHASE_SPU_TRANSFORM, p.stream);
@@ -483,7 +492,7 @@ static int spu_run_typed(const SpuProblem& p) {
         }
         const int rc = mode.inv2 ? spu_inv2_run(ws.Y2, ws.tc.part, B, N, D, sigma, p.status, p.stream)
                                  : spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status,
-                                              p.stream, mode.fwd2);
+                                              p.stream, mode.fwd2, p.row_index, p.src_rows);
         if (rc != LUVC_OK) return rc;
         if (!mode.coarse) {
             spu_energy_kernel<<<(unsigned)((bn + 31) / 32), 256, 0, p.stream>>>(ws.tc.part, E, N, mode.n_parts, bn, 0);
@@ -499,9 +508,9 @@ static int spu_run_typed(const SpuProblem& p) {
     } else {
         const int tiles = (D + BN - 1) / BN;
         spu_contract_kernel<T, true><<<dim3(tiles, (R + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
-            p.hidden, ws.Y, ws.tw, ws.scale, N, D, sigma);
+            p.hidden, ws.Y, ws.tw, ws.scale, N, D, sigma, p.row_index, p.src_rows);
         spu_contract_kernel<T, false><<<dim3(tiles, (N + BM - 1) / BM, B), kGemmThreads, 0, p.stream>>>(
-            ws.Y, ws.part, ws.tw, ws.scale, N, D, sigma);
+            ws.Y, ws.part, ws.tw, ws.scale, N, D, sigma, nullptr, 0);
         spu_energy_kernel<<<(unsigned)((bn + 31) / 32), 256, 0, p.stream>>>(ws.part, E, N, tiles, bn, 0);
         count_launch(3);
     }
@@ -509,12 +518,24 @@ static int spu_run_typed(const SpuProblem& p) {
     phase_begin(LUVC_PHASE_SPU_SELECT, p.stream);
     spu_select_kernel<<<B, kSelThreads, 0, p.stream>>>(E, p.out_idx, N, p.keep);
     phase_end(LUVC_PHASE_SPU_SELECT, p.stream);
-    phase_begin(LUVC_PHASE_SPU_GATHER, p.stream);
-    const int row_vec = (int)((size_t)D * sizeof(T) / 16);
-    spu_gather_kernel<<<dim3(p.keep, B), 128, 0, p.stream>>>(reinterpret_cast<const uint4*>(p.hidden), p.out_idx,
-                                                            reinterpret_cast<uint4*>(p.out_hidden), N, p.keep, row_vec);
-    phase_end(LUVC_PHASE_SPU_GATHER, p.stream);
-    count_launch(2);
+    count_launch();
+    if (p.out_hidden != nullptr && !indexed) {
+        phase_begin(LUVC_PHASE_SPU_GATHER, p.stream);
+        const int row_vec = (int)((size_t)D * sizeof(T) / 16);
+        spu_gather_kernel<<<dim3(p.keep, B), 128, 0, p.stream>>>(reinterpret_cast<const uint4*>(p.hidden), p.out_idx,
+                                                                reinterpret_cast<uint4*>(p.out_hidden), N, p.keep, row_vec);
+        phase_end(LUVC_PHASE_SPU_GATHER, p.stream);
+        count_launch();
+    }
+    return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
+}
+
+int spu_gather_rows(const void* hidden, const int32_t* idx, void* out, int B, int n_src, int keep, int D, int dtype,
+                    cudaStream_t stream) {
+    const int row_vec = (int)((size_t)D * (dtype == LUVC_F32 ? 4 : 2) / 16);
+    spu_gather_kernel<<<dim3(keep, B), 128, 0, stream>>>(reinterpret_cast<const uint4*>(hidden), idx,
+                                                         reinterpret_cast<uint4*>(out), n_src, keep, row_vec);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
 

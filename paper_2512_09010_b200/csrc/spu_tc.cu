@@ -113,6 +113,8 @@ struct TcArgs {
     const __nv_bfloat16* a[2];   // A parts: element (k, m) at a[p][batch * a_batch + k * lda + m]
     const __nv_bfloat16* b[2];   // B parts: element (nn, k) at b[p][batch * b_batch + nn * ldb + k]
     long long a_batch, b_batch;
+    const int32_t* a_rows;       // optional: row k of A is row a_rows[batch * a_rows_stride + k] of a[0] (gather on load)
+    int a_rows_stride;
     int lda, ldb;
     int m_total;                 // valid extent of the M index (multiple of 8)
     int n_total;                 // valid extent of the N index (rows of B)
@@ -175,7 +177,9 @@ __global__ void __launch_bounds__(kThreads, 1) spu_tc_kernel(const TcArgs g) {
                 const int m = m0 + grp * 8, kk = k0 + k;
                 const bool ok = m < g.m_total && kk < g.k_a;
                 const uint32_t dst = sbase + p * kABytes + grp * kASbo + (k >> 3) * kALbo + (k & 7) * 16;
-                cp_async16(dst, ok ? (const void*)(src + (size_t)kk * g.lda + m) : (const void*)src, ok);
+                const size_t row = (ok && g.a_rows != nullptr) ? (size_t)__ldg(g.a_rows + (size_t)batch * g.a_rows_stride + kk)
+                                                               : (size_t)kk;
+                cp_async16(dst, ok ? (const void*)(src + row * g.lda + m) : (const void*)src, ok);
             }
         }
         // B parts: tn rows x 8 K-chunks of 16 bytes
@@ -330,7 +334,8 @@ SpuTcPlan spu_tc_plan(int B, int N, int D, int sigma) {
 }
 
 int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, const float2* tw2, const float* scale,
-               int B, int N, int D, int sigma, int* status, cudaStream_t stream, bool have_yt) {
+               int B, int N, int D, int sigma, int* status, cudaStream_t stream, bool have_yt,
+               const int32_t* row_index, int src_rows) {
     const SpuTcPlan pl = spu_tc_plan(B, N, D, sigma);
     if (!have_yt || !pl.coarse) {
         const long long phi_n = (long long)pl.phi_elems;
@@ -353,7 +358,8 @@ int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, cons
         g.a[0] = reinterpret_cast<const __nv_bfloat16*>(hidden); g.a[1] = nullptr;
         g.b[0] = reinterpret_cast<const __nv_bfloat16*>(w.phi_hi);
         g.b[1] = reinterpret_cast<const __nv_bfloat16*>(w.phi_lo);
-        g.a_batch = (long long)N * D; g.b_batch = 0;
+        g.a_batch = (long long)(row_index ? src_rows : N) * D; g.b_batch = 0;
+        g.a_rows = row_index; g.a_rows_stride = N;
         g.lda = D; g.ldb = pl.n_pad;
         g.m_total = D; g.n_total = pl.r_pad; g.k_a = N; g.k_blocks = (N + TK - 1) / TK;
         const int tiles = (pl.r_pad + 255) / 256;

@@ -179,7 +179,10 @@ def test_cascade_entry_point(luvc, oracle_mod):
     # luvc_spu_cascade against the same stages composed by hand, and against the oracle's loop where
     # every stage of the oracle has a unique answer
     g = torch.Generator().manual_seed(21)
+    # second case of the list: the second stage (1024 tokens) is long enough for the two-stage kernels, so its
+    # rows are copied out first; the stages after it read through the index list again
     for dtype, shape, keeps, cutoffs in ((torch.bfloat16, (2, 1296, 136), (324, 130, 65), None),
+                                         (torch.bfloat16, (1, 2048, 40), (1024, 300, 77, 5), (0.25, 0.125, 0.0, 0.5)),
                                          (torch.float32, (1, 200, 64), (120, 60, 7), (0.3, 0.0, 1.0)),
                                          (torch.bfloat16, (3, 96, 72), (40,), (0.25,))):
         x = torch.randn(shape, generator=g).to(dtype)
