@@ -131,6 +131,7 @@ struct SpuFwd3Plan {
     int Q;
     int wide;           // 0: up to 4 bins per frequency class, 16 channels per item; 1: up to 16, 8 channels
     int slices;         // passes over the input, each covering 4 / 16 values of k2
+    int extra_k2;       // > 0: this one further value of k2 is kept on the CUDA cores (no second pass for it)
     int C, n_ctiles, n_items;
 };
 SpuFwd3Plan spu_fwd3_plan(int B, int N, int D, int sigma);

@@ -59,6 +59,8 @@ struct Fwd3Args {
     int* status;
     int B, N, D, Q, sigma, R;
     int n_ctiles, n_slices, n_items;
+    int extra_k2;             // > 0: one more value of k2 (= K2MAX) reaches into the band, for a few lanes only; those
+                              // bins are accumulated on the CUDA cores instead of costing a second pass over the input
 };
 
 // barriers
@@ -76,11 +78,13 @@ enum {
 __device__ __forceinline__ bool wait_bar(uint32_t bar, int parity, volatile int* s_fail, int* status) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer();
+    // a probe suspends the thread for a while by itself; the failure flag and the clock are looked at now and then
     for (int it = 0; it < kSpin; ++it) {
-        __nanosleep(40);                       // a waiting warp leaves the issue slots to the working ones
         if (mbar_try_wait(bar, parity)) return true;
-        if (*s_fail) return false;
-        if ((it & 63) == 63 && global_timer() - t0 > 1000000000ull) break;   // one second
+        if ((it & 15) == 15) {
+            if (*s_fail) return false;
+            if (global_timer() - t0 > 1000000000ull) break;   // one second
+        }
     }
     atomicCAS(status, 0, (int)LUVC_ERR_TIMEOUT);
     *s_fail = 1;
@@ -109,7 +113,8 @@ __device__ __forceinline__ uint32_t bf16x2_bits(float lo_half, float hi_half) {
 
 template <int NCOL> __device__ __forceinline__ void tmem_load(uint32_t addr, uint32_t (&v)[NCOL]) {
     if constexpr (NCOL == 2) tmem_ld2(addr, v);
-    else tmem_ld4(addr, v);
+    else if constexpr (NCOL == 4) tmem_ld4(addr, v);
+    else tmem_ld8(addr, v);
 }
 
 // Geometry of a variant.  A tile is 64 columns (QT tokens x C channels); a converter thread owns W
@@ -123,26 +128,28 @@ template <int NCOL> __device__ __forceinline__ void tmem_load(uint32_t addr, uin
 template <int C_, int N2_, int QPU_, int RING_>
 struct Geo {
     static constexpr int C = C_, N2 = N2_, QPU = QPU_, RING = RING_;
-    static constexpr int QT = kTN / C;                        // tokens per tile: 4 or 8
-    static constexpr int W = C / 4;                           // channels per converter thread: 4 or 2
+    static constexpr int QT = kTN / C;                        // tokens per tile: 2, 4 or 8
+    static constexpr int W = C / 4;                           // channels per converter thread: 8, 4 or 2
     static constexpr int CPU_ = 4 / QPU;                      // channels per unit: 2 or 1
     static constexpr int K2MAX = N2 / (2 * CPU_);             // bins of k2 per lane and channel
-    static constexpr int GROUPS = QT / QPU;                   // token groups per tile: 2
-    static constexpr int OUT_COLS = (C / CPU_) * N2;          // columns of the band spectrum in TMEM
+    static constexpr int GQ = QT / QPU;                       // token groups per tile: 1 or 2
+    static constexpr int UC = C / CPU_;                       // result units (column groups of the spectrum): 16 or 8
+    static constexpr int UT = W / CPU_;                       // result units of one converter thread: 4 or 2
+    static constexpr int OUT_COLS = UC * N2;                  // columns of the band spectrum in TMEM
     static constexpr int ACC0 = 0;                            // two stage-1 accumulators
     static constexpr int RING0 = 2 * kTN;
     static constexpr int OUT0 = RING0 + RING * kSlotCols;
     static constexpr int TMEM_COLS = 512;
-    static constexpr int ROWB = 2 * C;                        // bytes of one token row of a tile: 32 or 16
-    static constexpr uint32_t LAYOUT = C == 16 ? 6u : 0u;     // 32-byte swizzle, or none
+    static constexpr int ROWB = 2 * C;                        // bytes of one token row of a tile: 64, 32 or 16
+    static constexpr uint32_t LAYOUT = C == 32 ? 4u : (C == 16 ? 6u : 0u);   // 64-byte or 32-byte swizzle, or none
     static constexpr int STAGE_BYTES = kTN * kP * 2;
     static constexpr int W_BYTES = 16 * N2 * 2;               // one part (hi or lo) of one token group's matrix
     static_assert(OUT0 + OUT_COLS <= TMEM_COLS, "tensor memory budget");
-    static_assert(GROUPS == 2 && (W / CPU_) * GROUPS == 4 && (C / CPU_) * GROUPS == kUnits && kUnits * 8 == kSlotCols,
+    static_assert(W * QT == 16 && GQ * UT == 4 && GQ * UC == kUnits && kUnits * 8 == kSlotCols,
                   "a tile is sixteen units, four per converter thread");
 };
 
-template <typename G>
+template <typename G, bool EXTRA>
 __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_constant__ CUtensorMap tmap, const Fwd3Args a) {
     constexpr int C = G::C, N2 = G::N2, QPU = G::QPU, QT = G::QT, W = G::W;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -153,7 +160,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Q = a.Q, N = a.N, D = a.D, sigma = a.sigma;
     const int tiles_per_item = (Q + QT - 1) / QT;
-    const int n_groups = tiles_per_item * G::GROUPS;                    // token groups of a sequence (padded)
+    const int n_groups = tiles_per_item * G::GQ;                    // token groups of a sequence (padded)
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* s_fhi = smem;                                        // stage-1 matrix, 32 KB per part
     unsigned char* s_flo = smem + 32768;
@@ -315,19 +322,19 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
             ok = wait_bar_warp(bar(kBarGrpFull + g * 2 + slot), use & 1, fail, a.status);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t ring = tmem + (uint32_t)(G::RING0 + slot * kSlotCols + g * 16);
-            const uint32_t out = tmem + (uint32_t)(G::OUT0 + 2 * g * N2);
-            const uint64_t wg = w0 + (uint64_t)((tile * G::GROUPS * 2 * G::W_BYTES) >> 4);
+            const uint32_t ring = tmem + (uint32_t)(G::RING0 + slot * kSlotCols + g * G::UT * 8);
+            const uint32_t out = tmem + (uint32_t)(G::OUT0 + g * G::UT * N2);
+            const uint64_t wg = w0 + (uint64_t)((tile * G::GQ * 2 * G::W_BYTES) >> 4);
             const uint32_t first = tile == 0 ? 0u : 1u;
             if (elect_one()) {
-                // unit (token group gq, unit uu of the group's threads): operand columns (gq * 8 + 2 g + uu) * 8,
-                // result columns (2 g + uu) * N2, matrix of token group tile * 2 + gq
+                // unit (token group gq, result unit cu of this group's threads): operand columns
+                // (gq UC + g UT + cu) * 8, result columns (g UT + cu) * N2, matrix of token group tile * GQ + gq
 #pragma unroll
-                for (int gq = 0; gq < 2; ++gq)
+                for (int gq = 0; gq < G::GQ; ++gq)
 #pragma unroll
-                    for (int uu = 0; uu < 2; ++uu) {
+                    for (int cu = 0; cu < G::UT; ++cu) {
                         const uint64_t whi = wg + (uint64_t)((gq * 2 * G::W_BYTES) >> 4), wlo = whi + (uint64_t)(G::W_BYTES >> 4);
-                        const uint32_t opnd = ring + (uint32_t)(gq * 64 + uu * 8), res = out + (uint32_t)(uu * N2);
+                        const uint32_t opnd = ring + (uint32_t)((gq * G::UC + cu) * 8), res = out + (uint32_t)(cu * N2);
                         umma_bf16_ts(res, opnd, whi, idesc2, gq ? 1u : first);
                         umma_bf16_ts(res, opnd, wlo, idesc2, 1u);
                     }
@@ -363,6 +370,9 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
             // e^{-2 pi i m / N} = e^{-2 pi i (m >> 7) / Q} e^{-2 pi i (m & 127) / N}: two table entries
             const int d_angle = (int)(((unsigned long long)QT * (unsigned)kfe) % (unsigned)N);
             int angle = 0;
+            float2 extra[W];                                         // bin kfe + 128 extra_k2 of this lane's channels
+#pragma unroll
+            for (int c = 0; c < W; ++c) extra[c] = make_float2(0.f, 0.f);
             // The TMEM round trips are long (a load or a store takes several hundred cycles), so the loop is
             // software-pipelined: the next tile's values are requested before this tile's arithmetic, and
             // a tile's stores are only waited for (and its units handed to the MMA warp) one tile later.
@@ -390,13 +400,6 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarAccEmpty + buf));  // the accumulator may be overwritten
-                if (pending_slot >= 0) {                             // the previous tile's units are in place
-                    tmem_st_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(kBarGrpFull + g * 2 + pending_slot));
-                    pending_slot = -1;
-                }
                 if (tile + 1 < tiles_per_item) {                     // request the next tile's values
                     ok = wait_bar(bar(kBarAccFull + ((u + 1) & 1)), ((u + 1) >> 1) & 1, fail, a.status);
                     ok = __all_sync(0xffffffffu, ok);
@@ -410,18 +413,34 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                 uint32_t op[4][8];                                   // four units of four complex values: (hi pair, lo pair) each
 #pragma unroll
                 for (int ql = 0; ql < QT; ++ql) {
+                    if (ql == QT / 2 && pending_slot >= 0) {
+                        // half way through the arithmetic the previous tile's stores have long landed: hand its
+                        // units to the MMA warp now, which then has the other half to finish with them before
+                        // this tile's units go into the same columns
+                        tmem_st_wait();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kBarGrpFull + g * 2 + pending_slot));
+                        pending_slot = -1;
+                    }
                     const float2 rot = cmul(base, within[ql]);
                     // B = rot * (own + i cg other):  Re = rot.x own - cg rot.y other,  Im = rot.y own + cg rot.x other
                     const float ox = -cg * rot.y, oy = cg * rot.x;
+                    float2 wex = make_float2(0.f, 0.f);              // e^{-2 pi i q extra_k2 / Q} of this token
+                    if constexpr (EXTRA) wex = s_root[(int)(((long long)(tile * QT + ql) * a.extra_k2) % Q)];
 #pragma unroll
                     for (int c = 0; c < W; ++c) {
                         const float own = __uint_as_float(v[ql][c]);
                         const float other = __shfl_xor_sync(0xffffffffu, own, 1);
                         const float wx = fmaf(rot.x, own, ox * other), wy = fmaf(rot.y, own, oy * other);
+                        if constexpr (EXTRA) {
+                            extra[c].x = fmaf(wx, wex.x, fmaf(-wy, wex.y, extra[c].x));
+                            extra[c].y = fmaf(wx, wex.y, fmaf(wy, wex.x, extra[c].y));
+                        }
                         const uint32_t hi = bf16x2_bits(wx, wy);
                         const uint32_t lo = bf16x2_bits(wx - __uint_as_float(hi << 16), wy - __uint_as_float(hi & 0xffff0000u));
                         // unit and position of this value: two channels x two tokens, or one channel x four tokens
-                        const int unit = QPU == 2 ? ((ql >> 1) * 2 + (c >> 1)) : ((ql >> 2) * 2 + c);
+                        const int unit = QPU == 2 ? ((ql >> 1) * G::UT + (c >> 1)) : ((ql >> 2) * G::UT + c);
                         const int z = QPU == 2 ? ((ql & 1) * 2 + (c & 1)) : (ql & 3);
                         op[unit][2 * z] = hi;
                         op[unit][2 * z + 1] = lo;
@@ -435,12 +454,12 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                     if (!ok) break;
                     tc_fence_after();
                 }
-                // unit (token group gq, this thread's unit uu) sits at columns (gq * 8 + 2 g + uu) * 8 of the slot
-                const uint32_t ring = lane_addr + (uint32_t)(G::RING0 + slot * kSlotCols + g * 16);
-                tmem_st8(ring, op[0]);
-                tmem_st8(ring + 8, op[1]);
-                tmem_st8(ring + 64, op[2]);
-                tmem_st8(ring + 72, op[3]);
+                // unit (token group gq, this thread's result unit cu) sits at columns (gq UC + g UT + cu) * 8 of the slot
+                const uint32_t ring = lane_addr + (uint32_t)(G::RING0 + slot * kSlotCols + g * G::UT * 8);
+#pragma unroll
+                for (int gq = 0; gq < G::GQ; ++gq)
+#pragma unroll
+                    for (int cu = 0; cu < G::UT; ++cu) tmem_st8(ring + (uint32_t)((gq * G::UC + cu) * 8), op[gq * G::UT + cu]);
                 pending_slot = slot;
             }
             if (!ok) break;
@@ -461,11 +480,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                 const int ch0 = ctile * C + g * W;                   // first of this thread's channels
                 float* Yb = a.Y + (size_t)b * a.R * D + ch0;
                 const bool live = ch0 < D;                           // D is a multiple of 8 and ch0 of W: whole or absent
-                // this thread's two result units: columns [2g N2, 2g N2 + 2 N2) of the spectrum
+                // this thread's result units: columns [g UT N2, (g + 1) UT N2) of the spectrum, sixteen at a time
 #pragma unroll
-                for (int h = 0; h < (2 * N2) / 16; ++h) {
+                for (int h = 0; h < (G::UT * N2) / 16; ++h) {
                     uint32_t o[16];
-                    tmem_ld16(lane_addr + (uint32_t)(G::OUT0 + 2 * g * N2 + h * 16), o);
+                    tmem_ld16(lane_addr + (uint32_t)(G::OUT0 + g * G::UT * N2 + h * 16), o);
                     tmem_ld_wait_for(o);
                     if constexpr (QPU == 2) {
                         // unit h: channels 2h, 2h+1 of the thread; column = cc * 8 + k2 * 2 + ri
@@ -490,6 +509,17 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                             const float cr = __ldg(a.scale + k), ci = k >= 1 ? __ldg(a.scale + sigma + k) : 0.f;
                             Yb[(size_t)k * D + cc] = cr * __uint_as_float(o[k2 * 2]);
                             if (k >= 1) Yb[(size_t)(sigma + k) * D + cc] = ci * __uint_as_float(o[k2 * 2 + 1]);
+                        }
+                    }
+                }
+                if (EXTRA && live) {
+                    const int k = kfe + kP * a.extra_k2;
+                    if (k <= sigma) {
+                        const float cr = __ldg(a.scale + k), ci = __ldg(a.scale + sigma + k);
+#pragma unroll
+                        for (int c = 0; c < W; ++c) {
+                            Yb[(size_t)k * D + c] = cr * extra[c].x;
+                            Yb[(size_t)(sigma + k) * D + c] = ci * extra[c].y;
                         }
                     }
                 }
@@ -523,11 +553,11 @@ EncodeTiledFn encode_tiled_fn() {
 
 template <typename G>
 size_t fwd3_smem(int Q) {
-    const int tiles = (Q + G::QT - 1) / G::QT, groups = tiles * G::GROUPS;
+    const int tiles = (Q + G::QT - 1) / G::QT, groups = tiles * G::GQ;
     return 1024 + 65536 + (size_t)kStages * G::STAGE_BYTES + (size_t)groups * 2 * G::W_BYTES + (size_t)(Q + kP) * sizeof(float2);
 }
 
-template <typename G>
+template <typename G, bool EXTRA>
 cudaError_t launch_fwd3(const Fwd3Args& a, cudaStream_t stream) {
     // the tokens of one sequence as [q][p][channel]: token p Q + q sits 128-strided in memory
     EncodeTiledFn encode = encode_tiled_fn();
@@ -537,7 +567,8 @@ cudaError_t launch_fwd3(const Fwd3Args& a, cudaStream_t stream) {
     const cuuint64_t strides[3] = {(cuuint64_t)a.Q * a.D * 2, (cuuint64_t)a.D * 2, (cuuint64_t)a.N * a.D * 2};
     const cuuint32_t box[4] = {(cuuint32_t)G::C, (cuuint32_t)kP, (cuuint32_t)G::QT, 1u};
     const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-    const CUtensorMapSwizzle swz = G::C == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
+    const CUtensorMapSwizzle swz = G::C == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                 : G::C == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
     if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(a.x), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -549,13 +580,13 @@ cudaError_t launch_fwd3(const Fwd3Args& a, cudaStream_t stream) {
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    cudaFuncSetAttribute(spu_fwd3_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncSetAttribute(spu_fwd3_kernel<G, EXTRA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int grid = a.n_items < sms ? a.n_items : sms;
-    spu_fwd3_kernel<G><<<grid, kThreads, smem, stream>>>(tmap, a);
+    spu_fwd3_kernel<G, EXTRA><<<grid, kThreads, smem, stream>>>(tmap, a);
     return cudaGetLastError();
 }
 
-using GeoNarrow = Geo<16, 16, 2, 2>;     // up to 4 bins per frequency class, two operand slots
+using GeoNarrow = Geo<32, 16, 2, 1>;     // up to 4 bins per frequency class; 64-byte token rows keep TMA at full rate
 using GeoWide = Geo<8, 32, 4, 1>;        // up to 16 bins per frequency class (per slice), one operand slot
 
 }  // namespace
@@ -569,6 +600,11 @@ SpuFwd3Plan spu_fwd3_plan(int B, int N, int D, int sigma) {
     pl.wide = nk2 > GeoNarrow::K2MAX ? 1 : 0;
     const int k2max = pl.wide ? GeoWide::K2MAX : GeoNarrow::K2MAX;
     pl.slices = (nk2 + k2max - 1) / k2max;
+    pl.extra_k2 = 0;
+    if (pl.wide && nk2 == k2max + 1) {               // one value of k2 too many for one pass: the few lanes that reach
+        pl.slices = 1;                               // it (k1 <= sigma - 128 k2max) keep that bin in registers
+        pl.extra_k2 = k2max;
+    }
     pl.C = pl.wide ? GeoWide::C : GeoNarrow::C;
     pl.n_ctiles = (D + pl.C - 1) / pl.C;
     const long long items = (long long)B * pl.n_ctiles * pl.slices;
@@ -589,7 +625,9 @@ int spu_fwd3_run(const void* hidden, float* Y, const float* scale, int B, int N,
     a.Y = Y; a.scale = scale; a.status = status;
     a.B = B; a.N = N; a.D = D; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
-    const cudaError_t err = pl.wide ? launch_fwd3<GeoWide>(a, stream) : launch_fwd3<GeoNarrow>(a, stream);
+    a.extra_k2 = pl.extra_k2;
+    const cudaError_t err = !pl.wide ? launch_fwd3<GeoNarrow, false>(a, stream)
+                            : pl.extra_k2 ? launch_fwd3<GeoWide, true>(a, stream) : launch_fwd3<GeoWide, false>(a, stream);
     count_launch();
     return err == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
