@@ -111,6 +111,9 @@ int spu_tc_run(const SpuTcBuffers& w, const void* hidden, const float2* tw, cons
                int B, int N, int D, int sigma, int* status, cudaStream_t stream, bool have_yt,
                const int32_t* row_index = nullptr, int src_rows = 0);
 
+// Scratch for the operand images (stage-1 matrices, stage-2 tables) of one transform kernel.
+constexpr size_t kSpuImgBytes = 160 * 1024;
+
 // Two-stage forward transform of the bf16 path (spu_fwd2.cu): N = P * Q, P a multiple of 16.
 struct SpuFwd2Plan {
     int ok;             // 0: N has no usable factor, use the dense contraction
@@ -122,8 +125,9 @@ struct SpuFwd2Plan {
 };
 SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma);
 // Y[b][r][d] = c[r] * (band spectrum); also its transposed bf16 pair [b][d][r_pad] when yt_hi is given.
+// `img`: kSpuImgBytes of 16-byte aligned device scratch for the operand images a call builds once for all its CTAs.
 int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, void* yt_lo, int r_pad, int B, int N,
-                 int D, int sigma, int* status, cudaStream_t stream);
+                 int D, int sigma, int* status, cudaStream_t stream, void* img);
 
 // Forward transform with both stages on the tensor cores (spu_fwd3.cu): N = 128 Q, 8 <= Q <= 128.
 struct SpuFwd3Plan {
@@ -137,7 +141,7 @@ struct SpuFwd3Plan {
 SpuFwd3Plan spu_fwd3_plan(int B, int N, int D, int sigma);
 // Y[b][r][d] = c[r] * (band spectrum), the layout spu_fwd2_run writes.
 int spu_fwd3_run(const void* hidden, float* Y, const float* scale, int B, int N, int D, int sigma, int* status,
-                 cudaStream_t stream);
+                 cudaStream_t stream, void* img);
 
 // Two-stage inverse transform and energies of the bf16 path (spu_inv2.cu); needs the forward plan.
 struct SpuInv2Plan {
@@ -149,6 +153,6 @@ struct SpuInv2Plan {
     int n_parts;        // partial sums per point and sequence: part[b][n_parts][L]
 };
 SpuInv2Plan spu_inv2_plan(int B, int N, int D, int sigma);
-int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream);
+int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream, void* img);
 
 }  // namespace luvc

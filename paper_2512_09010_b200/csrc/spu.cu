@@ -388,6 +388,7 @@ struct Workspace {
     // bf16 path (tensor cores)
     SpuTcBuffers tc;
     float* Y2;       // band spectrum of the two-stage forward transform [B][2 sigma + 1][D]
+    void *img_fwd, *img_inv;   // operand images of the forward / inverse transform kernel, built once per call
 };
 
 // How the bf16 path runs a problem, and the points its inverse is evaluated on.
@@ -434,7 +435,11 @@ Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path, bool
             w.S = reinterpret_cast<float*>(take((size_t)B * m.L * 4));
             w.gpart = reinterpret_cast<float2*>(take(coarse_gpart_elems(B, m.L, sigma) * sizeof(float2)));
         }
-        if (m.fwd2) w.Y2 = reinterpret_cast<float*>(take((size_t)B * R * D * sizeof(float)));
+        if (m.fwd2) {
+            w.Y2 = reinterpret_cast<float*>(take((size_t)B * R * D * sizeof(float)));
+            w.img_fwd = take(kSpuImgBytes);
+            w.img_inv = take(kSpuImgBytes);
+        }
         w.tc.part = reinterpret_cast<float*>(take((size_t)B * m.n_parts * m.L * 4));
         if (!m.inv2) {      // the dense inverse (and, without the two-stage forward, the dense forward)
             if (!m.fwd2 || !pl.coarse) {
@@ -483,14 +488,14 @@ static int spu_run_typed(const SpuProblem& p) {
     count_launch();
     if constexpr (kTensor) {
         if (mode.fwd2 && mode.inv2 && spu_fwd3_plan(B, N, D, sigma).ok) {
-            const int rc1 = spu_fwd3_run(p.hidden, ws.Y2, ws.scale, B, N, D, sigma, p.status, p.stream);
+            const int rc1 = spu_fwd3_run(p.hidden, ws.Y2, ws.scale, B, N, D, sigma, p.status, p.stream, ws.img_fwd);
             if (rc1 != LUVC_OK) return rc1;
         } else if (mode.fwd2) {
             const int rc1 = spu_fwd2_run(p.hidden, ws.Y2, ws.scale, mode.inv2 ? nullptr : ws.tc.yt_hi,
-                                         mode.inv2 ? nullptr : ws.tc.yt_lo, pl.r_pad, B, N, D, sigma, p.status, p.stream);
+                                         mode.inv2 ? nullptr : ws.tc.yt_lo, pl.r_pad, B, N, D, sigma, p.status, p.stream, ws.img_fwd);
             if (rc1 != LUVC_OK) return rc1;
         }
-        const int rc = mode.inv2 ? spu_inv2_run(ws.Y2, ws.tc.part, B, N, D, sigma, p.status, p.stream)
+        const int rc = mode.inv2 ? spu_inv2_run(ws.Y2, ws.tc.part, B, N, D, sigma, p.status, p.stream, ws.img_inv)
                                  : spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status,
                                               p.stream, mode.fwd2, p.row_index, p.src_rows);
         if (rc != LUVC_OK) return rc;

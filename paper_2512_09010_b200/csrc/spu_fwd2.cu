@@ -54,10 +54,11 @@ struct FwdArgs {
                               // serves its own block of channels of the same tokens (P <= 64)
     int n_ctiles, n_slices, n_items;
     int static_tab;           // 1: the table of e^{-2 pi i q k2 / Q} for all q is built once per CTA (one slice only)
+    const unsigned char* f_img;   // both parts of the stage-1 matrix as they sit in shared memory (built once per call)
 };
 
 // barriers: 0,1 stage full | 2,3 accumulator full | 4,5 accumulator empty | 6,7 table ready
-enum { kBarFull = 0, kBarAccFull = 2, kBarAccEmpty = 4, kBarTab = 6, kBars = 8 };
+enum { kBarFull = 0, kBarAccFull = 2, kBarAccEmpty = 4, kBarTab = 6, kBarImg = 8, kBars = 9 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, int parity, volatile int* s_fail, int* status) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -209,32 +210,16 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
             mbar_init(bar(kBarAccEmpty + s), kEpiWarps);
             mbar_init(bar(kBarTab + s), kEpiWarps);
         }
+        mbar_init(bar(kBarImg), 1);
         s_fail = 0;
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
 
-    // stage-1 matrix, K-major: element (row j, column kk) at (j/8)*128 + (kk/8)*2048 + (j%8)*16 + (kk%8)*2;
-    // block-diagonal: row j = jb P + jr meets column kk = kb P + p only for jb == kb
-    for (int idx = tid; idx < 128 * KT; idx += kThreads) {
-        const int j = idx / KT, kk = idx - j * KT;
-        const int jb = j / P, jr = j - jb * P, kb = kk / P, p = kk - kb * P;
-        float v = 0.f;
-        if (j < KT && jb == kb) {
-            if (jr == 0) v = 1.f;
-            else if (jr == 1) v = (p & 1) ? -1.f : 1.f;
-            else {
-                const int m = ((jr >> 1) * p) % P;
-                float s, c;
-                sincospif(2.0f * (float)m / (float)P, &s, &c);
-                v = (jr & 1) ? -s : c;
-            }
-        }
-        const __nv_bfloat16 h = __float2bfloat16_rn(v);
-        const __nv_bfloat16 l = __float2bfloat16_rn(v - __bfloat162float(h));
-        const int off = (j >> 3) * 128 + (kk >> 3) * 2048 + (j & 7) * 16 + (kk & 7) * 2;
-        *reinterpret_cast<__nv_bfloat16*>(s_fhi + off) = h;
-        *reinterpret_cast<__nv_bfloat16*>(s_flo + off) = l;
+    // the stage-1 matrix (both parts) was built once per call in global memory, in its shared-memory layout
+    if (tid == 0) {
+        mbar_arrive_expect_tx(bar(kBarImg), (uint32_t)(2 * f_bytes));
+        bulk_load(smem_u32(s_fhi), a.f_img, (uint32_t)(2 * f_bytes), bar(kBarImg));
     }
     if (a.static_tab)
         for (int e = tid; e < Q * KB; e += kThreads) {
@@ -247,6 +232,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     volatile int* fail = &s_fail;
+    if (!__all_sync(0xffffffffu, wait_bar(bar(kBarImg), 0, fail, a.status))) {     // the matrix has landed
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+        return;
+    }
     const int tiles_per_item = (Q + QT - 1) / QT;
     const int item_channels = a.nblk * C;
 
@@ -397,6 +387,32 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+// Both parts of the stage-1 matrix in the layout the kernel's shared memory uses (K-major: element (row j,
+// column kk) at (j/8)*128 + (kk/8)*2048 + (j%8)*16 + (kk%8)*2; hi part first, lo part KT*256 bytes later),
+// block-diagonal: row j = jb P + jr meets column kk = kb P + p only for jb == kb.  Rows of a block: A[0],
+// A[P/2], then Re / Im of A[1 .. P/2-1].  Built once per call instead of once per CTA.
+__global__ void __launch_bounds__(256) spu_fwd2_img_kernel(unsigned char* __restrict__ img, int P, int KT) {
+    const int idx = blockIdx.x * 256 + threadIdx.x;
+    if (idx >= 128 * KT) return;
+    const int j = idx / KT, kk = idx - j * KT;
+    const int jb = j / P, jr = j - jb * P, kb = kk / P, p = kk - kb * P;
+    float v = 0.f;
+    if (j < KT && jb == kb) {
+        if (jr == 0) v = 1.f;
+        else if (jr == 1) v = (p & 1) ? -1.f : 1.f;
+        else {
+            const int m = ((jr >> 1) * p) % P;
+            float s, c;
+            sincospif(2.0f * (float)m / (float)P, &s, &c);
+            v = (jr & 1) ? -s : c;
+        }
+    }
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    const int off = (j >> 3) * 128 + (kk >> 3) * 2048 + (j & 7) * 16 + (kk & 7) * 2;
+    *reinterpret_cast<__nv_bfloat16*>(img + off) = h;
+    *reinterpret_cast<__nv_bfloat16*>(img + KT * 256 + off) = __float2bfloat16_rn(v - __bfloat162float(h));
+}
+
 // YT[b][d][r] (bf16 pair, r padded with zeros to r_pad) from Y[b][r][d]
 __global__ void __launch_bounds__(256) spu_y_transpose_kernel(const float* __restrict__ Y, __nv_bfloat16* __restrict__ hi,
                                                               __nv_bfloat16* __restrict__ lo, int R, int r_pad, int D) {
@@ -498,15 +514,21 @@ SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma) {
 }
 
 int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, void* yt_lo, int r_pad, int B, int N,
-                 int D, int sigma, int* status, cudaStream_t stream) {
+                 int D, int sigma, int* status, cudaStream_t stream, void* img) {
     const SpuFwd2Plan pl = spu_fwd2_plan(B, N, D, sigma);
     if (!pl.ok) return LUVC_ERR_INTERNAL;
+    {
+        const int KT = pl.nblk * pl.P;
+        spu_fwd2_img_kernel<<<(128 * KT + 255) / 256, 256, 0, stream>>>(static_cast<unsigned char*>(img), pl.P, KT);
+        count_launch();
+    }
     FwdArgs a;
     a.x = reinterpret_cast<const __nv_bfloat16*>(hidden);
     a.Y = Y; a.scale = scale; a.status = status;
     a.B = B; a.N = N; a.D = D; a.P = pl.P; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
     a.nblk = pl.nblk;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
+    a.f_img = static_cast<const unsigned char*>(img);
     a.static_tab = (pl.slices == 1 && (size_t)pl.Q * pl.KB * sizeof(float4) <= (size_t)kStaticTabBytes) ? 1 : 0;
     cudaError_t err;
     if (pl.KB == 2) err = launch_fwd2<2, 8>(a, pl, stream);

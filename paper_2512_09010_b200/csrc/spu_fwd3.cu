@@ -59,6 +59,7 @@ struct Fwd3Args {
     int* status;
     int B, N, D, Q, sigma, R;
     int n_ctiles, n_slices, n_items;
+    const unsigned char* img; // stage-1 matrix, stage-2 matrices and root tables in their shared-memory layouts (built once per call)
     int extra_k2;             // > 0: one more value of k2 (= K2MAX) reaches into the band, for a few lanes only; those
                               // bins are accumulated on the CUDA cores instead of costing a second pass over the input
 };
@@ -72,7 +73,8 @@ enum {
     kBarGrpEmpty = kBarGrpFull + 8,     // [4 groups][2] the MMAs that read those units are done
     kBarOutFull = kBarGrpEmpty + 8,     // the band spectrum of the work item is complete (four issuers)
     kBarOutEmpty = kBarOutFull + 1,     // every converter warp has read it
-    kBars = kBarOutEmpty + 1
+    kBarImg = kBarOutEmpty + 1,         // the operand images have landed
+    kBars = kBarImg + 1
 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, int parity, volatile int* s_fail, int* status) {
@@ -167,7 +169,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
     unsigned char* s_x = smem + 65536;                                  // input stages
     unsigned char* s_w = s_x + kStages * G::STAGE_BYTES;                // [n_groups][hi, lo][16 x N2] stage-2 matrices
     float2* s_root = reinterpret_cast<float2*>(s_w + (size_t)n_groups * 2 * G::W_BYTES);   // e^{-2 pi i m / Q}, m < Q
-    float2* s_fine = s_root + Q;                                                           // e^{-2 pi i m / N}, m < 128
+    float2* s_fine = s_root + ((Q + 1) & ~1);                                              // e^{-2 pi i m / N}, m < 128
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -183,57 +185,19 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
         }
         mbar_init(bar(kBarOutFull), 4);
         mbar_init(bar(kBarOutEmpty), kConvWarps);
+        mbar_init(bar(kBarImg), 1);
         s_fail = 0;
         mbar_fence_init();
     }
     if (warp == kConvWarps) tmem_alloc(smem_u32(&s_tmem), G::TMEM_COLS);
 
-    // stage-1 matrix, K-major: element (row j, column p) at (j/8)*128 + (p/8)*2048 + (j%8)*16 + (p%8)*2.
-    // Rows 0 / 1: A[0] and A[64] (real); rows 2i / 2i+1: Re and Im of A[i].
-    for (int idx = tid; idx < kP * kP; idx += kThreads) {
-        const int j = idx >> 7, p = idx & 127;
-        float v;
-        if (j == 0) v = 1.f;
-        else if (j == 1) v = (p & 1) ? -1.f : 1.f;
-        else {
-            const int m = ((j >> 1) * p) & 127;
-            float s, c;
-            sincospif((float)m * (1.0f / 64.0f), &s, &c);
-            v = (j & 1) ? -s : c;
-        }
-        const __nv_bfloat16 h = __float2bfloat16_rn(v);
-        const int off = (j >> 3) * 128 + (p >> 3) * 2048 + (j & 7) * 16 + (p & 7) * 2;
-        *reinterpret_cast<__nv_bfloat16*>(s_fhi + off) = h;
-        *reinterpret_cast<__nv_bfloat16*>(s_flo + off) = __float2bfloat16_rn(v - __bfloat162float(h));
-    }
-    for (int m = tid; m < Q; m += kThreads) s_root[m] = root_neg((unsigned)m, (unsigned)Q);
-    for (int m = tid; m < kP; m += kThreads) s_fine[m] = root_neg((unsigned)m, (unsigned)N);
-    __syncthreads();
-    // Stage-2 matrices, K-major [n][k]: element at (n/8)*128 + (k/8)*(N2*16) + (n%8)*16 + (k%8)*2.
-    //   k = z*4 + t: complex value z of the unit, t = Re hi, Im hi, Re lo, Im lo (the lo rows of the
-    //   hi-part matrix repeat the hi rows; the lo-part matrix has zeros there)
-    //   n = (channel of the unit, k2, re/im); block-diagonal over the channels of a unit
-    for (int idx = tid; idx < n_groups * 16 * N2; idx += kThreads) {
-        const int grp = idx / (16 * N2), rem = idx - grp * 16 * N2;
-        const int n = rem >> 4, k = rem & 15;
-        const int z = k >> 2, t = k & 3;
-        int qq, zc;
-        if constexpr (QPU == 2) { qq = z >> 1; zc = z & 1; } else { qq = z; zc = 0; }
-        const int per_ch = N2 / G::CPU_;
-        const int nc = n / per_ch, nr = n - nc * per_ch, k2 = nr >> 1, ri = nr & 1;
-        const int q = grp * QPU + qq;
-        float v = 0.f;
-        if (nc == zc && q < Q) {
-            const float2 w = s_root[(int)(((long long)q * k2) % Q)];    // e^{-2 pi i q k2 / Q}
-            // (Re, Im) of B times w: Re out = Re B w.x - Im B w.y, Im out = Re B w.y + Im B w.x
-            v = (t & 1) == 0 ? (ri == 0 ? w.x : w.y) : (ri == 0 ? -w.y : w.x);
-        }
-        const __nv_bfloat16 h = __float2bfloat16_rn(v);
-        const __nv_bfloat16 l = __float2bfloat16_rn(v - __bfloat162float(h));
-        const int off = (n >> 3) * 128 + (k >> 3) * (N2 * 16) + (n & 7) * 16 + (k & 7) * 2;
-        unsigned char* base = s_w + (size_t)grp * 2 * G::W_BYTES;
-        *reinterpret_cast<__nv_bfloat16*>(base + off) = h;
-        *reinterpret_cast<__nv_bfloat16*>(base + G::W_BYTES + off) = t < 2 ? l : __float2bfloat16_rn(0.f);
+    // The stage-1 matrix, the stage-2 matrices and the two root tables were built once per call in global
+    // memory, in the layouts used here: two bulk copies fetch them.
+    const int tab_bytes = n_groups * 2 * G::W_BYTES + (((Q + 1) & ~1) + kP) * (int)sizeof(float2);
+    if (tid == 0) {
+        mbar_arrive_expect_tx(bar(kBarImg), (uint32_t)(65536 + tab_bytes));
+        bulk_load(smem_u32(s_fhi), a.img, 65536u, bar(kBarImg));
+        bulk_load(smem_u32(s_w), a.img + 65536, (uint32_t)tab_bytes, bar(kBarImg));
     }
     fence_proxy_async();
     tc_fence_before();
@@ -241,6 +205,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     volatile int* fail = &s_fail;
+    if (!__all_sync(0xffffffffu, wait_bar(bar(kBarImg), 0, fail, a.status))) {
+        __syncthreads();
+        if (warp == kConvWarps) tmem_dealloc(tmem, G::TMEM_COLS);
+        return;
+    }
 
     int n_my_items = 0;
     for (int item = blockIdx.x; item < a.n_items; item += gridDim.x) ++n_my_items;
@@ -535,6 +504,63 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
     if (warp == kConvWarps) tmem_dealloc(tmem, G::TMEM_COLS);
 }
 
+// The operand images of one call, as the kernel's shared memory holds them:
+//   [0, 64 KB)   stage-1 matrix, hi part then lo part, K-major: element (row j, column p) at
+//                (j/8)*128 + (p/8)*2048 + (j%8)*16 + (p%8)*2; rows 0 / 1: A[0] and A[64] (real), rows 2i / 2i+1: Re and Im of A[i]
+//   then         the stage-2 matrices [n_groups][hi, lo][16 x N2], K-major [n][k]: element at
+//                (n/8)*128 + (k/8)*(N2*16) + (n%8)*16 + (k%8)*2;  k = z*4 + t: complex value z of the unit, t = Re hi,
+//                Im hi, Re lo, Im lo (the lo rows of the hi-part matrix repeat the hi rows; the lo-part matrix has zeros
+//                there);  n = (channel of the unit, k2, re/im), block-diagonal over the channels of a unit
+//   then         e^{-2 pi i m / Q}, m < Q (padded to an even count), and e^{-2 pi i m / N}, m < 128
+template <typename G>
+__global__ void __launch_bounds__(256) spu_fwd3_img_kernel(unsigned char* __restrict__ img, int Q, int N, int n_groups) {
+    constexpr int N2 = G::N2, QPU = G::QPU;
+    const int idx = blockIdx.x * 256 + threadIdx.x;
+    if (idx < kP * kP) {
+        const int j = idx >> 7, p = idx & 127;
+        float v;
+        if (j == 0) v = 1.f;
+        else if (j == 1) v = (p & 1) ? -1.f : 1.f;
+        else {
+            const int m = ((j >> 1) * p) & 127;
+            float s, c;
+            sincospif((float)m * (1.0f / 64.0f), &s, &c);
+            v = (j & 1) ? -s : c;
+        }
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        const int off = (j >> 3) * 128 + (p >> 3) * 2048 + (j & 7) * 16 + (p & 7) * 2;
+        *reinterpret_cast<__nv_bfloat16*>(img + off) = h;
+        *reinterpret_cast<__nv_bfloat16*>(img + 32768 + off) = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+    unsigned char* tabs = img + 65536;
+    if (idx < n_groups * 16 * N2) {
+        const int grp = idx / (16 * N2), rem = idx - grp * 16 * N2;
+        const int n = rem >> 4, k = rem & 15;
+        const int z = k >> 2, t = k & 3;
+        int qq, zc;
+        if constexpr (QPU == 2) { qq = z >> 1; zc = z & 1; } else { qq = z; zc = 0; }
+        const int per_ch = N2 / G::CPU_;
+        const int nc = n / per_ch, nr = n - nc * per_ch, k2 = nr >> 1, ri = nr & 1;
+        const int q = grp * QPU + qq;
+        float v = 0.f;
+        if (nc == zc && q < Q) {
+            const float2 w = root_neg((unsigned)(((long long)q * k2) % Q), (unsigned)Q);    // e^{-2 pi i q k2 / Q}
+            // (Re, Im) of B times w: Re out = Re B w.x - Im B w.y, Im out = Re B w.y + Im B w.x
+            v = (t & 1) == 0 ? (ri == 0 ? w.x : w.y) : (ri == 0 ? -w.y : w.x);
+        }
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        const __nv_bfloat16 l = __float2bfloat16_rn(v - __bfloat162float(h));
+        const int off = (n >> 3) * 128 + (k >> 3) * (N2 * 16) + (n & 7) * 16 + (k & 7) * 2;
+        unsigned char* base = tabs + (size_t)grp * 2 * G::W_BYTES;
+        *reinterpret_cast<__nv_bfloat16*>(base + off) = h;
+        *reinterpret_cast<__nv_bfloat16*>(base + G::W_BYTES + off) = t < 2 ? l : __float2bfloat16_rn(0.f);
+    }
+    float2* roots = reinterpret_cast<float2*>(tabs + (size_t)n_groups * 2 * G::W_BYTES);
+    const int q_even = (Q + 1) & ~1;
+    if (idx < q_even) roots[idx] = idx < Q ? root_neg((unsigned)idx, (unsigned)Q) : make_float2(0.f, 0.f);
+    if (idx < kP) roots[q_even + idx] = root_neg((unsigned)idx, (unsigned)N);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -554,7 +580,7 @@ EncodeTiledFn encode_tiled_fn() {
 template <typename G>
 size_t fwd3_smem(int Q) {
     const int tiles = (Q + G::QT - 1) / G::QT, groups = tiles * G::GQ;
-    return 1024 + 65536 + (size_t)kStages * G::STAGE_BYTES + (size_t)groups * 2 * G::W_BYTES + (size_t)(Q + kP) * sizeof(float2);
+    return 1024 + 65536 + (size_t)kStages * G::STAGE_BYTES + (size_t)groups * 2 * G::W_BYTES + (size_t)(((Q + 1) & ~1) + kP) * sizeof(float2);
 }
 
 template <typename G, bool EXTRA>
@@ -573,6 +599,11 @@ cudaError_t launch_fwd3(const Fwd3Args& a, cudaStream_t stream) {
                CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
+    {
+        const int tiles = (a.Q + G::QT - 1) / G::QT, groups = tiles * G::GQ;
+        const int n = kP * kP > groups * 16 * G::N2 ? kP * kP : groups * 16 * G::N2;
+        spu_fwd3_img_kernel<G><<<(n + 255) / 256, 256, 0, stream>>>(const_cast<unsigned char*>(a.img), a.Q, a.N, groups);
+    }
     const size_t smem = fwd3_smem<G>(a.Q);
     static int sms = 0;
     if (!sms) {
@@ -617,7 +648,7 @@ SpuFwd3Plan spu_fwd3_plan(int B, int N, int D, int sigma) {
 }
 
 int spu_fwd3_run(const void* hidden, float* Y, const float* scale, int B, int N, int D, int sigma, int* status,
-                 cudaStream_t stream) {
+                 cudaStream_t stream, void* img) {
     const SpuFwd3Plan pl = spu_fwd3_plan(B, N, D, sigma);
     if (!pl.ok) return LUVC_ERR_INTERNAL;
     Fwd3Args a;
@@ -626,9 +657,10 @@ int spu_fwd3_run(const void* hidden, float* Y, const float* scale, int B, int N,
     a.B = B; a.N = N; a.D = D; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
     a.extra_k2 = pl.extra_k2;
+    a.img = static_cast<const unsigned char*>(img);
     const cudaError_t err = !pl.wide ? launch_fwd3<GeoNarrow, false>(a, stream)
                             : pl.extra_k2 ? launch_fwd3<GeoWide, true>(a, stream) : launch_fwd3<GeoWide, false>(a, stream);
-    count_launch();
+    count_launch(2);
     return err == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
 

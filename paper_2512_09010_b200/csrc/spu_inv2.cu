@@ -42,9 +42,11 @@ struct InvArgs {
     int* status;
     int B, N, D, P, Q, sigma, R, nblk, J, L;
     int n_ctiles, n_items;
+    const unsigned char* img;   // stage-1 matrix (both parts) and the table of e^{2 pi i k2 jj / J}, in their
+                                // shared-memory layouts, built once per call
 };
 
-enum { kBarReady = 0, kBarAccFull = 2, kBars = 4 };
+enum { kBarReady = 0, kBarAccFull = 2, kBarImg = 4, kBars = 5 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, int parity, volatile int* s_fail, int* status) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -186,35 +188,19 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
             mbar_init(bar(kBarReady + s), kWarps);
             mbar_init(bar(kBarAccFull + s), 1);
         }
+        mbar_init(bar(kBarImg), 1);
         s_fail = 0;
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(smem_u32(&s_tmem), kTmemCols);
 
-    // A[m][kk] = F[kk mod P][m mod P] where row m = jb P + p and column kk = kb P + r share the block
-    // (jb == kb), K-major: element at (m/8)*128 + (kk/8)*2048 + (m%8)*16 + (kk%8)*2
-    for (int idx = tid; idx < 128 * KT; idx += kThreads) {
-        const int m = idx / KT, kk = idx - m * KT;
-        const int jb = m / P, p = m - jb * P, kb = kk / P, r = kk - kb * P;
-        float v = 0.f;
-        if (m < KT && jb == kb) {
-            if (r == 0) v = 1.f;
-            else if (r == 1) v = (p & 1) ? -1.f : 1.f;
-            else {
-                float s, c;
-                sincospif(2.0f * (float)(((r >> 1) * p) % P) / (float)P, &s, &c);
-                v = (r & 1) ? -s : c;
-            }
-        }
-        const __nv_bfloat16 h = __float2bfloat16_rn(v);
-        const int off = (m >> 3) * 128 + (kk >> 3) * 2048 + (m & 7) * 16 + (kk & 7) * 2;
-        *reinterpret_cast<__nv_bfloat16*>(s_fhi + off) = h;
-        *reinterpret_cast<__nv_bfloat16*>(s_flo + off) = __float2bfloat16_rn(v - __bfloat162float(h));
-    }
-    for (int e = tid; e < J * KB; e += kThreads) {
-        const int jj = e / KB, k2 = e - jj * KB;
-        const float2 w = root_pos(((unsigned)jj * (unsigned)k2) % (unsigned)J, J);
-        s_w[e] = make_float4(w.x, w.x, w.y, w.y);
+    // the operand matrix (both parts) and the table of e^{2 pi i k2 jj / J} were built once per call in global
+    // memory in the layouts used here: two bulk copies fetch them (the table sits behind the two B buffers)
+    const int w_bytes = J * KB * (int)sizeof(float4);
+    if (tid == 0) {
+        mbar_arrive_expect_tx(bar(kBarImg), (uint32_t)(2 * f_bytes + w_bytes));
+        bulk_load(smem_u32(s_fhi), a.img, (uint32_t)(2 * f_bytes), bar(kBarImg));
+        bulk_load(smem_u32(s_w), a.img + 2 * f_bytes, (uint32_t)w_bytes, bar(kBarImg));
     }
     fence_proxy_async();
     tc_fence_before();
@@ -222,6 +208,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     volatile int* fail = &s_fail;
+    if (!__all_sync(0xffffffffu, wait_bar(bar(kBarImg), 0, fail, a.status))) {     // matrix and table have landed
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+        return;
+    }
 
     const int quarter = warp & 3, grp = warp >> 2;
     const int j = quarter * 32 + lane;               // row (channel block jb, r) of G; row (jb, point p) of the result
@@ -372,6 +363,36 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+// A[m][kk] = F[kk mod P][m mod P] where row m = jb P + p and column kk = kb P + r share the block (jb == kb),
+// K-major: element at (m/8)*128 + (kk/8)*2048 + (m%8)*16 + (kk%8)*2, hi part then lo part (KT*256 bytes each);
+// behind them w[jj][k2] = e^{2 pi i k2 jj / J} as (w.x, w.x, w.y, w.y).  Built once per call.
+__global__ void __launch_bounds__(256) spu_inv2_img_kernel(unsigned char* __restrict__ img, int P, int KT, int J, int KB) {
+    const int idx = blockIdx.x * 256 + threadIdx.x;
+    if (idx < 128 * KT) {
+        const int m = idx / KT, kk = idx - m * KT;
+        const int jb = m / P, p = m - jb * P, kb = kk / P, r = kk - kb * P;
+        float v = 0.f;
+        if (m < KT && jb == kb) {
+            if (r == 0) v = 1.f;
+            else if (r == 1) v = (p & 1) ? -1.f : 1.f;
+            else {
+                float s, c;
+                sincospif(2.0f * (float)(((r >> 1) * p) % P) / (float)P, &s, &c);
+                v = (r & 1) ? -s : c;
+            }
+        }
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        const int off = (m >> 3) * 128 + (kk >> 3) * 2048 + (m & 7) * 16 + (kk & 7) * 2;
+        *reinterpret_cast<__nv_bfloat16*>(img + off) = h;
+        *reinterpret_cast<__nv_bfloat16*>(img + KT * 256 + off) = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+    if (idx < J * KB) {
+        const int jj = idx / KB, k2 = idx - jj * KB;
+        const float2 w = root_pos(((unsigned)jj * (unsigned)k2) % (unsigned)J, J);
+        reinterpret_cast<float4*>(img + 2 * KT * 256)[idx] = make_float4(w.x, w.x, w.y, w.y);
+    }
+}
+
 template <int KB, int W>
 cudaError_t launch_inv2(const InvArgs& a, cudaStream_t stream) {
     const int KT = a.nblk * a.P;
@@ -418,10 +439,16 @@ SpuInv2Plan spu_inv2_plan(int B, int N, int D, int sigma) {
     return pl;
 }
 
-int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream) {
+int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream, void* img) {
     const SpuInv2Plan pl = spu_inv2_plan(B, N, D, sigma);
     if (!pl.ok) return LUVC_ERR_INTERNAL;
+    {
+        const int KT = pl.nblk * pl.P, n = 128 * KT > pl.J * pl.KB ? 128 * KT : pl.J * pl.KB;
+        spu_inv2_img_kernel<<<(n + 255) / 256, 256, 0, stream>>>(static_cast<unsigned char*>(img), pl.P, KT, pl.J, pl.KB);
+        count_launch();
+    }
     InvArgs a;
+    a.img = static_cast<const unsigned char*>(img);
     a.Y = Y; a.part = part; a.status = status;
     a.B = B; a.N = N; a.D = D; a.P = pl.P; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
     a.nblk = pl.nblk; a.J = pl.J; a.L = pl.L; a.n_ctiles = pl.n_ctiles; a.n_items = pl.n_items;
