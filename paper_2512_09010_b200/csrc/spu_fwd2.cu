@@ -41,7 +41,7 @@ constexpr int kThreads = kEpiThreads;         // no producer warps: thread 0 als
 constexpr int kNmma = 256;                    // columns of a tile: QT tokens x C channels
 constexpr int kTmemCols = 512;                // two accumulator buffers
 constexpr int kSpin = 1 << 22;
-constexpr int kProducer = 96;                 // thread that issues TMA and MMA: lane 0 of a warp with the fewest bins
+constexpr int kProducer = 96;                 // its warp issues TMA and MMA (one elected lane): a warp with the fewest bins
 constexpr int kStaticTabBytes = 24 * 1024;
 
 struct FwdArgs {
@@ -256,29 +256,39 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
         const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
         const int c0 = ctile * item_channels, buf = v & 1;
         // boxes that reach past Q or D are filled with zeros there and still count in full
-        mbar_arrive_expect_tx(bar(kBarFull + buf), (uint32_t)stage_bytes);
-        for (int jb = 0; jb < a.nblk; ++jb)
-            tma_load_4d(xs + buf * stage_bytes + jb * blk_bytes, &tmap, bar(kBarFull + buf), c0 + jb * C, 0, tile * QT, b);
+        if (elect_one()) {
+            mbar_arrive_expect_tx(bar(kBarFull + buf), (uint32_t)stage_bytes);
+            for (int jb = 0; jb < a.nblk; ++jb)
+                tma_load_4d(xs + buf * stage_bytes + jb * blk_bytes, &tmap, bar(kBarFull + buf), c0 + jb * C, 0, tile * QT, b);
+        }
+        __syncwarp();
     };
     auto issue_mma = [&](int v) -> bool {   // needs tile v in its stage and accumulator v & 1 drained
         const int buf = v & 1;
-        if (!wait_bar(bar(kBarFull + buf), (v >> 1) & 1, fail, a.status)) return false;
-        if (v >= 2 && !wait_bar(bar(kBarAccEmpty + buf), ((v - 2) >> 1) & 1, fail, a.status)) return false;
+        if (!__all_sync(0xffffffffu, wait_bar(bar(kBarFull + buf), (v >> 1) & 1, fail, a.status))) return false;
+        if (v >= 2 && !__all_sync(0xffffffffu, wait_bar(bar(kBarAccEmpty + buf), ((v - 2) >> 1) & 1, fail, a.status))) return false;
         tc_fence_after();
         const uint32_t acc = tmem + (uint32_t)(buf * kNmma);
-        uint64_t ah = a_hi0, al = a_lo0;             // descriptors advance by adding to the address field
-        for (int jb = 0; jb < a.nblk; ++jb) {        // K rows of channel block jb
-            uint64_t bd = b0 + (uint64_t)((buf * stage_bytes + jb * blk_bytes) >> 4);
-            for (int kl = 0; kl < P / 16; ++kl) {
-                umma_bf16(acc, ah, bd, idesc, (jb | kl) ? 1u : 0u);
-                umma_bf16(acc, al, bd, idesc, 1u);
-                ah += 4096 >> 4; al += 4096 >> 4; bd += (16 * ROWB) >> 4;
+        if (elect_one()) {
+            uint64_t ah = a_hi0, al = a_lo0;             // descriptors advance by adding to the address field
+            for (int jb = 0; jb < a.nblk; ++jb) {        // K rows of channel block jb
+                uint64_t bd = b0 + (uint64_t)((buf * stage_bytes + jb * blk_bytes) >> 4);
+                for (int kl = 0; kl < P / 16; ++kl) {
+                    umma_bf16(acc, ah, bd, idesc, (jb | kl) ? 1u : 0u);
+                    umma_bf16(acc, al, bd, idesc, 1u);
+                    ah += 4096 >> 4; al += 4096 >> 4; bd += (16 * ROWB) >> 4;
+                }
             }
+            umma_commit(bar(kBarAccFull + buf));
         }
-        umma_commit(bar(kBarAccFull + buf));
+        __syncwarp();
         return true;
     };
-    if (tid == kProducer) {
+    // The producer is a whole warp running warp-uniform code, with one elected lane issuing: the descriptors
+    // then stay in uniform registers (a tcgen05.mma issued from divergent code costs its thread twice as long).
+    const int warp_u = __shfl_sync(0xffffffffu, warp, 0);
+    const bool producer = warp_u == kProducer / 32;
+    if (producer && total_tiles > 0) {
         issue_tma(0);
         if (total_tiles > 1) issue_tma(1);
         issue_mma(0);
@@ -333,7 +343,8 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                     tab = tw;
                 }
                 ok = wait_bar(bar(kBarAccFull + buf), par, fail, a.status) && ok;
-                if (tid == kProducer && ok) {
+                ok = __all_sync(0xffffffffu, ok);
+                if (producer && ok) {
                     // the MMAs of tile u are done: refill their stage, and start tile u + 1
                     if (u + 2 < total_tiles) issue_tma(u + 2);
                     if (u + 1 < total_tiles) ok = issue_mma(u + 1);

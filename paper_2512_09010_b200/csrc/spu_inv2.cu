@@ -214,6 +214,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
         return;
     }
 
+    const int warp_u = __shfl_sync(0xffffffffu, warp, 0);   // the same in every lane, and the compiler can tell
     const int quarter = warp & 3, grp = warp >> 2;
     const int j = quarter * 32 + lane;               // row (channel block jb, r) of G; row (jb, point p) of the result
     const int jb = j / P, jr = j - jb * P;
@@ -320,11 +321,13 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarReady + (t & 1)));
-            if (tid == 0) {
+            if (warp_u == 0) {
                 // every warp has written its share of B (and, before that, read the last of accumulator
-                // t & 1, which held tile t - 2): run the three products
-                ok = wait_bar(bar(kBarReady + (t & 1)), (t >> 1) & 1, fail, a.status);
-                if (ok) {
+                // t & 1, which held tile t - 2): run the three products.  The whole warp waits and one
+                // elected lane issues, in warp-uniform code, so that the descriptors stay in uniform
+                // registers (a tcgen05.mma issued from divergent code costs its thread twice as long).
+                ok = __all_sync(0xffffffffu, wait_bar(bar(kBarReady + (t & 1)), (t >> 1) & 1, fail, a.status));
+                if (ok && elect_one()) {
                     tc_fence_after();
                     const uint32_t acc = tmem + (uint32_t)((t & 1) * kNcol);
                     uint64_t ah = a_hi0, al = a_lo0;             // advance by adding to the address field
@@ -337,6 +340,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
                     }
                     umma_commit(bar(kBarAccFull + (t & 1)));
                 }
+                __syncwarp();
             }
             // meanwhile: the energies of the previous tile, whose MMAs ran under the arithmetic above
             if (t >= 1) ok = wait_bar(bar(kBarAccFull + ((t - 1) & 1)), ((t - 1) >> 1) & 1, fail, a.status) && ok;
