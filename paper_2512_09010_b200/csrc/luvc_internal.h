@@ -139,9 +139,26 @@ struct SpuFwd3Plan {
     int C, n_ctiles, n_items;
 };
 SpuFwd3Plan spu_fwd3_plan(int B, int N, int D, int sigma);
-// Y[b][r][d] = c[r] * (band spectrum), the layout spu_fwd2_run writes.
-int spu_fwd3_run(const void* hidden, float* Y, const float* scale, int B, int N, int D, int sigma, int* status,
-                 cudaStream_t stream, void* img);
+// Writes the band spectrum (times c[r]) in the operand form of spu_inv3.cu, ks_out K steps per channel, and, if one more
+// bin per frequency class reaches into the band than a pass holds, that bin's cos and sin values to yx[2][B][D].
+int spu_fwd3_run(const void* hidden, void* yop, int ks_out, float* yx, const float* scale, int B, int N, int D, int sigma,
+                 int* status, cudaStream_t stream, void* img);
+
+// Inverse transform and energies with both stages on the tensor cores (spu_inv3.cu): N = 128 Q, the band spectrum in
+// "operand form" (per sequence and channel: [K step][K chunk][128 lanes][16 B], four bf16 per bin).
+struct SpuInv3Plan {
+    int ok;             // 0: use the two-stage kernel of spu_inv2.cu
+    int coarse, J, L;   // as SpuInv2Plan
+    int KS;             // K steps of four bins each
+    int JP;             // points per channel held in tensor memory: 16, 40 or 72
+    int extra;          // 1: the bin k = 128 * 16 reaches into the band and is passed apart
+    int n_ctiles, n_items, n_parts;
+    size_t yop_bytes;   // size of the band spectrum in operand form
+};
+SpuInv3Plan spu_inv3_plan(int B, int N, int D, int sigma);
+// yx_re / yx_im: the cos and sin value of the bin k = 128 * 16 for (b, d) at [b * yx_stride + d] (read only if plan.extra).
+int spu_inv3_run(const void* yop, const float* yx_re, const float* yx_im, long long yx_stride, float* part, int B, int N,
+                 int D, int sigma, int* status, cudaStream_t stream, void* img);
 
 // Two-stage inverse transform and energies of the bf16 path (spu_inv2.cu); needs the forward plan.
 struct SpuInv2Plan {

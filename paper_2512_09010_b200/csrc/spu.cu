@@ -389,11 +389,14 @@ struct Workspace {
     SpuTcBuffers tc;
     float* Y2;       // band spectrum of the two-stage forward transform [B][2 sigma + 1][D]
     void *img_fwd, *img_inv;   // operand images of the forward / inverse transform kernel, built once per call
+    void* yop;       // band spectrum in the operand form of the tensor-core inverse
+    float* yx;       // [2][B][D] its one bin past sixteen per frequency class
 };
 
 // How the bf16 path runs a problem, and the points its inverse is evaluated on.
 struct Bf16Mode {
     bool fwd2, inv2;    // two-stage forward / inverse kernels (else the dense contractions of spu_tc.cu)
+    bool tc2;           // both of them with their second stage on the tensor cores too (spu_fwd3.cu, spu_inv3.cu)
     int coarse, L;      // the inverse is evaluated on L uniform points of the period (L = N: the tokens)
     int n_parts;        // partial energy sums per point
 };
@@ -404,9 +407,11 @@ Bf16Mode bf16_mode(int B, int N, int D, int sigma, bool dense) {
     m.fwd2 = !dense && spu_fwd2_plan(B, N, D, sigma).ok != 0;   // `dense`: rows come through an index, which only
                                                                 // the dense contractions can follow
     m.inv2 = m.fwd2 && iv.ok != 0;
+    const SpuInv3Plan iv3 = spu_inv3_plan(B, N, D, sigma);       // (needs the plan of spu_fwd3.cu)
+    m.tc2 = m.inv2 && iv3.ok != 0;
     m.coarse = m.inv2 ? iv.coarse : tc.coarse;
     m.L = m.inv2 ? iv.L : tc.L;
-    m.n_parts = m.inv2 ? iv.n_parts : 2 * tc.tiles2;
+    m.n_parts = m.tc2 ? iv3.n_parts : (m.inv2 ? iv.n_parts : 2 * tc.tiles2);
     return m;
 }
 
@@ -436,7 +441,12 @@ Workspace carve(void* ws, int B, int N, int D, int sigma, bool tensor_path, bool
             w.gpart = reinterpret_cast<float2*>(take(coarse_gpart_elems(B, m.L, sigma) * sizeof(float2)));
         }
         if (m.fwd2) {
-            w.Y2 = reinterpret_cast<float*>(take((size_t)B * R * D * sizeof(float)));
+            if (m.tc2) {
+                w.yop = take(spu_inv3_plan(B, N, D, sigma).yop_bytes);
+                w.yx = reinterpret_cast<float*>(take((size_t)2 * B * D * sizeof(float)));
+            } else {
+                w.Y2 = reinterpret_cast<float*>(take((size_t)B * R * D * sizeof(float)));
+            }
             w.img_fwd = take(kSpuImgBytes);
             w.img_inv = take(kSpuImgBytes);
         }
@@ -487,17 +497,23 @@ static int spu_run_typed(const SpuProblem& p) {
                                                                p.no_window);
     count_launch();
     if constexpr (kTensor) {
-        if (mode.fwd2 && mode.inv2 && spu_fwd3_plan(B, N, D, sigma).ok) {
-            const int rc1 = spu_fwd3_run(p.hidden, ws.Y2, ws.scale, B, N, D, sigma, p.status, p.stream, ws.img_fwd);
-            if (rc1 != LUVC_OK) return rc1;
-        } else if (mode.fwd2) {
-            const int rc1 = spu_fwd2_run(p.hidden, ws.Y2, ws.scale, mode.inv2 ? nullptr : ws.tc.yt_hi,
-                                         mode.inv2 ? nullptr : ws.tc.yt_lo, pl.r_pad, B, N, D, sigma, p.status, p.stream, ws.img_fwd);
-            if (rc1 != LUVC_OK) return rc1;
+        int rc;
+        if (mode.tc2) {
+            const SpuInv3Plan iv3 = spu_inv3_plan(B, N, D, sigma);
+            rc = spu_fwd3_run(p.hidden, ws.yop, iv3.KS, ws.yx, ws.scale, B, N, D, sigma, p.status, p.stream, ws.img_fwd);
+            if (rc != LUVC_OK) return rc;
+            rc = spu_inv3_run(ws.yop, ws.yx, ws.yx + (size_t)B * D, D, ws.tc.part, B, N, D, sigma, p.status, p.stream,
+                              ws.img_inv);
+        } else {
+            if (mode.fwd2) {
+                const int rc1 = spu_fwd2_run(p.hidden, ws.Y2, ws.scale, mode.inv2 ? nullptr : ws.tc.yt_hi,
+                                             mode.inv2 ? nullptr : ws.tc.yt_lo, pl.r_pad, B, N, D, sigma, p.status, p.stream, ws.img_fwd);
+                if (rc1 != LUVC_OK) return rc1;
+            }
+            rc = mode.inv2 ? spu_inv2_run(ws.Y2, ws.tc.part, B, N, D, sigma, p.status, p.stream, ws.img_inv)
+                           : spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status,
+                                        p.stream, mode.fwd2, p.row_index, p.src_rows);
         }
-        const int rc = mode.inv2 ? spu_inv2_run(ws.Y2, ws.tc.part, B, N, D, sigma, p.status, p.stream, ws.img_inv)
-                                 : spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status,
-                                              p.stream, mode.fwd2, p.row_index, p.src_rows);
         if (rc != LUVC_OK) return rc;
         if (!mode.coarse) {
             spu_energy_kernel<<<(unsigned)((bn + 31) / 32), 256, 0, p.stream>>>(ws.tc.part, E, N, mode.n_parts, bn, 0);

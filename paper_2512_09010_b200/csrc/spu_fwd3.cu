@@ -51,14 +51,14 @@ constexpr int kTN = 64;                       // columns of a tile = QT tokens x
 constexpr int kSlotCols = 2 * kTN;            // TMEM columns of the stage-2 operand of one tile (16 units of 8)
 constexpr int kUnits = 16;                    // stage-2 units of a tile: four per converter thread
 constexpr int kStages = 4;                    // input stages in shared memory
-constexpr int kOutStageBytes = 4 * 32 * 40 * 4;   // per lane quadrant up to 32 x 40 floats of the band spectrum on its way out
 
 struct Fwd3Args {
     const __nv_bfloat16* x;   // [B][N][D]
-    float* Y;                 // [B][R][D]
+    unsigned char* yop;       // band spectrum in operand form: [B][D][ks_out][2 K chunks][128 lanes][16 B]
+    float* yx;                // [2][B][D]: cos and sin value of the bin 128 * extra_k2 (written only if extra_k2 > 0)
     const float* scale;       // c[r], r < R
     int* status;
-    int B, N, D, Q, sigma, R;
+    int B, N, D, Q, sigma, ks_out;
     int n_ctiles, n_slices, n_items;
     const unsigned char* img; // stage-1 matrix, stage-2 matrices and root tables in their shared-memory layouts (built once per call)
     int extra_k2;             // > 0: one more value of k2 (= K2MAX) reaches into the band, for a few lanes only; those
@@ -152,99 +152,6 @@ struct Geo {
                   "a tile is sixteen units, four per converter thread");
 };
 
-// The band spectrum of one work item on its way out of tensor memory, staged through shared memory so that whole
-// channel runs of a row are written per instruction (called by every converter thread).  Pays for itself when a
-// row of the item is short (8 channels: each direct store would touch 32 sectors for 4 bytes each); with 32
-// channels per row the direct stores of the kernel are as fast and need no barriers.
-template <typename G>
-__device__ __forceinline__ void drain_item_staged(const Fwd3Args& a, uint32_t lane_addr, uint32_t out_empty_bar, float* s_out, int quarter,
-                            int g, int lane, int b, int ctile, int k2_lo) {
-    constexpr int C = G::C, N2 = G::N2, QPU = G::QPU, W = G::W;
-    const int D = a.D, sigma = a.sigma;
-    // All of this thread's result columns at once (64 values), then tensor memory is free for the next item.
-    uint32_t o[4][16];
-#pragma unroll
-    for (int h = 0; h < 4; ++h) tmem_ld16(lane_addr + (uint32_t)(G::OUT0 + g * G::UT * N2 + h * 16), o[h]);
-    tmem_ld_wait_for(reinterpret_cast<uint32_t(&)[16]>(o[0]));
-    tmem_ld_wait_for(reinterpret_cast<uint32_t(&)[16]>(o[1]));
-    tmem_ld_wait_for(reinterpret_cast<uint32_t(&)[16]>(o[2]));
-    tmem_ld_wait_for(reinterpret_cast<uint32_t(&)[16]>(o[3]));
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(out_empty_bar);
-    // A lane is a row of Y (one frequency), so a thread's values go to as many different rows as the warp
-    // has lanes: written straight from here every store would touch 32 sectors for a few bytes each.
-    // Instead the four warps of a TMEM lane quadrant (the four channel groups of the same 32 rows) pass
-    // their values through a small staging matrix in shared memory, one (k2, re/im) slice of the item at
-    // a time (kSlicesPerRound of them per round), and write whole channel runs of a row per instruction.
-    constexpr int kStride = C + (C == 8 ? 2 : 4);        // floats per staged row: padded against bank conflicts
-    constexpr int kSlicesPerRound = C == 8 ? 4 : 1;
-    constexpr int kSlices = 2 * G::K2MAX;                // slice s = k2 * 2 + re/im
-    float* stage = s_out + quarter * (kSlicesPerRound * 32 * kStride);
-    const int bar_id = 1 + quarter;                      // named barrier of this quadrant's four warps
-    float* Yb = a.Y + (size_t)b * a.R * D + ctile * C;
-#pragma unroll
-    for (int r0 = 0; r0 < kSlices; r0 += kSlicesPerRound) {
-        // ---- every thread puts its channels of the round's slices into its row of the staging matrices
-#pragma unroll
-        for (int sl = 0; sl < kSlicesPerRound; ++sl) {
-            const int s_idx = r0 + sl, k2 = s_idx >> 1, ri = s_idx & 1;
-            float* row = stage + (sl * 32 + lane) * kStride + g * W;
-            if constexpr (QPU == 2) {
-                // unit h (channels 2h, 2h+1 of the thread's W): column cc * 8 + k2 * 2 + ri of o[h]
-                float vals[W];
-#pragma unroll
-                for (int h = 0; h < W / 2; ++h) {
-                    vals[2 * h] = __uint_as_float(o[h][k2 * 2 + ri]);
-                    vals[2 * h + 1] = __uint_as_float(o[h][8 + k2 * 2 + ri]);
-                }
-#pragma unroll
-                for (int c = 0; c < W; c += 4)
-                    *reinterpret_cast<float4*>(row + c) = make_float4(vals[c], vals[c + 1], vals[c + 2], vals[c + 3]);
-            } else {
-                // channel cc: columns (k2 % 8) * 2 + ri of o[2 cc + k2 / 8]
-                *reinterpret_cast<float2*>(row) = make_float2(__uint_as_float(o[k2 >> 3][(k2 & 7) * 2 + ri]),
-                                                              __uint_as_float(o[2 + (k2 >> 3)][(k2 & 7) * 2 + ri]));
-            }
-        }
-        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-        // ---- and the four warps write the staged rows out, a whole run of channels per row
-        if constexpr (C == 8) {
-            // this warp takes slice r0 + g: 32 rows x 8 channels, four rows per instruction
-            const int s_idx = r0 + g, k2 = s_idx >> 1, ri = s_idx & 1;
-            const int ch = lane & 7;
-#pragma unroll
-            for (int it = 0; it < 8; ++it) {
-                const int rr = it * 4 + (lane >> 3);                     // row of the quadrant
-                const int jr = quarter * 32 + rr, ir = jr >> 1;
-                const int kfr = (ir == 0 ? ((jr & 1) ? kP / 2 : 0) : ((jr & 1) ? kP - ir : ir)) + kP * k2_lo;
-                const int k = kfr + kP * k2;
-                if (k <= sigma && ctile * C + ch < D && !(ri == 1 && k == 0)) {
-                    const float v = stage[(g * 32 + rr) * kStride + ch];
-                    const int rowi = ri ? sigma + k : k;
-                    Yb[(size_t)rowi * D + ch] = __ldg(a.scale + rowi) * v;
-                }
-            }
-        } else {
-            // one slice per round: this warp takes rows 8 g .. 8 g + 7, a lane per channel
-            const int k2 = r0 >> 1, ri = r0 & 1;
-#pragma unroll
-            for (int it = 0; it < 8; ++it) {
-                const int rr = g * 8 + it;
-                const int jr = quarter * 32 + rr, ir = jr >> 1;
-                const int kfr = (ir == 0 ? ((jr & 1) ? kP / 2 : 0) : ((jr & 1) ? kP - ir : ir)) + kP * k2_lo;
-                const int k = kfr + kP * k2;
-                if (k <= sigma && lane < C && ctile * C + lane < D && !(ri == 1 && k == 0)) {
-                    const float v = stage[rr * kStride + lane];
-                    const int rowi = ri ? sigma + k : k;
-                    Yb[(size_t)rowi * D + lane] = __ldg(a.scale + rowi) * v;
-                }
-            }
-        }
-        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-    }
-}
-
 template <typename G, bool EXTRA>
 __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_constant__ CUtensorMap tmap, const Fwd3Args a) {
     constexpr int C = G::C, N2 = G::N2, QPU = G::QPU, QT = G::QT, W = G::W;
@@ -264,7 +171,6 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
     unsigned char* s_w = s_x + kStages * G::STAGE_BYTES;                // [n_groups][hi, lo][16 x N2] stage-2 matrices
     float2* s_root = reinterpret_cast<float2*>(s_w + (size_t)n_groups * 2 * G::W_BYTES);   // e^{-2 pi i m / Q}, m < Q
     float2* s_fine = s_root + ((Q + 1) & ~1);                                              // e^{-2 pi i m / N}, m < 128
-    float* s_out = reinterpret_cast<float*>(s_fine + kP);                                  // staging of the band spectrum on its way out
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -534,52 +440,73 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                 if (lane == 0) mbar_arrive(bar(kBarGrpFull + g * 2 + pending_slot));
             }
             if (!ok) break;
-            // ---- the item's band spectrum: out of tensor memory, times the row constants, to Y
+            // ---- the item's band spectrum: out of tensor memory, times the row constants, split into bf16 pairs and
+            // stored in operand form: per channel and K chunk (two bins) the 128 lanes write 16 bytes each, side by side
             ok = wait_bar(bar(kBarOutFull), item_seq & 1, fail, a.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if constexpr (C == 8) {
-                drain_item_staged<G>(a, lane_addr, bar(kBarOutEmpty), s_out, quarter, g, lane, b, ctile, k2_lo);
-            } else {
-                // 32 channels per row: this thread's eight channels of a row are one 32-byte sector, written as float2 pairs
-                const int nb = kfe <= sigma ? min(G::K2MAX, (sigma - kfe) / kP + 1) : 0;   // bins of this lane in this slice
+            {
                 const int ch0 = ctile * C + g * W;                   // first of this thread's channels
-                float* Yb = a.Y + (size_t)b * a.R * D + ch0;
-                const bool live = ch0 < D;                           // D is a multiple of 8 and ch0 of W: whole or absent
+                const size_t chan_bytes = (size_t)a.ks_out * 4096;
+                unsigned char* yb = a.yop + ((size_t)b * D + ch0) * chan_bytes + (size_t)j * 16;
+                // two bins (k2, k2 + 1) of one channel: (Re hi, Im hi, Re lo, Im lo) each; bins past the band are zero
+                auto chunk = [&](const uint32_t* o, int k2) {
+                    uint32_t w[4];
 #pragma unroll
-                for (int h = 0; h < (G::UT * N2) / 16; ++h) {
-                    uint32_t o[16];
-                    tmem_ld16(lane_addr + (uint32_t)(G::OUT0 + g * G::UT * N2 + h * 16), o);
-                    tmem_ld_wait_for(o);
-                    // unit h: channels 2h, 2h+1 of the thread; column = cc * 8 + k2 * 2 + ri
+                    for (int z = 0; z < 2; ++z) {
+                        const int k = kfe + kP * (k2 + z);
+                        const bool in = k <= sigma;
+                        const float cr = in ? __ldg(a.scale + k) : 0.f, ci = (in && k >= 1) ? __ldg(a.scale + sigma + k) : 0.f;
+                        const float re = cr * __uint_as_float(o[2 * z]), im = ci * __uint_as_float(o[2 * z + 1]);
+                        const uint32_t hi = bf16x2_bits(re, im);
+                        w[2 * z] = hi;
+                        w[2 * z + 1] = bf16x2_bits(re - __uint_as_float(hi << 16), im - __uint_as_float(hi & 0xffff0000u));
+                    }
+                    return make_uint4(w[0], w[1], w[2], w[3]);
+                };
+                if constexpr (QPU == 2) {
+                    // unit h: channels 2h, 2h+1 of the thread; column = cc * 8 + k2 * 2 + ri: one K step of four bins
 #pragma unroll
-                    for (int k2 = 0; k2 < 4; ++k2) {
-                        if (k2 >= nb || !live) continue;
-                        const int k = kfe + kP * k2;
-                        const float cr = __ldg(a.scale + k), ci = k >= 1 ? __ldg(a.scale + sigma + k) : 0.f;
-                        float* yc = Yb + (size_t)k * D + 2 * h;
-                        *reinterpret_cast<float2*>(yc) = make_float2(cr * __uint_as_float(o[k2 * 2]), cr * __uint_as_float(o[8 + k2 * 2]));
-                        if (k >= 1)
-                            *reinterpret_cast<float2*>(yc + (size_t)sigma * D) =
-                                make_float2(ci * __uint_as_float(o[k2 * 2 + 1]), ci * __uint_as_float(o[8 + k2 * 2 + 1]));
+                    for (int h = 0; h < (G::UT * N2) / 16; ++h) {
+                        uint32_t o[16];
+                        tmem_ld16(lane_addr + (uint32_t)(G::OUT0 + g * G::UT * N2 + h * 16), o);
+                        tmem_ld_wait_for(o);
+#pragma unroll
+                        for (int cc = 0; cc < 2; ++cc) {
+                            if (ch0 + 2 * h + cc >= D) continue;
+                            unsigned char* yc = yb + (size_t)(2 * h + cc) * chan_bytes;
+                            *reinterpret_cast<uint4*>(yc) = chunk(o + cc * 8, 0);
+                            *reinterpret_cast<uint4*>(yc + 2048) = chunk(o + cc * 8 + 4, 2);
+                        }
+                    }
+                } else {
+                    // channel cc of the thread: 32 columns, k2 * 2 + ri: K step s holds bins 4 s .. 4 s + 3
+#pragma unroll
+                    for (int cc = 0; cc < W; ++cc) {
+                        for (int s2 = 0; s2 < a.ks_out; ++s2) {
+                            uint32_t o[8];
+                            tmem_ld8(lane_addr + (uint32_t)(G::OUT0 + g * G::UT * N2 + cc * N2 + s2 * 8), o);
+                            tmem_ld_wait_for(o);
+                            if (ch0 + cc >= D) continue;
+                            unsigned char* yc = yb + (size_t)cc * chan_bytes + (size_t)s2 * 4096;
+                            *reinterpret_cast<uint4*>(yc) = chunk(o, 4 * s2);
+                            *reinterpret_cast<uint4*>(yc + 2048) = chunk(o + 4, 4 * s2 + 2);
+                        }
                     }
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarOutEmpty));
-            }
-            {
                 if (EXTRA) {
-                    const int ch0 = ctile * C + g * W;
                     const int k = kfe + kP * a.extra_k2;
                     if (k <= sigma && ch0 < D) {
                         const float cr = __ldg(a.scale + k), ci = __ldg(a.scale + sigma + k);
-                        float* Ye = a.Y + (size_t)b * a.R * D + ch0;
+                        float* yx = a.yx + (size_t)b * D + ch0;
 #pragma unroll
                         for (int c = 0; c < W; ++c) {
-                            Ye[(size_t)k * D + c] = cr * extra[c].x;
-                            Ye[(size_t)(sigma + k) * D + c] = ci * extra[c].y;
+                            yx[c] = cr * extra[c].x;
+                            yx[(size_t)a.B * D + c] = ci * extra[c].y;
                         }
                     }
                 }
@@ -668,7 +595,7 @@ EncodeTiledFn encode_tiled_fn() {
 template <typename G>
 size_t fwd3_smem(int Q) {
     const int tiles = (Q + G::QT - 1) / G::QT, groups = tiles * G::GQ;
-    return 1024 + 65536 + (size_t)kStages * G::STAGE_BYTES + (size_t)groups * 2 * G::W_BYTES + (size_t)(((Q + 1) & ~1) + kP) * sizeof(float2) + kOutStageBytes;
+    return 1024 + 65536 + (size_t)kStages * G::STAGE_BYTES + (size_t)groups * 2 * G::W_BYTES + (size_t)(((Q + 1) & ~1) + kP) * sizeof(float2);
 }
 
 template <typename G, bool EXTRA>
@@ -735,14 +662,15 @@ SpuFwd3Plan spu_fwd3_plan(int B, int N, int D, int sigma) {
     return pl;
 }
 
-int spu_fwd3_run(const void* hidden, float* Y, const float* scale, int B, int N, int D, int sigma, int* status,
-                 cudaStream_t stream, void* img) {
+int spu_fwd3_run(const void* hidden, void* yop, int ks_out, float* yx, const float* scale, int B, int N, int D, int sigma,
+                 int* status, cudaStream_t stream, void* img) {
     const SpuFwd3Plan pl = spu_fwd3_plan(B, N, D, sigma);
     if (!pl.ok) return LUVC_ERR_INTERNAL;
     Fwd3Args a;
     a.x = reinterpret_cast<const __nv_bfloat16*>(hidden);
-    a.Y = Y; a.scale = scale; a.status = status;
-    a.B = B; a.N = N; a.D = D; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
+    if (pl.slices != 1 || ks_out * 4 > (pl.wide ? GeoWide::K2MAX : GeoNarrow::K2MAX)) return LUVC_ERR_INTERNAL;
+    a.yop = static_cast<unsigned char*>(yop); a.yx = yx; a.ks_out = ks_out; a.scale = scale; a.status = status;
+    a.B = B; a.N = N; a.D = D; a.Q = pl.Q; a.sigma = sigma;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
     a.extra_k2 = pl.extra_k2;
     a.img = static_cast<const unsigned char*>(img);
