@@ -260,6 +260,124 @@ __global__ void __launch_bounds__(256) spu_coarse_synthesis_kernel(const float2*
     }
 }
 
+// ---- the same interpolation in two stages, for L = P J samples and N = P Q tokens ---------------
+//
+// Analysis, sample j = J j1 + j2, coefficient f = f1 + P f2:
+//   g_f = (1/L) sum_{j2} e^{-2 pi i f2 j2 / J} [ e^{-2 pi i f1 j2 / L} sum_{j1} S_{J j1 + j2} e^{-2 pi i f1 j1 / P} ]
+// Synthesis, token n = Q n1 + n2:
+//   S(n) = Re sum_{f1} e^{2 pi i f1 n1 / P} [ e^{2 pi i f1 n2 / N} sum_{f2} g'_{f1 + P f2} e^{2 pi i f2 n2 / Q} ]
+// with g'_0 = g_0, g'_f = 2 g_f.  P (F / P + 1) (J + Q) + P^2 (J + Q) products per sequence instead of (F + 1)(L + N / 2),
+// every root taken from an exact table.  A CTA takes eight values of f1 (analysis) or of n2 (synthesis).
+
+constexpr int kInterpSlice = 8;
+
+__device__ __forceinline__ float2 cmul_f(float2 a, float2 b) {
+    return make_float2(a.x * b.x - a.y * b.y, fmaf(a.x, b.y, a.y * b.x));
+}
+
+// G[b][f] = g'_f, f <= F, from S[b][L]
+__global__ void __launch_bounds__(256) spu_interp_analysis_kernel(const float* __restrict__ S, float2* __restrict__ G,
+                                                                  int P, int J, int F) {
+    extern __shared__ __align__(16) unsigned char interp_smem[];
+    const int L = P * J, b = blockIdx.y, f1_0 = blockIdx.x * kInterpSlice;
+    float* s_val = reinterpret_cast<float*>(interp_smem);                        // [L]
+    float2* s_rp = reinterpret_cast<float2*>(s_val + ((L + 3) & ~3));             // e^{-2 pi i m / P}
+    float2* s_rj = s_rp + P;                                                      // e^{-2 pi i m / J}
+    float2* s_t = s_rj + J;                                                       // [kInterpSlice][J]
+    for (int i = threadIdx.x; i < L; i += 256) s_val[i] = S[(size_t)b * L + i];
+    for (int i = threadIdx.x; i < P; i += 256) { const float2 r = unit_root(i, P); s_rp[i] = make_float2(r.x, -r.y); }
+    for (int i = threadIdx.x; i < J; i += 256) { const float2 r = unit_root(i, J); s_rj[i] = make_float2(r.x, -r.y); }
+    __syncthreads();
+    for (int o = threadIdx.x; o < kInterpSlice * J; o += 256) {
+        const int fl = o / J, j2 = o - fl * J, f1 = f1_0 + fl;
+        float re = 0.f, im = 0.f;
+        if (f1 < P) {
+            int m = 0;                                   // f1 j1 mod P
+            for (int j1 = 0; j1 < P; ++j1) {
+                const float v = s_val[J * j1 + j2];
+                const float2 w = s_rp[m];
+                re = fmaf(v, w.x, re);
+                im = fmaf(v, w.y, im);
+                m += f1;
+                if (m >= P) m -= P;
+            }
+            const float2 tw = unit_root((long long)f1 * j2, L);       // f1 j2 < P J = L
+            const float2 t = cmul_f(make_float2(re, im), make_float2(tw.x, -tw.y));
+            re = t.x; im = t.y;
+        }
+        s_t[o] = make_float2(re, im);
+    }
+    __syncthreads();
+    const int nf2 = F / P + 1;
+    const float inv_l = 1.0f / (float)L;
+    for (int o = threadIdx.x; o < kInterpSlice * nf2; o += 256) {
+        const int fl = o / nf2, f2 = o - fl * nf2, f1 = f1_0 + fl, f = f1 + P * f2;
+        if (f1 >= P || f > F) continue;
+        float re = 0.f, im = 0.f;
+        int m = 0;                                       // f2 j2 mod J
+        const int step = f2 % J;
+        for (int j2 = 0; j2 < J; ++j2) {
+            const float2 t = s_t[fl * J + j2], w = s_rj[m];
+            re = fmaf(t.x, w.x, fmaf(-t.y, w.y, re));
+            im = fmaf(t.x, w.y, fmaf(t.y, w.x, im));
+            m += step;
+            if (m >= J) m -= J;
+        }
+        const float sc = f == 0 ? inv_l : 2.0f * inv_l;
+        G[(size_t)b * (F + 1) + f] = make_float2(re * sc, im * sc);
+    }
+}
+
+// E[b][n] = sqrt(max(0, S(n))) from G[b][f]
+__global__ void __launch_bounds__(256) spu_interp_synthesis_kernel(const float2* __restrict__ G, float* __restrict__ E,
+                                                                   int P, int Q, int F) {
+    extern __shared__ __align__(16) unsigned char interp_smem[];
+    const int N = P * Q, b = blockIdx.y, n2_0 = blockIdx.x * kInterpSlice;
+    float2* s_g = reinterpret_cast<float2*>(interp_smem);      // [F + 1]
+    float2* s_rp = s_g + F + 1;                                 // e^{2 pi i m / P}
+    float2* s_rq = s_rp + P;                                    // e^{2 pi i m / Q}
+    float2* s_u = s_rq + Q;                                     // [P][kInterpSlice]
+    for (int i = threadIdx.x; i <= F; i += 256) s_g[i] = G[(size_t)b * (F + 1) + i];
+    for (int i = threadIdx.x; i < P; i += 256) s_rp[i] = unit_root(i, P);
+    for (int i = threadIdx.x; i < Q; i += 256) s_rq[i] = unit_root(i, Q);
+    __syncthreads();
+    for (int o = threadIdx.x; o < P * kInterpSlice; o += 256) {
+        const int f1 = o / kInterpSlice, n2 = n2_0 + (o % kInterpSlice);
+        float re = 0.f, im = 0.f;
+        if (n2 < Q) {
+            int m = 0;                                   // f2 n2 mod Q
+            for (int f = f1; f <= F; f += P) {
+                const float2 g = s_g[f], w = s_rq[m];
+                re = fmaf(g.x, w.x, fmaf(-g.y, w.y, re));
+                im = fmaf(g.x, w.y, fmaf(g.y, w.x, im));
+                m += n2;
+                if (m >= Q) m -= Q;
+            }
+            const float2 t = cmul_f(make_float2(re, im), unit_root((long long)f1 * n2, N));   // f1 n2 < P Q = N
+            re = t.x; im = t.y;
+        }
+        s_u[o] = make_float2(re, im);
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < P * kInterpSlice; o += 256) {
+        const int n1 = o / kInterpSlice, nl = o % kInterpSlice, n2 = n2_0 + nl;
+        if (n2 >= Q) continue;
+        float acc = 0.f;
+        int m = 0;                                       // f1 n1 mod P
+        for (int f1 = 0; f1 < P; ++f1) {
+            const float2 u = s_u[f1 * kInterpSlice + nl], w = s_rp[m];
+            acc = fmaf(u.x, w.x, fmaf(-u.y, w.y, acc));
+            m += n1;
+            if (m >= P) m -= P;
+        }
+        E[(size_t)b * N + (size_t)Q * n1 + n2] = sqrtf(fmaxf(acc, 0.f));
+    }
+}
+
+size_t interp_analysis_smem(int P, int J) { return ((size_t)((P * J + 3) & ~3)) * 4 + (size_t)(P + J + kInterpSlice * J) * 8; }
+size_t interp_synthesis_smem(int P, int Q, int F) { return (size_t)(F + 1 + P + Q + P * kInterpSlice) * 8; }
+constexpr size_t kInterpSmemMax = 200 * 1024;
+
 // ---- order-preserving top-k ---------------------------------------------------
 
 constexpr int kSelThreads = 1024;
@@ -399,6 +517,7 @@ struct Bf16Mode {
     bool tc2;           // both of them with their second stage on the tensor cores too (spu_fwd3.cu, spu_inv3.cu)
     int coarse, L;      // the inverse is evaluated on L uniform points of the period (L = N: the tokens)
     int n_parts;        // partial energy sums per point
+    int P, Q, J;        // two-stage kernels: N = P Q tokens, L = P J points
 };
 Bf16Mode bf16_mode(int B, int N, int D, int sigma, bool dense) {
     const SpuTcPlan tc = spu_tc_plan(B, N, D, sigma);
@@ -412,6 +531,7 @@ Bf16Mode bf16_mode(int B, int N, int D, int sigma, bool dense) {
     m.coarse = m.inv2 ? iv.coarse : tc.coarse;
     m.L = m.inv2 ? iv.L : tc.L;
     m.n_parts = m.tc2 ? iv3.n_parts : (m.inv2 ? iv.n_parts : 2 * tc.tiles2);
+    m.P = m.inv2 ? iv.P : 0; m.Q = m.inv2 ? iv.Q : 0; m.J = m.inv2 ? iv.J : 0;
     return m;
 }
 
@@ -522,8 +642,20 @@ static int spu_run_typed(const SpuProblem& p) {
             const int L = mode.L, F = 2 * sigma, chunks = (L + kSpecChunk - 1) / kSpecChunk;
             const long long bl = (long long)B * L;
             spu_energy_kernel<<<(unsigned)((bl + 31) / 32), 256, 0, p.stream>>>(ws.tc.part, ws.S, L, mode.n_parts, bl, 1);
-            spu_coarse_spectrum_kernel<<<dim3((F + 128) / 128, chunks, B), 128, 0, p.stream>>>(ws.S, ws.gpart, L, F);
-            spu_coarse_synthesis_kernel<<<dim3((N / 2 + 256) / 256, B), 256, 0, p.stream>>>(ws.gpart, E, N, L, F, chunks);
+            const size_t sm_a = mode.inv2 ? interp_analysis_smem(mode.P, mode.J) : 0;
+            const size_t sm_s = mode.inv2 ? interp_synthesis_smem(mode.P, mode.Q, F) : 0;
+            if (mode.inv2 && sm_a <= kInterpSmemMax && sm_s <= kInterpSmemMax) {
+                // L = P J and N = P Q: the interpolation factors into two short stages
+                cudaFuncSetAttribute(spu_interp_analysis_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_a);
+                cudaFuncSetAttribute(spu_interp_synthesis_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_s);
+                spu_interp_analysis_kernel<<<dim3((mode.P + kInterpSlice - 1) / kInterpSlice, B), 256, sm_a, p.stream>>>(
+                    ws.S, ws.gpart, mode.P, mode.J, F);
+                spu_interp_synthesis_kernel<<<dim3((mode.Q + kInterpSlice - 1) / kInterpSlice, B), 256, sm_s, p.stream>>>(
+                    ws.gpart, E, mode.P, mode.Q, F);
+            } else {
+                spu_coarse_spectrum_kernel<<<dim3((F + 128) / 128, chunks, B), 128, 0, p.stream>>>(ws.S, ws.gpart, L, F);
+                spu_coarse_synthesis_kernel<<<dim3((N / 2 + 256) / 256, B), 256, 0, p.stream>>>(ws.gpart, E, N, L, F, chunks);
+            }
             count_launch(3);
         }
     } else {
