@@ -343,6 +343,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
             float2 extra[W];                                         // bin kfe + 128 extra_k2 of this lane's channels
 #pragma unroll
             for (int c = 0; c < W; ++c) extra[c] = make_float2(0.f, 0.f);
+            // only the warps with a lane that reaches that bin accumulate it; the angle q extra_k2 mod Q is carried
+            // along in integers from token to token
+            const bool need_x = EXTRA && __any_sync(0xffffffffu, kfe + kP * a.extra_k2 <= sigma);
+            int x_angle = 0;
+            const int x_step = EXTRA ? a.extra_k2 % Q : 0;
             // The TMEM round trips are long (a load or a store takes several hundred cycles), so the loop is
             // software-pipelined: the next tile's values are requested before this tile's arithmetic, and
             // a tile's stores are only waited for (and its units handed to the MMA warp) one tile later.
@@ -397,15 +402,23 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                     // B = rot * (own + i cg other):  Re = rot.x own - cg rot.y other,  Im = rot.y own + cg rot.x other
                     const float ox = -cg * rot.y, oy = cg * rot.x;
                     float2 wex = make_float2(0.f, 0.f);              // e^{-2 pi i q extra_k2 / Q} of this token
-                    if constexpr (EXTRA) wex = s_root[(int)(((long long)(tile * QT + ql) * a.extra_k2) % Q)];
+                    if constexpr (EXTRA) {
+                        if (need_x) {
+                            wex = s_root[x_angle];
+                            x_angle += x_step;
+                            if (x_angle >= Q) x_angle -= Q;
+                        }
+                    }
 #pragma unroll
                     for (int c = 0; c < W; ++c) {
                         const float own = __uint_as_float(v[ql][c]);
                         const float other = __shfl_xor_sync(0xffffffffu, own, 1);
                         const float wx = fmaf(rot.x, own, ox * other), wy = fmaf(rot.y, own, oy * other);
                         if constexpr (EXTRA) {
-                            extra[c].x = fmaf(wx, wex.x, fmaf(-wy, wex.y, extra[c].x));
-                            extra[c].y = fmaf(wx, wex.y, fmaf(wy, wex.x, extra[c].y));
+                            if (need_x) {
+                                extra[c].x = fmaf(wx, wex.x, fmaf(-wy, wex.y, extra[c].x));
+                                extra[c].y = fmaf(wx, wex.y, fmaf(wy, wex.x, extra[c].y));
+                            }
                         }
                         const uint32_t hi = bf16x2_bits(wx, wy);
                         const uint32_t lo = bf16x2_bits(wx - __uint_as_float(hi << 16), wy - __uint_as_float(hi & 0xffff0000u));
