@@ -6,13 +6,19 @@ visual-encoder grid, then luvc_spu_prune on the LLM-side hidden states of the me
 (configurations 2 and 3; the seeded projection between the two stands in for the projector and
 is not timed), or the two stress operators back to back (configuration 4).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|4] [--cutoff C] [--impl reference]
+                    [--no-per-config] [--no-cpu-baseline] [--oim-matching bipartite]
 
 Prints ONE JSON line (rank 0).  `value` is vision tokens per second with inputs resident in HBM,
 timed with CUDA events on the launching stream; `e2e` is the same metric through the host-buffer
 C-ABI entry points (host->device and device->host copies inside the timed region); `roofline`
-describes the dominant kernel (the OIM merge-step kernel) against the measured HBM copy rate;
-`cpu_baseline` is the CPU oracle timed on this machine's host cores on a bounded sample.
+describes the dominant kernel (the OIM chain kernel) against the measured HBM copy rate read from
+MEASURED_PEAKS.json at run time: `achieved` by the algorithmic bytes of a launch, `dram` by the DRAM
+bytes of the ncu capture recorded in profiles/ncu_traffic.json (null once the kernel's source has
+changed since), `floor` by input-once-plus-outputs-once; `per_config` repeats the device-timed
+numbers for configs[2], [3] and [4] with the OIM and SPU roofline objects and, for configs[4], all
+nine (cutoff, keep) pairs of the prune; `cpu_baseline` is the CPU oracle timed on this machine's host
+cores on a bounded sample (plus the single-thread time of configs[0]).
 """
 from __future__ import annotations
 
@@ -64,6 +70,9 @@ def parse_args():
     ap.add_argument("--oim-matching", default="adjacent", choices=["adjacent", "bipartite"],
                     help="bipartite: time the full-line matching variant of OIM instead (device-timed numbers only: "
                          "no end-to-end and no CPU-baseline leg)")
+    ap.add_argument("--cutoff", type=float, default=0.0,
+                    help="pass band of the prune as a fraction of the band (0 = the workload's own: 0.05 for "
+                         "configs[4], the default 0.125 otherwise)")
     ap.add_argument("--cpu-sample", type=int, default=0, help="units of the batch the CPU oracle is timed on (0 = auto)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true",
@@ -74,7 +83,7 @@ def parse_args():
 # ----------------------------------------------------------------------------- workloads
 
 
-def workload_spec(k):
+def workload_spec(k, cutoff=0.0):
     import luvc_inputs as gi
 
     c = gi.CONFIGS[k]
@@ -87,6 +96,8 @@ def workload_spec(k):
         T = c["target"]
         spec["spu"] = (c["B"] // c.get("frames", 1), T * c.get("frames", 1), c["D_llm"])
         spec["tokens"] = c["B"] * c["H"] * c["W"]
+    if cutoff > 0:
+        spec["cutoff"] = cutoff
     return spec
 
 
@@ -265,7 +276,7 @@ def run_reference(args):
     import luvc_inputs as gi
     import oracle
 
-    spec = workload_spec(args.workload)
+    spec = workload_spec(args.workload, args.cutoff)
     k = spec["id"]
     sample = args.cpu_sample or max(1, auto_cpu_sample(spec) // 4)
     B = spec["oim"][0]
@@ -462,7 +473,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
 
-    spec = workload_spec(args.workload)
+    spec = workload_spec(args.workload, args.cutoff)
     k = spec["id"]
     B, H, W, D = spec["oim"]
     sb, sn, sd = spec["spu"]
