@@ -55,10 +55,12 @@ struct FwdArgs {
     int n_ctiles, n_slices, n_items;
     int static_tab;           // 1: the table of e^{-2 pi i q k2 / Q} for all q is built once per CTA (one slice only)
     const unsigned char* f_img;   // both parts of the stage-1 matrix as they sit in shared memory (built once per call)
+    int n_stages;             // input stages in shared memory: 3 where they fit (copies run two tiles ahead), else 2
 };
 
-// barriers: 0,1 stage full | 2,3 accumulator full | 4,5 accumulator empty | 6,7 table ready
-enum { kBarFull = 0, kBarAccFull = 2, kBarAccEmpty = 4, kBarTab = 6, kBarImg = 8, kBars = 9 };
+// barriers: 0-2 stage full | 3,4 accumulator full | 5,6 accumulator empty | 7,8 table ready | 9 operand image landed
+enum { kBarFull = 0, kBarAccFull = 3, kBarAccEmpty = 5, kBarTab = 7, kBarImg = 9, kBars = 10 };
+constexpr int kMaxStages = 3;
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, int parity, volatile int* s_fail, int* status) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -175,6 +177,48 @@ __device__ __forceinline__ void stage2_tile(uint32_t taddr, int nq, const float4
     }
 }
 
+// The same for few bins per thread (KB <= 4): instead of rotating every stage-1 value by e^{-2 pi i q k1 / N} and
+// then multiplying it by a table entry per bin, the thread carries the whole factor g[t] = e^{-2 pi i q k_t / N} of
+// each of its bins from token to token (one complex product per bin and token, whatever the number of channels)
+// and a value costs two packed FMAs per bin: y += g (own + i c other) = (g.x, g.y) own + (-g.y, g.x) c other.
+// On the odd lane of a pair g carries the factor -i (see stage2_tile).
+template <int KB, int CH, int NB>
+__device__ __forceinline__ void stage2_tile_few(uint32_t taddr, int nq, float2 (&g)[KB], const float2 (&gstep)[KB], float cg,
+                                                bool warp_active, uint32_t acc_empty_bar, int lane, float2 (&y)[KB][2 * CH]) {
+    constexpr int C = 8 * CH, W = 2 * CH;
+    uint32_t v[W], vn[W];
+    tmem_load<W>(taddr, vn);
+    for (int ql = 0; ql < nq; ++ql) {
+        tmem_ld_wait_for(vn);
+#pragma unroll
+        for (int c = 0; c < W; ++c) v[c] = vn[c];
+        if (ql + 1 < nq) {
+            tmem_load<W>(taddr + (uint32_t)((ql + 1) * C), vn);   // in flight under this token's arithmetic
+        } else {                     // this warp has read all it needs of the buffer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar);
+        }
+        if (!warp_active) continue;
+        float2 gp[NB], gq[NB];
+#pragma unroll
+        for (int t = 0; t < NB; ++t) { gp[t] = g[t]; gq[t] = make_float2(-g[t].y, g[t].x); }
+#pragma unroll
+        for (int c = 0; c < W; ++c) {
+            const float own = __uint_as_float(v[c]);
+            const float other = cg * __shfl_xor_sync(0xffffffffu, own, 1);
+            const float2 oo = make_float2(own, own), cc = make_float2(other, other);
+#pragma unroll
+            for (int t = 0; t < NB; ++t) {
+                y[t][c] = __ffma2_rn(gp[t], oo, y[t][c]);
+                y[t][c] = __ffma2_rn(gq[t], cc, y[t][c]);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < KB; ++t) g[t] = cmul(g[t], gstep[t]);
+    }
+}
+
 // KB: band bins per frequency class held by a thread; CH: channels per thread (C = 8 CH per block).
 template <int KB, int CH>
 __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_constant__ CUtensorMap tmap, const FwdArgs a) {
@@ -199,13 +243,14 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     unsigned char* s_fhi = smem;
     unsigned char* s_flo = smem + f_bytes;
     unsigned char* s_x = smem + 2 * f_bytes;
-    float4* s_tab = reinterpret_cast<float4*>(s_x + 2 * stage_bytes);   // [Q * KB] or [2][QT * KB]
+    const int nst = a.n_stages;
+    float4* s_tab = reinterpret_cast<float4*>(s_x + nst * stage_bytes);   // [Q * KB] or [2][QT * KB]
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     if (tid == 0) {
+        for (int s = 0; s < kMaxStages; ++s) mbar_init(bar(kBarFull + s), 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(kBarFull + s), 1);
             mbar_init(bar(kBarAccFull + s), 1);
             mbar_init(bar(kBarAccEmpty + s), kEpiWarps);
             mbar_init(bar(kBarTab + s), kEpiWarps);
@@ -221,7 +266,8 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
         mbar_arrive_expect_tx(bar(kBarImg), (uint32_t)(2 * f_bytes));
         bulk_load(smem_u32(s_fhi), a.f_img, (uint32_t)(2 * f_bytes), bar(kBarImg));
     }
-    if (a.static_tab)
+    constexpr bool kFew = KB <= 4;               // few bins: the per-bin factors are carried in registers, no table
+    if (!kFew && a.static_tab)
         for (int e = tid; e < Q * KB; e += kThreads) {
             const int q = e / KB, k2 = e - q * KB;
             s_tab[e] = root_neg_packed(((unsigned)q * (unsigned)k2) % (unsigned)Q, Q);
@@ -250,11 +296,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     const uint64_t b0 = LAYOUT ? make_desc_layout(xs, P * ROWB, 8 * ROWB, LAYOUT) : make_desc(xs, 128, P * 16);
 
     // producer steps (one thread only)
-    auto issue_tma = [&](int v) {           // tile v of this CTA's sequence of tiles -> stage v & 1
+    auto issue_tma = [&](int v) {           // tile v of this CTA's sequence of tiles -> stage v % nst
         const int item = blockIdx.x + (v / tiles_per_item) * gridDim.x, tile = v % tiles_per_item;
         const int rest = item / a.n_slices;
         const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
-        const int c0 = ctile * item_channels, buf = v & 1;
+        const int c0 = ctile * item_channels, buf = v % nst;
         // boxes that reach past Q or D are filled with zeros there and still count in full
         if (elect_one()) {
             mbar_arrive_expect_tx(bar(kBarFull + buf), (uint32_t)stage_bytes);
@@ -264,15 +310,15 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
         __syncwarp();
     };
     auto issue_mma = [&](int v) -> bool {   // needs tile v in its stage and accumulator v & 1 drained
-        const int buf = v & 1;
-        if (!__all_sync(0xffffffffu, wait_bar(bar(kBarFull + buf), (v >> 1) & 1, fail, a.status))) return false;
+        const int buf = v & 1, st = v % nst;
+        if (!__all_sync(0xffffffffu, wait_bar(bar(kBarFull + st), (v / nst) & 1, fail, a.status))) return false;
         if (v >= 2 && !__all_sync(0xffffffffu, wait_bar(bar(kBarAccEmpty + buf), ((v - 2) >> 1) & 1, fail, a.status))) return false;
         tc_fence_after();
         const uint32_t acc = tmem + (uint32_t)(buf * kNmma);
         if (elect_one()) {
             uint64_t ah = a_hi0, al = a_lo0;             // descriptors advance by adding to the address field
             for (int jb = 0; jb < a.nblk; ++jb) {        // K rows of channel block jb
-                uint64_t bd = b0 + (uint64_t)((buf * stage_bytes + jb * blk_bytes) >> 4);
+                uint64_t bd = b0 + (uint64_t)((st * stage_bytes + jb * blk_bytes) >> 4);
                 for (int kl = 0; kl < P / 16; ++kl) {
                     umma_bf16(acc, ah, bd, idesc, (jb | kl) ? 1u : 0u);
                     umma_bf16(acc, al, bd, idesc, 1u);
@@ -289,8 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     const int warp_u = __shfl_sync(0xffffffffu, warp, 0);
     const bool producer = warp_u == kProducer / 32;
     if (producer && total_tiles > 0) {
-        issue_tma(0);
-        if (total_tiles > 1) issue_tma(1);
+        for (int v = 0; v < nst && v < total_tiles; ++v) issue_tma(v);
         issue_mma(0);
     }
     __syncwarp();
@@ -327,11 +372,17 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                 for (int c = 0; c < 2 * CH; ++c) y[t][c] = make_float2(0.f, 0.f);
 
             float2 rot = make_float2(1.f, 0.f);
+            float2 gk[KB], gstep[KB];                    // few bins: e^{-2 pi i q k_t / N} and its step from token to token
+#pragma unroll
+            for (int t = 0; t < KB; ++t) {
+                gk[t] = make_float2(1.f, 0.f);
+                gstep[t] = kFew ? root_neg((unsigned)((kf + P * (k2_lo + t)) % N), N) : make_float2(1.f, 0.f);
+            }
             for (int tile = 0; tile < tiles_per_item; ++tile, ++u) {
                 const int q0 = tile * QT, nq = min(QT, Q - q0), buf = u & 1, par = (u >> 1) & 1;
                 // table of e^{-2 pi i q k2 / Q} for the tile's tokens and the slice's k2
                 const float4* tab = s_tab + q0 * KB;
-                if (!a.static_tab) {
+                if (!kFew && !a.static_tab) {
                     float4* tw = s_tab + buf * (QT * KB);
                     for (int e = tid; e < QT * KB; e += kEpiThreads) {
                         const int ql = e / KB, k2 = k2_lo + (e - ql * KB);
@@ -346,19 +397,35 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
                 ok = __all_sync(0xffffffffu, ok);
                 if (producer && ok) {
                     // the MMAs of tile u are done: refill their stage, and start tile u + 1
-                    if (u + 2 < total_tiles) issue_tma(u + 2);
+                    if (u + nst < total_tiles) issue_tma(u + nst);
                     if (u + 1 < total_tiles) ok = issue_mma(u + 1);
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 if ((tile & 15) == 0) {     // exact restart of e^{-2 pi i q k / N}; in between it is carried along
-                    rot = root_neg(((unsigned)q0 * (unsigned)kf) % (unsigned)N, N);   // q0 kf < Q P = N
-                    if (odd && !special) rot = make_float2(rot.y, -rot.x);           // times -i (see stage2_tile)
+                    if constexpr (kFew) {
+#pragma unroll
+                        for (int t = 0; t < KB; ++t) {
+                            const unsigned long long m = (unsigned long long)q0 * (unsigned)(kf + P * (k2_lo + t));
+                            gk[t] = root_neg((unsigned)(m % (unsigned)N), N);
+                            if (odd && !special) gk[t] = make_float2(gk[t].y, -gk[t].x);      // times -i (see stage2_tile)
+                        }
+                    } else {
+                        rot = root_neg(((unsigned)q0 * (unsigned)kf) % (unsigned)N, N);   // q0 kf < Q P = N
+                        if (odd && !special) rot = make_float2(rot.y, -rot.x);           // times -i (see stage2_tile)
+                    }
                 }
                 const uint32_t taddr = lane_addr + (uint32_t)(buf * kNmma + grp * 2 * CH);
                 const uint32_t eb = bar(kBarAccEmpty + buf);
-                if (nb_w == KB)
+                if constexpr (kFew) {
+                    if (nb_w == KB)
+                        stage2_tile_few<KB, CH, KB>(taddr, nq, gk, gstep, cg, warp_active, eb, lane, y);
+                    else if (nb_w == KB - 1 || KB == 2)
+                        stage2_tile_few<KB, CH, (KB > 1 ? KB - 1 : 1)>(taddr, nq, gk, gstep, cg, warp_active, eb, lane, y);
+                    else
+                        stage2_tile_few<KB, CH, (KB >= 4 ? KB / 2 : KB)>(taddr, nq, gk, gstep, cg, warp_active, eb, lane, y);
+                } else if (nb_w == KB)
                     stage2_tile<KB, CH, KB>(taddr, nq, tab, rot, step, cg, warp_active, eb, lane, y);
                 else if (nb_w == KB - 1 || KB == 2)
                     stage2_tile<KB, CH, (KB > 1 ? KB - 1 : 1)>(taddr, nq, tab, rot, step, cg, warp_active, eb, lane, y);
@@ -464,9 +531,10 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 template <int KB, int CH>
-cudaError_t launch_fwd2(const FwdArgs& a, const SpuFwd2Plan& pl, cudaStream_t stream) {
+cudaError_t launch_fwd2(const FwdArgs& a_in, const SpuFwd2Plan& pl, cudaStream_t stream) {
     constexpr int C = 8 * CH, QT = kNmma / C;
-    const int KT = a.nblk * a.P;
+    const int KT = a_in.nblk * a_in.P;
+    FwdArgs a = a_in;
     // the tokens of one sequence as [q][p][channel]: token p Q + q sits P-strided in memory
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
@@ -483,7 +551,9 @@ cudaError_t launch_fwd2(const FwdArgs& a, const SpuFwd2Plan& pl, cudaStream_t st
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
     const size_t tab_bytes = a.static_tab ? (size_t)a.Q * KB * sizeof(float4) : (size_t)2 * QT * KB * sizeof(float4);
-    const size_t smem = 1024 + (size_t)2 * KT * 256 + (size_t)2 * kNmma * KT * 2 + tab_bytes;
+    const size_t fixed = 1024 + (size_t)2 * KT * 256 + tab_bytes, stage = (size_t)kNmma * KT * 2;
+    a.n_stages = fixed + kMaxStages * stage <= (size_t)226 * 1024 ? kMaxStages : 2;
+    const size_t smem = fixed + a.n_stages * stage;
     static int sms = 0;
     if (!sms) {
         int dev = 0;

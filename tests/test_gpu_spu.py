@@ -56,17 +56,20 @@ def test_small_sequences_match_the_oracle(luvc, oracle_mod, dtype, B, N, D, keep
     (2, 112, 40, 30, 0.5),      # N = 16 x 7: eight channel blocks on the diagonal of the stage-1 operand
     (1, 592, 24, 100, 1.0),     # N = 16 x 37, full band: two bin slices forward, dense inverse
     (2, 592, 16, 50, 0.3),      # same N, narrower band: two-stage inverse with 9 bins per row
-    (1, 2048, 72, 500, 1.0),    # P = 128, sigma = N/2: 9 bins per class, inverse on the tokens themselves
+    (1, 2048, 72, 500, 1.0),    # P = 128, sigma = N/2: 9 bins per class, inverse on the tokens themselves (CUDA-core second stages)
     (2, 2048, 40, 300, 0.5),    # inverse not coarse (4 sigma + 2 > 3N/4)
-    (1, 4096, 16, 1000, 0.9),   # 17 bins per class, one channel per thread
+    (1, 4096, 16, 1000, 0.9),   # 15 bins per class: wide forward geometry, inverse with 32 points per channel, four K steps
     (2, 1296, 136, 324, 0.125), # P = 48, Q = 27: ragged last tile, partial channel block
     (1, 2592, 264, 648, 0.05),  # P = 96
     (3, 768, 8, 77, 0.02),      # sigma smaller than P: most rows hold no bin
     (2, 1024, 48, 100, 0.3),    # N = 128 x 8: both stages on the tensor cores, two bins per class
     (1, 2048, 24, 300, 0.4),    # four bins per class (the narrow-band variant's limit), partial channel tile
     (2, 1152, 72, 200, 0.25),   # Q = 9: ragged last tile of tokens
-    (1, 4096, 40, 500, 1.0),    # seventeen bins per class: two slices of the wide-band variant
+    (1, 4096, 40, 500, 1.0),    # seventeen bins per class on a short sequence (CUDA-core second stages)
     (1, 16384, 24, 1638, 0.05), # the stress length: Q = 128, 32 tiles per item
+    (1, 16384, 16, 1000, 0.2),  # 13 bins per class, 52 points per channel: the largest inverse geometry without a 17th bin
+    (1, 8192, 64, 500, 0.2),    # 7 bins per class: two K steps, 26 points per channel
+    (2, 4096, 40, 400, 0.6),    # 10 bins per class, a last work item of 8 channels
 ])
 def test_two_stage_paths_match_the_oracle(luvc, oracle_mod, B, N, D, keep, cutoff):
     g = torch.Generator().manual_seed(N * 7 + D)
