@@ -161,6 +161,60 @@ __device__ __forceinline__ void stage2_tile(const float2 (&y)[KB][W], const floa
     }
 }
 
+// The same for few bins per lane (KB <= 4): the lane carries g[t] = e^{2 pi i jj k_t / L} of each of its bins from
+// point to point (k_t = its frequency + P t; times i on the odd lane of a pair, so that its own share of G is the real
+// part of C = sum_t Y_t g[t] and the partner's share the imaginary part), which replaces both the table of
+// e^{2 pi i k2 jj / J} and the rotation by e^{2 pi i k1 jj / L}.  G = Re C + gc (partner's Im C).
+template <int KB, int W, int NB>
+__device__ __forceinline__ void stage2_tile_few(const float2 (&y)[KB][W], float2 (&g)[KB], const float2 (&gstep)[KB], int jj0, int J,
+                                                float gc, unsigned char* b_hi, unsigned char* b_lo, int sbo, int row, int col0) {
+    constexpr int C = 4 * W, TJ = kNcol / C;
+    constexpr int HV = W >= 8 ? 8 : W;        // bf16 values per store
+#pragma unroll 1
+    for (int jl = 0; jl < TJ; ++jl) {
+        const int jj = jj0 + jl;
+        float gv[W];
+        if (jj < J) {
+            float2 gx[NB], gy[NB];
+#pragma unroll
+            for (int t = 0; t < NB; ++t) { gx[t] = make_float2(g[t].x, g[t].x); gy[t] = make_float2(g[t].y, g[t].y); }
+#pragma unroll
+            for (int c = 0; c < W; ++c) {
+                float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int t = 0; t < NB; ++t) {
+                    sa = __ffma2_rn(gx[t], y[t][c], sa);
+                    sb = __ffma2_rn(gy[t], y[t][c], sb);
+                }
+                const float cx = sa.x - sb.y, cy = sa.y + sb.x;
+                gv[c] = fmaf(gc, __shfl_xor_sync(0xffffffffu, cy, 1), cx);
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < W; ++c) gv[c] = 0.f;
+        }
+#pragma unroll
+        for (int t = 0; t < KB; ++t) g[t] = cmul(g[t], gstep[t]);
+        if (row < 0) continue;                 // a lane past the rows in use only takes part in the exchange
+        const int n = jl * C + col0;
+        const int off = (n >> 3) * sbo + (n & 7) * 2 + (row >> 3) * 128 + (row & 7) * 16;
+#pragma unroll
+        for (int h = 0; h < W / HV; ++h) {
+            uint32_t hv[HV / 2], lv[HV / 2];
+#pragma unroll
+            for (int c = 0; c < HV; c += 2) {
+                const float x0 = gv[h * HV + c], x1 = gv[h * HV + c + 1];
+                const __nv_bfloat16 a0 = __float2bfloat16_rn(x0), a1 = __float2bfloat16_rn(x1);
+                hv[c / 2] = pack_bf16(a0, a1);
+                lv[c / 2] = pack_bf16(__float2bfloat16_rn(x0 - __bfloat162float(a0)),
+                                      __float2bfloat16_rn(x1 - __bfloat162float(a1)));
+            }
+            store_bf16<HV>(b_hi + off + h * sbo, hv);
+            store_bf16<HV>(b_lo + off + h * sbo, lv);
+        }
+    }
+}
+
 // KB: band bins per lane; W: channels per thread (C = 4 W per channel block, TJ = 64 / C points per tile).
 template <int KB, int W>
 __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) {
@@ -226,6 +280,13 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     const int tiles_per_item = (J + TJ - 1) / TJ;
     const int item_channels = a.nblk * C;
     const float2 step = root_pos((unsigned)kf % (unsigned)L, L);
+    constexpr bool kFew = KB <= 4;               // few bins: the per-bin factors are carried in registers
+    float2 gk[KB], gstep[KB];
+#pragma unroll
+    for (int q = 0; q < KB; ++q) {
+        gk[q] = make_float2(1.f, 0.f);
+        gstep[q] = kFew ? root_pos((unsigned)((kf + P * q) % L), L) : make_float2(1.f, 0.f);
+    }
     const uint32_t idesc = make_idesc_bf16(128, kNcol, false, true);
     const uint64_t a_hi0 = make_desc(smem_u32(s_fhi), 2048, 128), a_lo0 = make_desc(smem_u32(s_flo), 2048, 128);
     const uint64_t b_d0 = make_desc(smem_u32(s_b), 128, sbo);
@@ -303,7 +364,25 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
         for (int tile = 0; tile < tiles_per_item; ++tile, ++t) {
             const int jj0 = tile * TJ;
             // buffer t & 1 of B is free: every warp has seen the MMAs of tile t - 2 finish (below, one tile ago)
-            if (warp_active) {
+            if (kFew && warp_active) {
+                if ((tile & 15) == 0) {         // exact restart of the carried factors; in between they are advanced point by point
+#pragma unroll
+                    for (int q = 0; q < KB; ++q) {
+                        const unsigned long long m = (unsigned long long)jj0 * (unsigned)(kf + P * q);
+                        gk[q] = root_pos((unsigned)(m % (unsigned)L), L);
+                        if (odd && !special) gk[q] = make_float2(-gk[q].y, gk[q].x);      // times i
+                    }
+                }
+                unsigned char* bh = s_b + (t & 1) * b_buf;
+                unsigned char* bl = bh + b_part;
+                const int col0 = grp * W;
+                if (nb_w == KB)
+                    stage2_tile_few<KB, W, KB>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
+                else if (nb_w == KB - 1 || KB == 2)
+                    stage2_tile_few<KB, W, (KB > 1 ? KB - 1 : 1)>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
+                else
+                    stage2_tile_few<KB, W, (KB >= 4 ? KB / 2 : KB)>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
+            } else if (warp_active) {
                 const float2 rot = root_pos(((unsigned)kf * (unsigned)jj0) % (unsigned)L, L);   // kf jj0 < P J = L
                 unsigned char* bh = s_b + (t & 1) * b_buf;
                 unsigned char* bl = bh + b_part;
