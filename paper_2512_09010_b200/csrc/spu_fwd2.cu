@@ -583,6 +583,9 @@ SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma) {
         const int slices = (nk2 + kbs[v] - 1) / kbs[v];
         if (best < 0 || slices < pl.slices) { best = v; pl.slices = slices; }
     }
+    // A small batch in wide channel tiles leaves most SMs without a work item: with up to two bins per class the
+    // four-bin variant does the same arithmetic on tiles of half the channels, which doubles the items.
+    if (best == 0 && (long long)B * ((D + 64 * pl.nblk - 1) / (64 * pl.nblk)) * pl.slices <= 74) best = 1;
     pl.KB = kbs[best];
     pl.CH = chs[best];
     const int C = 8 * pl.CH * pl.nblk;                 // channels of one work item

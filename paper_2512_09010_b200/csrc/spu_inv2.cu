@@ -506,7 +506,9 @@ SpuInv2Plan spu_inv2_plan(int B, int N, int D, int sigma) {
     pl.J = pl.coarse ? (int)jc : pl.Q;
     pl.L = pl.P * pl.J;
     const int nk2 = sigma / pl.P + 1;
-    if (nk2 <= 2) { pl.KB = 2; pl.CHT = 16; }
+    // (up to two bins per class: the four-bin variant when the wide channel tiles of the two-bin variant would leave
+    // most SMs without a work item)
+    if (nk2 <= 2 && (long long)B * ((D + 64 * pl.nblk - 1) / (64 * pl.nblk)) > 74) { pl.KB = 2; pl.CHT = 16; }
     else if (nk2 <= 4) { pl.KB = 4; pl.CHT = 8; }
     else if (nk2 <= 9) { pl.KB = 9; pl.CHT = 4; }
     else if (nk2 <= 17) { pl.KB = 17; pl.CHT = 2; }
