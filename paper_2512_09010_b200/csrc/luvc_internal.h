@@ -133,8 +133,9 @@ int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, 
 struct SpuFwd3Plan {
     int ok;             // 0: use the two-stage kernel of spu_fwd2.cu (or the dense contraction)
     int Q;
-    int wide;           // 0: up to 4 bins per frequency class, 16 channels per item; 1: up to 16, 8 channels
-    int slices;         // passes over the input, each covering 4 / 16 values of k2
+    int geo;            // bins per frequency class and channels per item: 0: up to 4 x 32; 1: up to 8 x 16; 2: up to 16 x 8
+    int wide;           // geo != 0
+    int slices;         // passes over the input, each covering 4 / 8 / 16 values of k2
     int extra_k2;       // > 0: this one further value of k2 is kept on the CUDA cores (no second pass for it)
     int C, n_ctiles, n_items;
 };

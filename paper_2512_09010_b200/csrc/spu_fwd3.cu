@@ -61,6 +61,7 @@ struct Fwd3Args {
     int B, N, D, Q, sigma, ks_out;
     int n_ctiles, n_slices, n_items;
     const unsigned char* img; // stage-1 matrix, stage-2 matrices and root tables in their shared-memory layouts (built once per call)
+    int extra_in_op;          // 1: that extra bin goes into the operand form (one more K step) instead of yx
     int extra_k2;             // > 0: one more value of k2 (= K2MAX) reaches into the band, for a few lanes only; those
                               // bins are accumulated on the CUDA cores instead of costing a second pass over the input
 };
@@ -478,40 +479,61 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                     }
                     return make_uint4(w[0], w[1], w[2], w[3]);
                 };
+                // All of this thread's result columns at once (UT N2 = 64 in every geometry), then the accumulators are
+                // free for the next work item while the values are scaled, split and stored.
+                static_assert(G::UT * N2 == 64, "a converter thread owns 64 result columns");
+                uint32_t o[4][16];
+#pragma unroll
+                for (int h = 0; h < 4; ++h) tmem_ld16(lane_addr + (uint32_t)(G::OUT0 + g * 64 + h * 16), o[h]);
+#pragma unroll
+                for (int h = 0; h < 4; ++h) tmem_ld_wait_for(o[h]);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarOutEmpty));
                 if constexpr (QPU == 2) {
                     // unit h: channels 2h, 2h+1 of the thread; column = cc * 8 + k2 * 2 + ri: one K step of four bins
 #pragma unroll
-                    for (int h = 0; h < (G::UT * N2) / 16; ++h) {
-                        uint32_t o[16];
-                        tmem_ld16(lane_addr + (uint32_t)(G::OUT0 + g * G::UT * N2 + h * 16), o);
-                        tmem_ld_wait_for(o);
+                    for (int h = 0; h < 4; ++h) {
 #pragma unroll
                         for (int cc = 0; cc < 2; ++cc) {
                             if (ch0 + 2 * h + cc >= D) continue;
                             unsigned char* yc = yb + (size_t)(2 * h + cc) * chan_bytes;
-                            *reinterpret_cast<uint4*>(yc) = chunk(o + cc * 8, 0);
-                            *reinterpret_cast<uint4*>(yc + 2048) = chunk(o + cc * 8 + 4, 2);
+                            *reinterpret_cast<uint4*>(yc) = chunk(o[h] + cc * 8, 0);
+                            *reinterpret_cast<uint4*>(yc + 2048) = chunk(o[h] + cc * 8 + 4, 2);
                         }
                     }
                 } else {
-                    // channel cc of the thread: 32 columns, k2 * 2 + ri: K step s holds bins 4 s .. 4 s + 3
+                    // channel cc of the thread: N2 columns, k2 * 2 + ri: K step s holds bins 4 s .. 4 s + 3
+                    const int ks_held = min(a.ks_out, N2 / 8);       // K steps whose bins were accumulated in tensor memory
 #pragma unroll
                     for (int cc = 0; cc < W; ++cc) {
-                        for (int s2 = 0; s2 < a.ks_out; ++s2) {
-                            uint32_t o[8];
-                            tmem_ld8(lane_addr + (uint32_t)(G::OUT0 + g * G::UT * N2 + cc * N2 + s2 * 8), o);
-                            tmem_ld_wait_for(o);
-                            if (ch0 + cc >= D) continue;
+#pragma unroll
+                        for (int s2 = 0; s2 < N2 / 8; ++s2) {
+                            if (s2 >= ks_held || ch0 + cc >= D) continue;
+                            const int col = cc * N2 + s2 * 8;        // compile-time after unrolling
                             unsigned char* yc = yb + (size_t)cc * chan_bytes + (size_t)s2 * 4096;
-                            *reinterpret_cast<uint4*>(yc) = chunk(o, 4 * s2);
-                            *reinterpret_cast<uint4*>(yc + 2048) = chunk(o + 4, 4 * s2 + 2);
+                            *reinterpret_cast<uint4*>(yc) = chunk(o[col / 16] + (col % 16), 4 * s2);
+                            *reinterpret_cast<uint4*>(yc + 2048) = chunk(o[col / 16] + (col % 16) + 4, 4 * s2 + 2);
                         }
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarOutEmpty));
-                if (EXTRA) {
+                if (EXTRA && a.extra_in_op) {
+                    // the extra bin opens one more K step of the operand form: its first bin on the lanes that reach it,
+                    // zeros everywhere else
+                    const int k = kfe + kP * a.extra_k2;
+                    const bool in = k <= sigma;
+                    const float cr = in ? __ldg(a.scale + k) : 0.f, ci = in ? __ldg(a.scale + sigma + k) : 0.f;
+#pragma unroll
+                    for (int c = 0; c < W; ++c) {
+                        if (ch0 + c >= D) continue;
+                        const float re = cr * extra[c].x, im = ci * extra[c].y;
+                        const uint32_t hi = bf16x2_bits(re, im);
+                        const uint32_t lo = bf16x2_bits(re - __uint_as_float(hi << 16), im - __uint_as_float(hi & 0xffff0000u));
+                        unsigned char* yc = yb + (size_t)c * chan_bytes + (size_t)(a.extra_k2 / 4) * 4096;
+                        *reinterpret_cast<uint4*>(yc) = make_uint4(hi, lo, 0u, 0u);
+                        *reinterpret_cast<uint4*>(yc + 2048) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                } else if (EXTRA) {
                     const int k = kfe + kP * a.extra_k2;
                     if (k <= sigma && ch0 < D) {
                         const float cr = __ldg(a.scale + k), ci = __ldg(a.scale + sigma + k);
@@ -646,7 +668,9 @@ cudaError_t launch_fwd3(const Fwd3Args& a, cudaStream_t stream) {
 }
 
 using GeoNarrow = Geo<32, 16, 2, 1>;     // up to 4 bins per frequency class; 64-byte token rows keep TMA at full rate
-using GeoWide = Geo<8, 32, 4, 1>;        // up to 16 bins per frequency class (per slice), one operand slot
+using GeoMid = Geo<16, 16, 4, 1>;        // up to 8 bins per frequency class; 32-byte token rows
+using GeoWide = Geo<8, 32, 4, 1>;        // up to 16 bins per frequency class (per slice); 16-byte token rows cap the TMA feed
+                                         // near 1.5 TB/s, which is why the middle geometry exists
 
 }  // namespace
 
@@ -656,20 +680,23 @@ SpuFwd3Plan spu_fwd3_plan(int B, int N, int D, int sigma) {
     pl.Q = N / kP;
     if (pl.Q < 8 || pl.Q > 128) return pl;           // the stage-2 matrices of a whole sequence stay in shared memory
     const int nk2 = sigma / kP + 1;                  // values of k2 that reach into the band
-    pl.wide = nk2 > GeoNarrow::K2MAX ? 1 : 0;
-    const int k2max = pl.wide ? GeoWide::K2MAX : GeoNarrow::K2MAX;
+    // geometry: 0 narrow, 1 middle, 2 wide; one value of k2 more than the geometry holds is still one pass: the few lanes
+    // that reach it (k1 <= sigma - 128 k2max) keep that bin in registers
+    pl.geo = nk2 <= GeoNarrow::K2MAX ? 0 : (nk2 <= GeoMid::K2MAX + 1 ? 1 : 2);
+    pl.wide = pl.geo != 0;
+    const int k2max = pl.geo == 0 ? GeoNarrow::K2MAX : (pl.geo == 1 ? GeoMid::K2MAX : GeoWide::K2MAX);
     pl.slices = (nk2 + k2max - 1) / k2max;
     pl.extra_k2 = 0;
-    if (pl.wide && nk2 == k2max + 1) {               // one value of k2 too many for one pass: the few lanes that reach
-        pl.slices = 1;                               // it (k1 <= sigma - 128 k2max) keep that bin in registers
+    if (pl.geo != 0 && nk2 == k2max + 1) {
+        pl.slices = 1;
         pl.extra_k2 = k2max;
     }
-    pl.C = pl.wide ? GeoWide::C : GeoNarrow::C;
+    pl.C = pl.geo == 0 ? GeoNarrow::C : (pl.geo == 1 ? GeoMid::C : GeoWide::C);
     pl.n_ctiles = (D + pl.C - 1) / pl.C;
     const long long items = (long long)B * pl.n_ctiles * pl.slices;
     if (items > 0x7fffffffll) return pl;
     pl.n_items = (int)items;
-    const size_t smem = pl.wide ? fwd3_smem<GeoWide>(pl.Q) : fwd3_smem<GeoNarrow>(pl.Q);
+    const size_t smem = pl.geo == 0 ? fwd3_smem<GeoNarrow>(pl.Q) : (pl.geo == 1 ? fwd3_smem<GeoMid>(pl.Q) : fwd3_smem<GeoWide>(pl.Q));
     if (smem > 220 * 1024) return pl;
     pl.ok = 1;
     return pl;
@@ -681,13 +708,17 @@ int spu_fwd3_run(const void* hidden, void* yop, int ks_out, float* yx, const flo
     if (!pl.ok) return LUVC_ERR_INTERNAL;
     Fwd3Args a;
     a.x = reinterpret_cast<const __nv_bfloat16*>(hidden);
-    if (pl.slices != 1 || ks_out * 4 > (pl.wide ? GeoWide::K2MAX : GeoNarrow::K2MAX)) return LUVC_ERR_INTERNAL;
+    const int k2max = pl.geo == 0 ? GeoNarrow::K2MAX : (pl.geo == 1 ? GeoMid::K2MAX : GeoWide::K2MAX);
+    // the extra bin of the middle geometry becomes one more K step of the operand form; that of the wide one goes to yx
+    a.extra_in_op = (pl.extra_k2 && ks_out * 4 > k2max) ? 1 : 0;
+    if (pl.slices != 1 || ks_out * 4 > k2max + (a.extra_in_op ? 4 : 0)) return LUVC_ERR_INTERNAL;
     a.yop = static_cast<unsigned char*>(yop); a.yx = yx; a.ks_out = ks_out; a.scale = scale; a.status = status;
     a.B = B; a.N = N; a.D = D; a.Q = pl.Q; a.sigma = sigma;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
     a.extra_k2 = pl.extra_k2;
     a.img = static_cast<const unsigned char*>(img);
-    const cudaError_t err = !pl.wide ? launch_fwd3<GeoNarrow, false>(a, stream)
+    const cudaError_t err = pl.geo == 0 ? launch_fwd3<GeoNarrow, false>(a, stream)
+                            : pl.geo == 1 ? (pl.extra_k2 ? launch_fwd3<GeoMid, true>(a, stream) : launch_fwd3<GeoMid, false>(a, stream))
                             : pl.extra_k2 ? launch_fwd3<GeoWide, true>(a, stream) : launch_fwd3<GeoWide, false>(a, stream);
     count_launch(2);
     return err == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
