@@ -153,7 +153,7 @@ struct Geo {
                   "a tile is sixteen units, four per converter thread");
 };
 
-template <typename G, bool EXTRA>
+template <typename G, int EXTRA>          // EXTRA: 0 none; 1 the extra bin on the converters; 2 on the issuing warps (k1 = 0 only)
 __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_constant__ CUtensorMap tmap, const Fwd3Args a) {
     constexpr int C = G::C, N2 = G::N2, QPU = G::QPU, QT = G::QT, W = G::W;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -172,6 +172,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
     unsigned char* s_w = s_x + kStages * G::STAGE_BYTES;                // [n_groups][hi, lo][16 x N2] stage-2 matrices
     float2* s_root = reinterpret_cast<float2*>(s_w + (size_t)n_groups * 2 * G::W_BYTES);   // e^{-2 pi i m / Q}, m < Q
     float2* s_fine = s_root + ((Q + 1) & ~1);                                              // e^{-2 pi i m / N}, m < 128
+    uint32_t* s_dc = reinterpret_cast<uint32_t*>(s_fine + kP);                             // [4 groups][3][16] stage-1 values of k1 = 0
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -281,6 +282,12 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
         const int g = warp_u - kConvWarps - 1;
         const uint32_t idesc2 = make_idesc_bf16(128, N2, false, false);
         const uint64_t w0 = make_desc(smem_u32(s_w), N2 * 16, 128);
+        // the extra bin of k1 = 0 (extra_dc): lane i < 16 takes value i = ql W + c of a tile, token q = tile QT + ql
+        constexpr bool dc = EXTRA == 2;
+        const int dc_ql = (lane & 15) / W, dc_c = (lane & 15) % W;
+        const int dc_step = dc ? (QT * a.extra_k2) % Q : 0;
+        int dc_angle = 0;
+        float2 dc_acc = make_float2(0.f, 0.f);
         bool ok = true;
         for (int u = 0; u < total_tiles && ok; ++u) {
             const int tile = u % tiles_per_item, item_seq = u / tiles_per_item;
@@ -313,6 +320,46 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                 if (tile == tiles_per_item - 1) umma_commit(bar(kBarOutFull));
             }
             __syncwarp();
+            if constexpr (dc) {
+                if (tile == 0) {
+                    dc_angle = (dc_ql * a.extra_k2) % Q;
+                    dc_acc = make_float2(0.f, 0.f);
+                }
+                if (lane < 16) {
+                    const float val = __uint_as_float(s_dc[(g * 3 + u % 3) * 16 + lane]);
+                    const float2 wex = s_root[dc_angle];             // e^{-2 pi i q extra_k2 / Q}
+                    dc_acc.x = fmaf(val, wex.x, dc_acc.x);
+                    dc_acc.y = fmaf(val, wex.y, dc_acc.y);
+                }
+                dc_angle += dc_step;
+                if (dc_angle >= Q) dc_angle -= Q;
+                if (tile == tiles_per_item - 1) {
+                    // sum over the tokens of a tile, then lane c holds channel c of this group
+                    float2 t = lane < 16 ? dc_acc : make_float2(0.f, 0.f);
+#pragma unroll
+                    for (int off = W; off < 16; off <<= 1) {
+                        t.x += __shfl_xor_sync(0xffffffffu, t.x, off);
+                        t.y += __shfl_xor_sync(0xffffffffu, t.y, off);
+                    }
+                    const int item = blockIdx.x + item_seq * gridDim.x, rest = item / a.n_slices;
+                    const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
+                    const int ch = ctile * C + g * W + lane;
+                    if (lane < W && ch < D) {
+                        const int k = kP * a.extra_k2;
+                        const float re = __ldg(a.scale + k) * t.x, im = __ldg(a.scale + sigma + k) * t.y;
+                        if (a.extra_in_op) {
+                            const uint32_t hi = bf16x2_bits(re, im);
+                            const uint32_t lo = bf16x2_bits(re - __uint_as_float(hi << 16), im - __uint_as_float(hi & 0xffff0000u));
+                            unsigned char* yc = a.yop + ((size_t)b * D + ch) * ((size_t)a.ks_out * 4096) + (size_t)(a.extra_k2 / 4) * 4096;
+                            *reinterpret_cast<uint4*>(yc) = make_uint4(hi, lo, 0u, 0u);                 // TMEM lane 0 = k1 = 0
+                            *reinterpret_cast<uint4*>(yc + 2048) = make_uint4(0u, 0u, 0u, 0u);
+                        } else {
+                            a.yx[(size_t)b * D + ch] = re;
+                            a.yx[(size_t)a.B * D + (size_t)b * D + ch] = im;
+                        }
+                    }
+                }
+            }
         }
     } else {
         // ------------------------------------------------------------------ converters
@@ -346,9 +393,9 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
             for (int c = 0; c < W; ++c) extra[c] = make_float2(0.f, 0.f);
             // only the warps with a lane that reaches that bin accumulate it; the angle q extra_k2 mod Q is carried
             // along in integers from token to token
-            const bool need_x = EXTRA && __any_sync(0xffffffffu, kfe + kP * a.extra_k2 <= sigma);
+            const bool need_x = EXTRA == 1 && __any_sync(0xffffffffu, kfe + kP * a.extra_k2 <= sigma);
             int x_angle = 0;
-            const int x_step = EXTRA ? a.extra_k2 % Q : 0;
+            const int x_step = EXTRA == 1 ? a.extra_k2 % Q : 0;
             // The TMEM round trips are long (a load or a store takes several hundred cycles), so the loop is
             // software-pipelined: the next tile's values are requested before this tile's arithmetic, and
             // a tile's stores are only waited for (and its units handed to the MMA warp) one tile later.
@@ -376,6 +423,20 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarAccEmpty + buf));  // the accumulator may be overwritten
+                if constexpr (EXTRA == 2) {
+                    // k1 = 0 (TMEM lane 0): its stage-1 values of this tile for the warp that forms the extra bin.  Three
+                    // buffers: the one of tile u - 3 was read before the MMAs of tile u - 2 were issued, and their
+                    // completion was waited for at the end of tile u - 1
+                    if (j == 0) {
+                        uint4* dst = reinterpret_cast<uint4*>(s_dc + (g * 3 + u % 3) * 16);
+#pragma unroll
+                        for (int i4 = 0; i4 < 4; ++i4) {
+                            const int i = i4 * 4;
+                            dst[i4] = make_uint4(v[i / W][i % W], v[(i + 1) / W][(i + 1) % W], v[(i + 2) / W][(i + 2) % W],
+                                                 v[(i + 3) / W][(i + 3) % W]);
+                        }
+                    }
+                }
                 if (tile + 1 < tiles_per_item) {                     // request the next tile's values
                     ok = wait_bar(bar(kBarAccFull + ((u + 1) & 1)), ((u + 1) >> 1) & 1, fail, a.status);
                     ok = __all_sync(0xffffffffu, ok);
@@ -403,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                     // B = rot * (own + i cg other):  Re = rot.x own - cg rot.y other,  Im = rot.y own + cg rot.x other
                     const float ox = -cg * rot.y, oy = cg * rot.x;
                     float2 wex = make_float2(0.f, 0.f);              // e^{-2 pi i q extra_k2 / Q} of this token
-                    if constexpr (EXTRA) {
+                    if constexpr (EXTRA == 1) {
                         if (need_x) {
                             wex = s_root[x_angle];
                             x_angle += x_step;
@@ -415,7 +476,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                         const float own = __uint_as_float(v[ql][c]);
                         const float other = __shfl_xor_sync(0xffffffffu, own, 1);
                         const float wx = fmaf(rot.x, own, ox * other), wy = fmaf(rot.y, own, oy * other);
-                        if constexpr (EXTRA) {
+                        if constexpr (EXTRA == 1) {
                             if (need_x) {
                                 extra[c].x = fmaf(wx, wex.x, fmaf(-wy, wex.y, extra[c].x));
                                 extra[c].y = fmaf(wx, wex.y, fmaf(wy, wex.x, extra[c].y));
@@ -517,7 +578,18 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                         }
                     }
                 }
-                if (EXTRA && a.extra_in_op) {
+                if (EXTRA == 2 && a.extra_in_op) {
+                    // one more K step of the operand form: zeros on every lane but TMEM lane 0, whose bin the issuing warp writes
+                    if (j != 0) {
+#pragma unroll
+                        for (int c = 0; c < W; ++c) {
+                            if (ch0 + c >= D) continue;
+                            unsigned char* yc = yb + (size_t)c * chan_bytes + (size_t)(a.extra_k2 / 4) * 4096;
+                            *reinterpret_cast<uint4*>(yc) = make_uint4(0u, 0u, 0u, 0u);
+                            *reinterpret_cast<uint4*>(yc + 2048) = make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
+                } else if (EXTRA == 1 && a.extra_in_op) {
                     // the extra bin opens one more K step of the operand form: its first bin on the lanes that reach it,
                     // zeros everywhere else
                     const int k = kfe + kP * a.extra_k2;
@@ -533,7 +605,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                         *reinterpret_cast<uint4*>(yc) = make_uint4(hi, lo, 0u, 0u);
                         *reinterpret_cast<uint4*>(yc + 2048) = make_uint4(0u, 0u, 0u, 0u);
                     }
-                } else if (EXTRA) {
+                } else if (EXTRA == 1) {
                     const int k = kfe + kP * a.extra_k2;
                     if (k <= sigma && ch0 < D) {
                         const float cr = __ldg(a.scale + k), ci = __ldg(a.scale + sigma + k);
@@ -630,10 +702,10 @@ EncodeTiledFn encode_tiled_fn() {
 template <typename G>
 size_t fwd3_smem(int Q) {
     const int tiles = (Q + G::QT - 1) / G::QT, groups = tiles * G::GQ;
-    return 1024 + 65536 + (size_t)kStages * G::STAGE_BYTES + (size_t)groups * 2 * G::W_BYTES + (size_t)(((Q + 1) & ~1) + kP) * sizeof(float2);
+    return 1024 + 65536 + (size_t)kStages * G::STAGE_BYTES + (size_t)groups * 2 * G::W_BYTES + (size_t)(((Q + 1) & ~1) + kP) * sizeof(float2) + 4 * 3 * 16 * sizeof(uint32_t);
 }
 
-template <typename G, bool EXTRA>
+template <typename G, int EXTRA>
 cudaError_t launch_fwd3(const Fwd3Args& a, cudaStream_t stream) {
     // the tokens of one sequence as [q][p][channel]: token p Q + q sits 128-strided in memory
     EncodeTiledFn encode = encode_tiled_fn();
@@ -716,10 +788,14 @@ int spu_fwd3_run(const void* hidden, void* yop, int ks_out, float* yx, const flo
     a.B = B; a.N = N; a.D = D; a.Q = pl.Q; a.sigma = sigma;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
     a.extra_k2 = pl.extra_k2;
+    // only k1 = 0 reaches the extra bin (sigma = 128 extra_k2): the stage-2 issuing warps form it from the lane-0 values
+    // the converters leave in shared memory; else the converter warps that reach it accumulate it
+    const int xm = !pl.extra_k2 ? 0 : (sigma == kP * pl.extra_k2 ? 2 : 1);
     a.img = static_cast<const unsigned char*>(img);
-    const cudaError_t err = pl.geo == 0 ? launch_fwd3<GeoNarrow, false>(a, stream)
-                            : pl.geo == 1 ? (pl.extra_k2 ? launch_fwd3<GeoMid, true>(a, stream) : launch_fwd3<GeoMid, false>(a, stream))
-                            : pl.extra_k2 ? launch_fwd3<GeoWide, true>(a, stream) : launch_fwd3<GeoWide, false>(a, stream);
+    cudaError_t err;
+    if (pl.geo == 0) err = launch_fwd3<GeoNarrow, 0>(a, stream);
+    else if (pl.geo == 1) err = xm == 0 ? launch_fwd3<GeoMid, 0>(a, stream) : (xm == 1 ? launch_fwd3<GeoMid, 1>(a, stream) : launch_fwd3<GeoMid, 2>(a, stream));
+    else err = xm == 0 ? launch_fwd3<GeoWide, 0>(a, stream) : (xm == 1 ? launch_fwd3<GeoWide, 1>(a, stream) : launch_fwd3<GeoWide, 2>(a, stream));
     count_launch(2);
     return err == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }
