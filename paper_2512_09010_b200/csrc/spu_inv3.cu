@@ -365,21 +365,18 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv3_kernel(const Inv3Args a)
                 unsigned char* bl = bh + G::B_PART;
                 const uint32_t d2 = lane_addr + (uint32_t)(G::D20 + dbuf * CT * N2);
                 // unit u = (channel ct of the tile, chunk grp + 4 m of its points): 8 columns of the stage-2' result
-                uint32_t v[8], vn[8];
-                tmem_ld8(d2 + (uint32_t)(grp * 8), vn);
+                uint32_t vb[2][8];                       // units alternate between the two: one in use, one in flight
+                tmem_ld8(d2 + (uint32_t)(grp * 8), vb[0]);
 #pragma unroll
                 for (int u = 0; u < G::UNITS; ++u) {
                     const int ct = u / G::MYCH, m = u % G::MYCH;
                     const int ch = grp + 4 * m;
                     const bool live = ch < G::NCH;       // the same for the whole warp
-                    if (live) {
-                        tmem_ld_wait_for(vn);
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) v[c] = vn[c];
-                    }
+                    uint32_t (&v)[8] = vb[u & 1];
+                    if (live) tmem_ld_wait_for(v);
                     if (u + 1 < G::UNITS) {
                         const int ct1 = (u + 1) / G::MYCH, m1 = (u + 1) % G::MYCH;
-                        if (grp + 4 * m1 < G::NCH) tmem_ld8(d2 + (uint32_t)(ct1 * N2 + (grp + 4 * m1) * 8), vn);
+                        if (grp + 4 * m1 < G::NCH) tmem_ld8(d2 + (uint32_t)(ct1 * N2 + (grp + 4 * m1) * 8), vb[(u + 1) & 1]);
                     }
                     if (!live) continue;
                     float g[4];
