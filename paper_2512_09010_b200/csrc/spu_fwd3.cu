@@ -605,18 +605,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
                         *reinterpret_cast<uint4*>(yc) = make_uint4(hi, lo, 0u, 0u);
                         *reinterpret_cast<uint4*>(yc + 2048) = make_uint4(0u, 0u, 0u, 0u);
                     }
-                } else if (EXTRA == 1) {
-                    const int k = kfe + kP * a.extra_k2;
-                    if (k <= sigma && ch0 < D) {
-                        const float cr = __ldg(a.scale + k), ci = __ldg(a.scale + sigma + k);
-                        float* yx = a.yx + (size_t)b * D + ch0;
-#pragma unroll
-                        for (int c = 0; c < W; ++c) {
-                            yx[c] = cr * extra[c].x;
-                            yx[(size_t)a.B * D + c] = ci * extra[c].y;
-                        }
-                    }
-                }
+                }                                        // (EXTRA == 1 always goes into the operand form)
             }
         }
     }
@@ -784,6 +773,7 @@ int spu_fwd3_run(const void* hidden, void* yop, int ks_out, float* yx, const flo
     // the extra bin of the middle geometry becomes one more K step of the operand form; that of the wide one goes to yx
     a.extra_in_op = (pl.extra_k2 && ks_out * 4 > k2max) ? 1 : 0;
     if (pl.slices != 1 || ks_out * 4 > k2max + (a.extra_in_op ? 4 : 0)) return LUVC_ERR_INTERNAL;
+    if (pl.extra_k2 && !a.extra_in_op && sigma != kP * pl.extra_k2) return LUVC_ERR_INTERNAL;   // yx holds the bin of k1 = 0 only
     a.yop = static_cast<unsigned char*>(yop); a.yx = yx; a.ks_out = ks_out; a.scale = scale; a.status = status;
     a.B = B; a.N = N; a.D = D; a.Q = pl.Q; a.sigma = sigma;
     a.n_ctiles = pl.n_ctiles; a.n_slices = pl.slices; a.n_items = pl.n_items;
@@ -795,7 +785,8 @@ int spu_fwd3_run(const void* hidden, void* yop, int ks_out, float* yx, const flo
     cudaError_t err;
     if (pl.geo == 0) err = launch_fwd3<GeoNarrow, 0>(a, stream);
     else if (pl.geo == 1) err = xm == 0 ? launch_fwd3<GeoMid, 0>(a, stream) : (xm == 1 ? launch_fwd3<GeoMid, 1>(a, stream) : launch_fwd3<GeoMid, 2>(a, stream));
-    else err = xm == 0 ? launch_fwd3<GeoWide, 0>(a, stream) : (xm == 1 ? launch_fwd3<GeoWide, 1>(a, stream) : launch_fwd3<GeoWide, 2>(a, stream));
+    else if (xm == 1) return LUVC_ERR_INTERNAL;      // a 17th bin that several frequency classes reach: not planned (spu_inv3_plan)
+    else err = xm == 0 ? launch_fwd3<GeoWide, 0>(a, stream) : launch_fwd3<GeoWide, 2>(a, stream);
     count_launch(2);
     return err == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
 }

@@ -530,6 +530,7 @@ SpuInv3Plan spu_inv3_plan(int B, int N, int D, int sigma) {
     const int nk2 = sigma / kP + 1;
     if (nk2 > 17) return pl;
     pl.extra = nk2 == 17 ? 1 : 0;
+    if (pl.extra && sigma != 16 * kP) return pl;     // the 17th bin is passed apart only as the single bin of k1 = 0
     pl.KS = ((pl.extra ? 16 : nk2) + 3) / 4;
     pl.JP = pl.J <= 16 ? 16 : (pl.J <= 40 ? 40 : (pl.J <= 72 ? 72 : 0));
     if (!pl.JP || (pl.extra && pl.JP != 72)) return pl;

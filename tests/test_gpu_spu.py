@@ -70,6 +70,8 @@ def test_small_sequences_match_the_oracle(luvc, oracle_mod, dtype, B, N, D, keep
     (1, 16384, 16, 1000, 0.2),  # 13 bins per class, 52 points per channel: the largest inverse geometry without a 17th bin
     (1, 8192, 64, 500, 0.2),    # 7 bins per class: two K steps, 26 points per channel
     (2, 4096, 40, 400, 0.6),    # 10 bins per class, a last work item of 8 channels
+    (1, 16384, 16, 1000, 0.13), # sigma = 1064: a 9th bin that several frequency classes reach
+    (1, 16384, 16, 1000, 0.2505),  # sigma = 2052: a 17th bin that several classes reach
 ])
 def test_two_stage_paths_match_the_oracle(luvc, oracle_mod, B, N, D, keep, cutoff):
     g = torch.Generator().manual_seed(N * 7 + D)
