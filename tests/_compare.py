@@ -96,13 +96,16 @@ def check_spu_selection(scores_ref, gpu_idx, keep):
     return bool(keep == N or tau_in > tau_out * (1 + DECISION_TOL))   # True: the kept set is unique
 
 
-def assert_scores_close(gpu_scores, ref, what="scores"):
+def assert_scores_close(gpu_scores, ref, what="scores", median_tol=1e-5):
     """Energies of Eq. 8 against the oracle's.  A score is the norm of a filtered signal (Eq. 7) that,
     next to a strong token, is a sum of large ringing terms of both signs: arithmetic that carries
     16-17 significant bits per operand (fp32 accumulation of bf16-pair products, 2^-17 = 7.6e-6)
     is exact relative to those TERMS, not to their sum, which can be a hundred times smaller in a
     null of the ringing.  So the bound is 1e-4 of the score itself plus 1e-5 of the largest score
-    within 32 tokens (circular); half of all scores must still agree to 1e-5 of themselves."""
+    within 32 tokens (circular); half of all scores must still agree to `median_tol` of themselves
+    (1e-5 on the factored paths; the dense band contractions, whose N-term sums are accumulated in tensor
+    memory with truncating fp32 additions, are given the full 1e-4 by the tests that reach them with long
+    sequences)."""
     ref = np.asarray(ref, dtype=np.float64)
     got = np.asarray(gpu_scores, dtype=np.float64)
     n = ref.shape[0]
@@ -114,4 +117,4 @@ def assert_scores_close(gpu_scores, ref, what="scores"):
     worst = float((err / (np.abs(ref) + 1e-30)).max()) if n else 0.0
     assert np.all(err <= bound), "%s: worst relative error %.3g" % (what, worst)
     if n >= 16:
-        assert np.median(err / (np.abs(ref) + 1e-30)) <= 1e-5, "%s: median relative error too large" % what
+        assert np.median(err / (np.abs(ref) + 1e-30)) <= median_tol, "%s: median relative error too large" % what

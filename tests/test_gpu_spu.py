@@ -22,7 +22,7 @@ def _run(luvc, x_dev, keep, cutoff, **kw):
     return idx.cpu().numpy(), hid, scores.cpu().numpy()
 
 
-def _check(luvc, oracle_mod, x, keep, cutoff, no_window=False, method="fft"):
+def _check(luvc, oracle_mod, x, keep, cutoff, no_window=False, method="fft", median_tol=1e-5):
     idx, hid, scores = _run(luvc, x.cuda(), keep, cutoff, no_window=no_window)
     xh = x.float().numpy()
     B, N, D = xh.shape
@@ -31,7 +31,7 @@ def _check(luvc, oracle_mod, x, keep, cutoff, no_window=False, method="fft"):
     unique = 0
     for b in range(B):
         ref = oracle_mod.spu_scores(xh[b], sigma, hamming=not no_window, method=method)
-        assert_scores_close(scores[b], ref, "sequence %d scores" % b)
+        assert_scores_close(scores[b], ref, "sequence %d scores" % b, median_tol=median_tol)
         if check_spu_selection(ref, idx[b], keep):
             np.testing.assert_array_equal(idx[b], oracle_mod.spu_select(ref, keep))
             unique += 1
@@ -80,6 +80,35 @@ def test_two_stage_paths_match_the_oracle(luvc, oracle_mod, B, N, D, keep, cutof
     n = torch.arange(N, dtype=torch.float32)[None, :, None]
     x = (x.float() + 2.0 * torch.cos(2 * np.pi * 3 * n / N + torch.arange(D)[None, None, :])).to(torch.bfloat16)
     _check(luvc, oracle_mod, x, keep, cutoff)
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_shapes_match_the_oracle(luvc, oracle_mod, seed):
+    # Twelve seeded shapes per seed over the three families of sequence lengths (128 Q: both stages on the tensor
+    # cores where the band allows; P Q with P a multiple of 16: CUDA-core second stages; anything else: dense
+    # contractions), any cutoff and any keep: whichever kernels the plan picks, scores and kept set follow the oracle.
+    import random
+    rng = random.Random(seed)
+    for it in range(12):
+        kind = rng.choice(["tc", "tc", "two", "any"])
+        if kind == "tc":
+            N = 128 * rng.randint(8, 128)
+        elif kind == "two":
+            N = 16 * rng.randint(1, 8) * rng.randint(2, 80)
+        else:
+            N = rng.randint(2, 3000)
+        D = 8 * rng.randint(1, 8)
+        B = rng.randint(1, 2)
+        cutoff = rng.choice([0.05, 0.125, 0.25, 0.5, 1.0, rng.uniform(0.01, 1.0), rng.uniform(0.01, 0.3)])
+        keep = rng.randint(1, N)
+        g = torch.Generator().manual_seed(seed * 7919 + it)
+        x = torch.randn((B, N, D), generator=g)
+        n = torch.arange(N, dtype=torch.float32)[None, :, None]
+        x = (x + 2.0 * torch.cos(2 * np.pi * 3 * n / N + torch.arange(D)[None, None, :])).to(torch.bfloat16)
+        # (the dense contractions accumulate N-term sums in tensor memory, whose fp32 additions truncate: a bias of
+        # about N / 16 * 2^-24 relative, 6e-5 at 16384 tokens, inside the 1e-4 bound but above the factored paths' 1e-5)
+        _check(luvc, oracle_mod, x, keep, cutoff, median_tol=1e-4)
+        assert luvc.check_status() == 0
 
 
 def test_flat_pass_band_option(luvc, oracle_mod):
