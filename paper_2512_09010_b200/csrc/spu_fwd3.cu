@@ -16,13 +16,21 @@
 // write back into tensor memory as bf16 hi + lo pairs (row = lane, K along the columns); its B
 // operand comes from a table in shared memory (per group of tokens a 16 x N2 matrix, bf16 hi and lo
 // parts; block-diagonal over two channels in the narrow-band variant); the band spectrum accumulates
-// in TMEM over the whole sequence and is written out once per work item:
-//   Y[b][r][d], r = k (cos rows, 0..sigma) and r = sigma + k (sin rows, k >= 1), times the row
-//   constants c[r] (mask of Eq. 5/6, 1/N and the weight of the conjugate half).
+// in TMEM over the whole sequence and is written out once per work item, times the row constants
+// (mask of Eq. 5/6, 1/N and the weight of the conjugate half), in the "operand form" that the
+// inverse kernel of spu_inv3.cu multiplies from: per sequence and channel, for every TMEM lane its
+// bins k2 = 0, 1, .. as four bf16 each (Re hi, Im hi, Re lo, Im lo), 16 bytes per lane and pair of
+// bins, the 128 lanes side by side.
 // What is left on the CUDA cores per stage-1 value is one TMEM read, one lane exchange, the twiddle
-// (two packed FMAs) and the split into two bf16 pairs: the same for every band width.
+// and the split into two bf16 pairs: the same for every band width.
 //
-// A CTA is persistent over work items (sequence x channel tile x slice of 16 values of k2) and runs
+// Three geometries share the 512 TMEM columns (two stage-1 accumulators, one operand slot, 64 result
+// columns per converter thread): 32 channels x 4 bins per frequency class, 16 x 8 and 8 x 16.  One
+// value of k2 more than the geometry holds still costs no second pass: the lanes that reach it keep
+// that bin on the CUDA cores (EXTRA = 1), and when only k1 = 0 reaches it (sigma a multiple of 128)
+// the stage-2 issuing warps form it from the lane-0 values of each tile (EXTRA = 2).
+//
+// A CTA is persistent over work items (sequence x channel tile x slice of k2 values) and runs
 // sixteen converter warps (four per TMEM lane quadrant: a group of four warps, one per quadrant,
 // shares the same channels of a tile), one warp that issues the TMA copies and stage 1, and one
 // warp per converter group that issues that group's stage-2 MMAs: a tcgen05.mma costs its issuing
