@@ -127,7 +127,7 @@ SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma);
 // Y[b][r][d] = c[r] * (band spectrum); also its transposed bf16 pair [b][d][r_pad] when yt_hi is given.
 // `img`: kSpuImgBytes of 16-byte aligned device scratch for the operand images a call builds once for all its CTAs.
 int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, void* yt_lo, int r_pad, int B, int N,
-                 int D, int sigma, int* status, cudaStream_t stream, void* img);
+                 int D, int sigma, int* status, cudaStream_t stream, void* img, bool img_ready = false);
 
 // Forward transform with both stages on the tensor cores (spu_fwd3.cu): N = 128 Q, 8 <= Q <= 128.
 struct SpuFwd3Plan {
@@ -171,6 +171,8 @@ struct SpuInv2Plan {
     int n_parts;        // partial sums per point and sequence: part[b][n_parts][L]
 };
 SpuInv2Plan spu_inv2_plan(int B, int N, int D, int sigma);
-int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream, void* img);
+// img_ready: the caller has built the image already (spu_images.cuh).
+int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream, void* img,
+                 bool img_ready = false);
 
 }  // namespace luvc

@@ -17,6 +17,7 @@
 #include <cuda_bf16.h>
 
 #include "luvc_internal.h"
+#include "spu_images.cuh"
 
 namespace luvc {
 namespace {
@@ -27,8 +28,25 @@ constexpr int kGemmThreads = 256;
 // cos / sin of 2 pi j / N for j = 0..N-1, and the per-row constants c[r].
 // scale has `scale_len` >= 2 sigma + 1 entries; the extra ones are zero.
 // tw2 (may be null) is the same table for a period of L points.
-__global__ void spu_tables_kernel(float2* tw, float2* tw2, float* scale, int N, int L, int sigma, int scale_len,
-                                  int no_window) {
+// Blocks past the first `tab_blocks` build the operand images of the two-stage transform kernels (when given):
+// `f_blocks` blocks the forward kernel's, the rest the inverse kernel's, so that a call has one set-up launch.
+struct SpuImages {
+    unsigned char* fwd;     // null: no images in this launch
+    unsigned char* inv;
+    int P, KT, J, KB_inv, tab_blocks, f_blocks;
+};
+__global__ void __launch_bounds__(256) spu_tables_kernel(float2* tw, float2* tw2, float* scale, int N, int L, int sigma,
+                                                         int scale_len, int no_window, const SpuImages im) {
+    if (im.fwd != nullptr && (int)blockIdx.x >= im.tab_blocks) {
+        const int rel = (int)blockIdx.x - im.tab_blocks;
+        if (rel < im.f_blocks) {
+            const int idx = rel * 256 + threadIdx.x;
+            if (idx < 128 * im.KT) spu_fwd2_img_element(im.fwd, im.P, im.KT, idx);
+        } else {
+            spu_inv2_img_element(im.inv, im.P, im.KT, im.J, im.KB_inv, (rel - im.f_blocks) * 256 + threadIdx.x);
+        }
+        return;
+    }
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < N) {
         double s, c;
@@ -613,8 +631,22 @@ static int spu_run_typed(const SpuProblem& p) {
     const int tab = max(max(N, pl.r_pad), pl.L);
     const long long bn = (long long)B * N;
     phase_begin(LUVC_PHASE_SPU_TRANSFORM, p.stream);
-    spu_tables_kernel<<<(tab + 255) / 256, 256, 0, p.stream>>>(ws.tw, ws.tw2, ws.scale, N, pl.L, sigma, pl.r_pad,
-                                                               p.no_window);
+    SpuImages im = {};
+    im.tab_blocks = (tab + 255) / 256;
+    int img_blocks = 0;
+    if constexpr (kTensor) {
+        if (mode.fwd2 && mode.inv2 && !mode.tc2) {      // both two-stage kernels run: their images ride along
+            const SpuFwd2Plan fp = spu_fwd2_plan(B, N, D, sigma);
+            const SpuInv2Plan ip = spu_inv2_plan(B, N, D, sigma);
+            im.fwd = static_cast<unsigned char*>(ws.img_fwd);
+            im.inv = static_cast<unsigned char*>(ws.img_inv);
+            im.P = fp.P; im.KT = fp.nblk * fp.P; im.J = ip.J; im.KB_inv = ip.KB;
+            im.f_blocks = (128 * im.KT + 255) / 256;
+            img_blocks = im.f_blocks + (max(128 * im.KT, ip.J * ip.KB) + 255) / 256;
+        }
+    }
+    spu_tables_kernel<<<im.tab_blocks + img_blocks, 256, 0, p.stream>>>(ws.tw, ws.tw2, ws.scale, N, pl.L, sigma, pl.r_pad,
+                                                                        p.no_window, im);
     count_launch();
     if constexpr (kTensor) {
         int rc;
@@ -627,10 +659,11 @@ static int spu_run_typed(const SpuProblem& p) {
         } else {
             if (mode.fwd2) {
                 const int rc1 = spu_fwd2_run(p.hidden, ws.Y2, ws.scale, mode.inv2 ? nullptr : ws.tc.yt_hi,
-                                             mode.inv2 ? nullptr : ws.tc.yt_lo, pl.r_pad, B, N, D, sigma, p.status, p.stream, ws.img_fwd);
+                                             mode.inv2 ? nullptr : ws.tc.yt_lo, pl.r_pad, B, N, D, sigma, p.status, p.stream, ws.img_fwd,
+                                             im.fwd != nullptr);
                 if (rc1 != LUVC_OK) return rc1;
             }
-            rc = mode.inv2 ? spu_inv2_run(ws.Y2, ws.tc.part, B, N, D, sigma, p.status, p.stream, ws.img_inv)
+            rc = mode.inv2 ? spu_inv2_run(ws.Y2, ws.tc.part, B, N, D, sigma, p.status, p.stream, ws.img_inv, im.fwd != nullptr)
                            : spu_tc_run(ws.tc, p.hidden, ws.tw, ws.tw2, ws.scale, B, N, D, sigma, p.status,
                                         p.stream, mode.fwd2, p.row_index, p.src_rows);
         }

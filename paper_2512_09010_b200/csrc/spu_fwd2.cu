@@ -29,6 +29,7 @@
 
 #include "luvc_internal.h"
 #include "sm100_ptx.cuh"
+#include "spu_images.cuh"
 
 namespace luvc {
 namespace {
@@ -465,30 +466,10 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd2_kernel(const __grid_cons
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
-// Both parts of the stage-1 matrix in the layout the kernel's shared memory uses (K-major: element (row j,
-// column kk) at (j/8)*128 + (kk/8)*2048 + (j%8)*16 + (kk%8)*2; hi part first, lo part KT*256 bytes later),
-// block-diagonal: row j = jb P + jr meets column kk = kb P + p only for jb == kb.  Rows of a block: A[0],
-// A[P/2], then Re / Im of A[1 .. P/2-1].  Built once per call instead of once per CTA.
+// The stage-1 matrix image (spu_images.cuh), built once per call instead of once per CTA.
 __global__ void __launch_bounds__(256) spu_fwd2_img_kernel(unsigned char* __restrict__ img, int P, int KT) {
     const int idx = blockIdx.x * 256 + threadIdx.x;
-    if (idx >= 128 * KT) return;
-    const int j = idx / KT, kk = idx - j * KT;
-    const int jb = j / P, jr = j - jb * P, kb = kk / P, p = kk - kb * P;
-    float v = 0.f;
-    if (j < KT && jb == kb) {
-        if (jr == 0) v = 1.f;
-        else if (jr == 1) v = (p & 1) ? -1.f : 1.f;
-        else {
-            const int m = ((jr >> 1) * p) % P;
-            float s, c;
-            sincospif(2.0f * (float)m / (float)P, &s, &c);
-            v = (jr & 1) ? -s : c;
-        }
-    }
-    const __nv_bfloat16 h = __float2bfloat16_rn(v);
-    const int off = (j >> 3) * 128 + (kk >> 3) * 2048 + (j & 7) * 16 + (kk & 7) * 2;
-    *reinterpret_cast<__nv_bfloat16*>(img + off) = h;
-    *reinterpret_cast<__nv_bfloat16*>(img + KT * 256 + off) = __float2bfloat16_rn(v - __bfloat162float(h));
+    if (idx < 128 * KT) spu_fwd2_img_element(img, P, KT, idx);
 }
 
 // YT[b][d][r] (bf16 pair, r padded with zeros to r_pad) from Y[b][r][d]
@@ -598,10 +579,10 @@ SpuFwd2Plan spu_fwd2_plan(int B, int N, int D, int sigma) {
 }
 
 int spu_fwd2_run(const void* hidden, float* Y, const float* scale, void* yt_hi, void* yt_lo, int r_pad, int B, int N,
-                 int D, int sigma, int* status, cudaStream_t stream, void* img) {
+                 int D, int sigma, int* status, cudaStream_t stream, void* img, bool img_ready) {
     const SpuFwd2Plan pl = spu_fwd2_plan(B, N, D, sigma);
     if (!pl.ok) return LUVC_ERR_INTERNAL;
-    {
+    if (!img_ready) {
         const int KT = pl.nblk * pl.P;
         spu_fwd2_img_kernel<<<(128 * KT + 255) / 256, 256, 0, stream>>>(static_cast<unsigned char*>(img), pl.P, KT);
         count_launch();

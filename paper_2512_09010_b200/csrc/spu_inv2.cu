@@ -24,6 +24,7 @@
 
 #include "luvc_internal.h"
 #include "sm100_ptx.cuh"
+#include "spu_images.cuh"
 
 namespace luvc {
 namespace {
@@ -446,34 +447,9 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
-// A[m][kk] = F[kk mod P][m mod P] where row m = jb P + p and column kk = kb P + r share the block (jb == kb),
-// K-major: element at (m/8)*128 + (kk/8)*2048 + (m%8)*16 + (kk%8)*2, hi part then lo part (KT*256 bytes each);
-// behind them w[jj][k2] = e^{2 pi i k2 jj / J} as (w.x, w.x, w.y, w.y).  Built once per call.
+// The operand image and the table of e^{2 pi i k2 jj / J} (spu_images.cuh), built once per call.
 __global__ void __launch_bounds__(256) spu_inv2_img_kernel(unsigned char* __restrict__ img, int P, int KT, int J, int KB) {
-    const int idx = blockIdx.x * 256 + threadIdx.x;
-    if (idx < 128 * KT) {
-        const int m = idx / KT, kk = idx - m * KT;
-        const int jb = m / P, p = m - jb * P, kb = kk / P, r = kk - kb * P;
-        float v = 0.f;
-        if (m < KT && jb == kb) {
-            if (r == 0) v = 1.f;
-            else if (r == 1) v = (p & 1) ? -1.f : 1.f;
-            else {
-                float s, c;
-                sincospif(2.0f * (float)(((r >> 1) * p) % P) / (float)P, &s, &c);
-                v = (r & 1) ? -s : c;
-            }
-        }
-        const __nv_bfloat16 h = __float2bfloat16_rn(v);
-        const int off = (m >> 3) * 128 + (kk >> 3) * 2048 + (m & 7) * 16 + (kk & 7) * 2;
-        *reinterpret_cast<__nv_bfloat16*>(img + off) = h;
-        *reinterpret_cast<__nv_bfloat16*>(img + KT * 256 + off) = __float2bfloat16_rn(v - __bfloat162float(h));
-    }
-    if (idx < J * KB) {
-        const int jj = idx / KB, k2 = idx - jj * KB;
-        const float2 w = root_pos(((unsigned)jj * (unsigned)k2) % (unsigned)J, J);
-        reinterpret_cast<float4*>(img + 2 * KT * 256)[idx] = make_float4(w.x, w.x, w.y, w.y);
-    }
+    spu_inv2_img_element(img, P, KT, J, KB, blockIdx.x * 256 + threadIdx.x);
 }
 
 template <int KB, int W>
@@ -524,10 +500,11 @@ SpuInv2Plan spu_inv2_plan(int B, int N, int D, int sigma) {
     return pl;
 }
 
-int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream, void* img) {
+int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, int* status, cudaStream_t stream, void* img,
+                 bool img_ready) {
     const SpuInv2Plan pl = spu_inv2_plan(B, N, D, sigma);
     if (!pl.ok) return LUVC_ERR_INTERNAL;
-    {
+    if (!img_ready) {
         const int KT = pl.nblk * pl.P, n = 128 * KT > pl.J * pl.KB ? 128 * KT : pl.J * pl.KB;
         spu_inv2_img_kernel<<<(n + 255) / 256, 256, 0, stream>>>(static_cast<unsigned char*>(img), pl.P, KT, pl.J, pl.KB);
         count_launch();
