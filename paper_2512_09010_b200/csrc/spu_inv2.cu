@@ -33,8 +33,8 @@ using namespace ptx;
 
 constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
-constexpr int kNcol = 64;                     // columns of a tile: TJ points x C channels
-constexpr int kTmemCols = 128;                // two accumulator buffers
+// Columns of a tile (TJ points x C channels) are a template parameter NC: 64, or 128 for the few-bin variants, whose
+// tiles are short on arithmetic and long on hand-overs (two accumulator buffers of NC columns in tensor memory).
 constexpr int kSpin = 1 << 22;
 
 struct InvArgs {
@@ -85,11 +85,11 @@ template <int NV> __device__ __forceinline__ void store_bf16(unsigned char* dst,
 
 // Row `row` of G for the tile's points and this thread's W channels, as a bf16 pair into the B tile.
 // NB bins of this lane's frequency are summed (compile time).  G = ga C.x + gb C.y + gc (partner's value).
-template <int KB, int W, int NB>
+template <int KB, int W, int NB, int NC>
 __device__ __forceinline__ void stage2_tile(const float2 (&y)[KB][W], const float4* __restrict__ w_tab, int jj0, int J,
                                             float2 rot, float2 step, float ga, float gb, float gc, bool odd,
                                             unsigned char* b_hi, unsigned char* b_lo, int sbo, int row, int col0) {
-    constexpr int C = 4 * W, TJ = kNcol / C;
+    constexpr int C = 4 * W, TJ = NC / C;
     constexpr int HV = W >= 8 ? 8 : W;        // bf16 values per store
 #pragma unroll 1
     for (int jl = 0; jl < TJ; ++jl) {
@@ -166,10 +166,10 @@ __device__ __forceinline__ void stage2_tile(const float2 (&y)[KB][W], const floa
 // point to point (k_t = its frequency + P t; times i on the odd lane of a pair, so that its own share of G is the real
 // part of C = sum_t Y_t g[t] and the partner's share the imaginary part), which replaces both the table of
 // e^{2 pi i k2 jj / J} and the rotation by e^{2 pi i k1 jj / L}.  G = Re C + gc (partner's Im C).
-template <int KB, int W, int NB>
+template <int KB, int W, int NB, int NC>
 __device__ __forceinline__ void stage2_tile_few(const float2 (&y)[KB][W], float2 (&g)[KB], const float2 (&gstep)[KB], int jj0, int J,
                                                 float gc, unsigned char* b_hi, unsigned char* b_lo, int sbo, int row, int col0) {
-    constexpr int C = 4 * W, TJ = kNcol / C;
+    constexpr int C = 4 * W, TJ = NC / C;
     constexpr int HV = W >= 8 ? 8 : W;        // bf16 values per store
 #pragma unroll 1
     for (int jl = 0; jl < TJ; ++jl) {
@@ -217,9 +217,10 @@ __device__ __forceinline__ void stage2_tile_few(const float2 (&y)[KB][W], float2
 }
 
 // KB: band bins per lane; W: channels per thread (C = 4 W per channel block, TJ = 64 / C points per tile).
-template <int KB, int W>
+template <int KB, int W, int NC>
 __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) {
-    constexpr int C = 4 * W, TJ = kNcol / C;
+    constexpr int C = 4 * W, TJ = NC / C;
+    constexpr int kNcol = NC, kTmemCols = 2 * NC;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long s_bar[kBars];
     __shared__ uint32_t s_tmem;
@@ -230,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     const int KT = a.nblk * P;                   // rows in use = K extent of the contraction
     const int f_bytes = KT * 256;                // one part of A: KT / 8 K chunks x 128 rows x 16 B
     const int sbo = KT * 16;                     // B: distance between 8-column groups (KT / 8 K groups x 128 B)
-    const int b_part = 8 * sbo, b_buf = 2 * b_part;
+    const int b_part = (NC / 8) * sbo, b_buf = 2 * b_part;
     unsigned char* s_fhi = smem;
     unsigned char* s_flo = smem + f_bytes;
     unsigned char* s_b = smem + 2 * f_bytes;     // [2 buffers][hi, lo][8 column groups][KT / 8][128 B]
@@ -298,26 +299,30 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
     //   C = 64: the point's channel quarter grp;  C = 32: point grp / 2, channel half grp % 2
     //   C = 16: point grp;                         C = 8: points 2 grp and 2 grp + 1
     constexpr int SPLIT = C == 64 ? 4 : (C == 32 ? 2 : 1);          // partial sums per (channel block, point)
-    auto read_tile = [&](int t, int b, int ctile, int jj0) {
-        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((t & 1) * kNcol + grp * 16);
-        uint32_t v[16];
-        tmem_ld16(taddr, v);
-        tmem_ld_wait_for(v);
-        tc_fence_before();
-        if (!active) return;
-        const int sub = C == 64 ? grp : (C == 32 ? (grp & 1) : 0);
-        float* out = a.part + ((size_t)b * (a.n_ctiles * a.nblk * SPLIT) + (ctile * a.nblk + jb) * SPLIT + sub) * L +
-                     (size_t)jr * J;
-        constexpr int PTS = C >= 16 ? 1 : 2;          // points among the 16 columns
-        constexpr int WP = 16 / PTS;                  // columns per point
+    auto read_tile = [&](int t, int b, int ctile, int jj_first) {
 #pragma unroll
-        for (int pt = 0; pt < PTS; ++pt) {
-            float sum = 0.f;
+        for (int hf = 0; hf < NC / 64; ++hf) {               // each 64 columns of the tile as above
+            const int jj0 = jj_first + hf * (64 / C);
+            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((t & 1) * kNcol + hf * 64 + grp * 16);
+            uint32_t v[16];
+            tmem_ld16(taddr, v);
+            tmem_ld_wait_for(v);
+            if (!active) continue;
+            const int sub = C == 64 ? grp : (C == 32 ? (grp & 1) : 0);
+            float* out = a.part + ((size_t)b * (a.n_ctiles * a.nblk * SPLIT) + (ctile * a.nblk + jb) * SPLIT + sub) * L +
+                         (size_t)jr * J;
+            constexpr int PTS = C >= 16 ? 1 : 2;          // points among the 16 columns
+            constexpr int WP = 16 / PTS;                  // columns per point
 #pragma unroll
-            for (int q = 0; q < WP; ++q) { const float x = __uint_as_float(v[pt * WP + q]); sum = fmaf(x, x, sum); }
-            const int jl = C == 64 ? 0 : (C == 32 ? (grp >> 1) : (C == 16 ? grp : 2 * grp + pt));
-            if (jj0 + jl < J) out[jj0 + jl] = sum;
+            for (int pt = 0; pt < PTS; ++pt) {
+                float sum = 0.f;
+#pragma unroll
+                for (int q = 0; q < WP; ++q) { const float x = __uint_as_float(v[pt * WP + q]); sum = fmaf(x, x, sum); }
+                const int jl = C == 64 ? 0 : (C == 32 ? (grp >> 1) : (C == 16 ? grp : 2 * grp + pt));
+                if (jj0 + jl < J) out[jj0 + jl] = sum;
+            }
         }
+        tc_fence_before();
     };
 
     int t = 0;                                       // tiles issued so far by this CTA
@@ -378,11 +383,11 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
                 unsigned char* bl = bh + b_part;
                 const int col0 = grp * W;
                 if (nb_w == KB)
-                    stage2_tile_few<KB, W, KB>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
+                    stage2_tile_few<KB, W, KB, NC>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
                 else if (nb_w == KB - 1 || KB == 2)
-                    stage2_tile_few<KB, W, (KB > 1 ? KB - 1 : 1)>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
+                    stage2_tile_few<KB, W, (KB > 1 ? KB - 1 : 1), NC>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
                 else
-                    stage2_tile_few<KB, W, (KB >= 4 ? KB / 2 : KB)>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
+                    stage2_tile_few<KB, W, (KB >= 4 ? KB / 2 : KB), NC>(y, gk, gstep, jj0, J, gc, bh, bl, sbo, active ? j : -1, col0);
             } else if (warp_active) {
                 const float2 rot = root_pos(((unsigned)kf * (unsigned)jj0) % (unsigned)L, L);   // kf jj0 < P J = L
                 unsigned char* bh = s_b + (t & 1) * b_buf;
@@ -390,13 +395,13 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv2_kernel(const InvArgs a) 
                 const int col0 = grp * W;
                 // lanes past the rows in use take part in the exchange with zeros and store nothing
                 if (nb_w == KB)
-                    stage2_tile<KB, W, KB>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
+                    stage2_tile<KB, W, KB, NC>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
                 else if (nb_w == KB - 1 || KB == 2)
-                    stage2_tile<KB, W, (KB > 1 ? KB - 1 : 1)>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
+                    stage2_tile<KB, W, (KB > 1 ? KB - 1 : 1), NC>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
                 else if (KB >= 4 && nb_w <= KB / 2)
-                    stage2_tile<KB, W, (KB >= 4 ? KB / 2 : KB)>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
+                    stage2_tile<KB, W, (KB >= 4 ? KB / 2 : KB), NC>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
                 else
-                    stage2_tile<KB, W, KB>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
+                    stage2_tile<KB, W, KB, NC>(y, s_w, jj0, J, rot, step, ga, gb, gc, odd, bh, bl, sbo, active ? j : -1, col0);
             }
             fence_proxy_async();
             __syncwarp();
@@ -452,19 +457,19 @@ __global__ void __launch_bounds__(256) spu_inv2_img_kernel(unsigned char* __rest
     spu_inv2_img_element(img, P, KT, J, KB, blockIdx.x * 256 + threadIdx.x);
 }
 
-template <int KB, int W>
+template <int KB, int W, int NC = 64>
 cudaError_t launch_inv2(const InvArgs& a, cudaStream_t stream) {
     const int KT = a.nblk * a.P;
-    const size_t smem = (size_t)2 * KT * 256 + (size_t)2 * KT * 256 + (size_t)a.J * KB * sizeof(float4);
+    const size_t smem = (size_t)2 * KT * 256 + (size_t)(NC / 32) * KT * 256 + (size_t)a.J * KB * sizeof(float4);
     static int sms = 0;
     if (!sms) {
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    cudaFuncSetAttribute(spu_inv2_kernel<KB, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncSetAttribute(spu_inv2_kernel<KB, W, NC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int grid = a.n_items < sms ? a.n_items : sms;
-    spu_inv2_kernel<KB, W><<<grid, kThreads, smem, stream>>>(a);
+    spu_inv2_kernel<KB, W, NC><<<grid, kThreads, smem, stream>>>(a);
     return cudaGetLastError();
 }
 
@@ -515,8 +520,8 @@ int spu_inv2_run(const float* Y, float* part, int B, int N, int D, int sigma, in
     a.B = B; a.N = N; a.D = D; a.P = pl.P; a.Q = pl.Q; a.sigma = sigma; a.R = 2 * sigma + 1;
     a.nblk = pl.nblk; a.J = pl.J; a.L = pl.L; a.n_ctiles = pl.n_ctiles; a.n_items = pl.n_items;
     cudaError_t err;
-    if (pl.KB == 2) err = launch_inv2<2, 16>(a, stream);
-    else if (pl.KB == 4) err = launch_inv2<4, 8>(a, stream);
+    if (pl.KB == 2) err = launch_inv2<2, 16, 128>(a, stream);
+    else if (pl.KB == 4) err = launch_inv2<4, 8, 128>(a, stream);
     else if (pl.KB == 9) err = launch_inv2<9, 4>(a, stream);
     else err = launch_inv2<17, 2>(a, stream);
     count_launch();
