@@ -152,6 +152,7 @@ struct SpuInv3Plan {
     int coarse, J, L;   // as SpuInv2Plan
     int KS;             // K steps of four bins each
     int JP;             // points per channel held in tensor memory: 16, 40 or 72
+    int CT;             // channels per tile of the second contraction: 4, 2 or 1
     int extra;          // 1: the bin k = 128 * 16 reaches into the band and is passed apart
     int n_ctiles, n_items, n_parts;
     size_t yop_bytes;   // size of the band spectrum in operand form

@@ -97,16 +97,15 @@ __device__ __forceinline__ uint32_t bf16x2_bits(float lo_half, float hi_half) {
 // Geometry of a variant.
 //   JP   points jj per channel held by the stage-2' result (J rounded up to a multiple of 8)
 //   CT   channels per tile of stage 1'
-template <int JP_, int CT_>
+template <int JP_, int CT_, int NBUF_>
 struct IGeo {
-    static constexpr int JP = JP_, CT = CT_;
+    static constexpr int JP = JP_, CT = CT_, NBUF = NBUF_;    // NBUF: shared-memory buffers of the stage-2' operand (2 or 3)
     static constexpr int N2 = 2 * JP;                         // columns of the stage-2' result per channel: (point, re/im)
-    static constexpr int NP = (JP + 15) / 16 * 16;            // columns of stage 1' per channel
-    static constexpr int TCOL = CT * NP;                      // N of the stage-1' MMAs
-    static constexpr int BCOLS = CT * JP;                     // columns of the stage-1' operand that are written
+    static constexpr int BCOLS = CT * JP;                     // columns of the stage-1' operand that are written: (channel, point)
+    static constexpr int TCOL = (BCOLS + 15) / 16 * 16;       // N of the stage-1' MMAs
     static constexpr int NCH = JP / 4;                        // chunks of four points per channel
-    static constexpr int MYCH = (NCH + 3) / 4;                // chunks per converter thread and channel
-    static constexpr int UNITS = CT * MYCH;                   // chunks per converter thread and tile
+    static constexpr int TOTCH = CT * NCH;                    // chunks of a tile, dealt out to the four warps of a lane quadrant
+    static constexpr int UNITS = (TOTCH + 3) / 4;             // chunks per converter thread and tile
     static constexpr int ECOLS = TCOL / 4;                    // result columns per converter thread
     static constexpr int ACC0 = 0, D20 = 2 * TCOL;
     static constexpr int TMEM_COLS = 512;
@@ -114,7 +113,8 @@ struct IGeo {
     static constexpr int B_BUF = 2 * B_PART;
     static constexpr int W_BYTES = 32 * N2;                   // one part of one K step's stage-2' matrix: 16 x N2 bf16
     static_assert(JP % 8 == 0 && D20 + 2 * CT * N2 <= TMEM_COLS, "tensor memory budget");
-    static_assert(CT == 1 || (CT == 4 && JP == 16), "four channels per tile only with sixteen points");
+    static_assert(CT == 1 || JP % ECOLS == 0, "a converter thread's result columns belong to one channel");
+    static_assert(NBUF == 2 || NBUF == 3, "operand buffers");
 };
 
 template <typename G, bool EXTRA>
@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv3_kernel(const Inv3Args a)
             const int ctile = c_item % a.n_ctiles, b = c_item / a.n_ctiles;
             const int c = ctile * kItemChannels + c_tile * CT;
             const int nch = min(CT, D - c);
-            const int buf = c_v % kA2Bufs;
+            const int buf = c_v % G::NBUF;
             if (elect_one()) {
                 const uint32_t bytes = (uint32_t)(nch * KS * kChanBytes);
                 mbar_arrive_expect_tx(bar(kBarA2Full + buf), bytes);
@@ -204,21 +204,20 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv3_kernel(const Inv3Args a)
             ++c_v;
             if (++c_tile == item_tiles(c_item)) { c_tile = 0; c_item += gridDim.x; }
         };
-        issue_copy();
-        issue_copy();
+        for (int q = 0; q < G::NBUF - 1; ++q) issue_copy();
         int v = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
             const int nt = item_tiles(item);
             const int c_first = (item % a.n_ctiles) * kItemChannels;
             for (int tile = 0; tile < nt && ok; ++tile, ++v) {
-                // the copy two tiles ahead reuses the buffer of tile v - 1, whose MMAs were issued a tile ago
-                if (c_v == v + 2) {
-                    if (v >= 1) ok = wait_bar_warp(bar(kBarA2Empty + (v + 2) % kA2Bufs), ((v - 1) / kA2Bufs) & 1, fail, a.status);
+                // the copy NBUF - 1 tiles ahead reuses the buffer of tile v - 1, whose MMAs were issued a tile ago
+                if (c_v == v + G::NBUF - 1) {
+                    if (v >= 1) ok = wait_bar_warp(bar(kBarA2Empty + (v + G::NBUF - 1) % G::NBUF), ((v - 1) / G::NBUF) & 1, fail, a.status);
                     if (!ok) break;
                     issue_copy();
                 }
-                ok = wait_bar_warp(bar(kBarA2Full + v % kA2Bufs), (v / kA2Bufs) & 1, fail, a.status);
+                ok = wait_bar_warp(bar(kBarA2Full + v % G::NBUF), (v / G::NBUF) & 1, fail, a.status);
                 if (ok && v >= 2) ok = wait_bar_warp(bar(kBarD2Empty + (v & 1)), ((v - 2) >> 1) & 1, fail, a.status);
                 if (!ok) break;
                 tc_fence_after();
@@ -227,14 +226,14 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv3_kernel(const Inv3Args a)
                     for (int ct = 0; ct < nch; ++ct) {
                         const uint32_t d2 = tmem + (uint32_t)(G::D20 + (v & 1) * CT * N2 + ct * N2);
                         for (int s = 0; s < KS; ++s) {
-                            const uint64_t ad = a0 + (uint64_t)(((v % kA2Bufs) * a2_bytes + (ct * KS + s) * kChanBytes) >> 4);
+                            const uint64_t ad = a0 + (uint64_t)(((v % G::NBUF) * a2_bytes + (ct * KS + s) * kChanBytes) >> 4);
                             const uint64_t whi = w0 + (uint64_t)((s * 2 * G::W_BYTES) >> 4), wlo = whi + (uint64_t)(G::W_BYTES >> 4);
                             umma_bf16(d2, ad, whi, idesc2, s ? 1u : 0u);
                             umma_bf16(d2, ad, wlo, idesc2, 1u);
                         }
                     }
                     umma_commit(bar(kBarD2Full + (v & 1)));
-                    umma_commit(bar(kBarA2Empty + v % kA2Bufs));
+                    umma_commit(bar(kBarA2Empty + v % G::NBUF));
                 }
                 __syncwarp();
             }
@@ -293,18 +292,21 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv3_kernel(const Inv3Args a)
         const int kf = special ? (odd ? kP / 2 : 0) : (odd ? kP - i : i);       // this lane's frequency
         const float gc = special ? 0.f : 1.f;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-        // twiddles e^{2 pi i kf jj / L} of this thread's points jj = 4 (grp + 4 m) + e, times i on the odd lane of a
-        // pair: then the own contribution to G is the real part and the partner's is the imaginary part
-        float2 rot[G::MYCH][4];
+        // twiddles e^{2 pi i kf jj / L} of this thread's points: unit u is chunk c = grp + 4 u of the tile's chunks
+        // (channel c / NCH, points 4 (c % NCH) + e), times i on the odd lane of a pair: then the own contribution
+        // to G is the real part and the partner's is the imaginary part
+        float2 rot[G::UNITS][4];
 #pragma unroll
-        for (int m = 0; m < G::MYCH; ++m)
+        for (int u = 0; u < G::UNITS; ++u)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int jj = 4 * (grp + 4 * m) + e;
+                const int jj = 4 * ((grp + 4 * u) % G::NCH) + e;
                 float2 r = root_pos((unsigned)(((long long)kf * jj) % L), (unsigned)L);
                 if (odd && !special) r = make_float2(-r.y, r.x);
-                rot[m][e] = r;
+                rot[u][e] = r;
             }
+        // this thread's ECOLS result columns grp ECOLS + q are points e_jj0 + q of channel e_ct of the tile
+        const int e_ct = (grp * G::ECOLS) / JP, e_jj0 = (grp * G::ECOLS) % JP;
         float en[G::ECOLS];                              // energies of this thread's result columns, summed over the item
 #pragma unroll
         for (int q = 0; q < G::ECOLS; ++q) en[q] = 0.f;
@@ -332,17 +334,16 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv3_kernel(const Inv3Args a)
             for (int q = 0; q < G::ECOLS; ++q) {
                 constexpr int kFirst = G::ECOLS >= 16 ? 16 : 8;
                 float x = __uint_as_float(q < kFirst ? x0[q < kFirst ? q : 0] : x1[q >= kFirst ? q - kFirst : 0]);
-                if constexpr (EXTRA) x += s_e[(tt & 1) * JP + min(grp * G::ECOLS + q, JP - 1)];
+                if constexpr (EXTRA) x += s_e[(tt & 1) * JP + min(e_jj0 + q, JP - 1)];
                 en[q] = fmaf(x, x, en[q]);
             }
         };
         // the item's energies: part[b][ctile (x channel of the tile)][p J + jj]
         auto flush = [&](int b, int ctile) {
-            constexpr int SPLIT = CT == 4 ? 4 : 1;
-            float* out = a.part + ((size_t)b * a.n_parts + (size_t)ctile * SPLIT + (CT == 4 ? grp : 0)) * L + (size_t)j * J;
+            float* out = a.part + ((size_t)b * a.n_parts + (size_t)ctile * CT + e_ct) * L + (size_t)j * J;
 #pragma unroll
             for (int q = 0; q < G::ECOLS; ++q) {
-                const int jj = CT == 4 ? q : grp * G::ECOLS + q;
+                const int jj = e_jj0 + q;
                 if (jj < J) out[jj] = en[q];
                 en[q] = 0.f;
             }
@@ -364,26 +365,26 @@ __global__ void __launch_bounds__(kThreads, 1) spu_inv3_kernel(const Inv3Args a)
                 unsigned char* bh = s_b + dbuf * G::B_BUF;
                 unsigned char* bl = bh + G::B_PART;
                 const uint32_t d2 = lane_addr + (uint32_t)(G::D20 + dbuf * CT * N2);
-                // unit u = (channel ct of the tile, chunk grp + 4 m of its points): 8 columns of the stage-2' result
+                // unit u = chunk grp + 4 u of the tile: 8 columns of the stage-2' result of its channel
                 uint32_t vb[2][8];                       // units alternate between the two: one in use, one in flight
                 tmem_ld8(d2 + (uint32_t)(grp * 8), vb[0]);
 #pragma unroll
                 for (int u = 0; u < G::UNITS; ++u) {
-                    const int ct = u / G::MYCH, m = u % G::MYCH;
-                    const int ch = grp + 4 * m;
-                    const bool live = ch < G::NCH;       // the same for the whole warp
+                    const int c = grp + 4 * u;
+                    const int ct = c / G::NCH, ch = c % G::NCH;
+                    const bool live = c < G::TOTCH;      // the same for the whole warp
                     uint32_t (&v)[8] = vb[u & 1];
                     if (live) tmem_ld_wait_for(v);
                     if (u + 1 < G::UNITS) {
-                        const int ct1 = (u + 1) / G::MYCH, m1 = (u + 1) % G::MYCH;
-                        if (grp + 4 * m1 < G::NCH) tmem_ld8(d2 + (uint32_t)(ct1 * N2 + (grp + 4 * m1) * 8), vb[(u + 1) & 1]);
+                        const int c1 = c + 4;
+                        if (c1 < G::TOTCH) tmem_ld8(d2 + (uint32_t)((c1 / G::NCH) * N2 + (c1 % G::NCH) * 8), vb[(u + 1) & 1]);
                     }
                     if (!live) continue;
                     float g[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float sx = __uint_as_float(v[2 * e]), sy = __uint_as_float(v[2 * e + 1]);
-                        const float2 r = rot[m][e];
+                        const float2 r = rot[u][e];
                         const float cx = fmaf(r.x, sx, -r.y * sy), cy = fmaf(r.x, sy, r.y * sx);
                         const float got = __shfl_xor_sync(0xffffffffu, cy, 1);
                         g[e] = fmaf(gc, got, cx);
@@ -488,7 +489,7 @@ __global__ void __launch_bounds__(256) spu_inv3_img_kernel(unsigned char* __rest
 template <typename G>
 size_t inv3_smem(int KS) {
     return 1024 + 65536 + (size_t)KS * 2 * G::W_BYTES + (size_t)G::JP * sizeof(float2) + (size_t)2 * G::JP * sizeof(float) +
-           (size_t)2 * G::B_BUF + (size_t)kA2Bufs * G::CT * KS * kChanBytes;
+           (size_t)2 * G::B_BUF + (size_t)G::NBUF * G::CT * KS * kChanBytes;
 }
 
 template <typename G, bool EXTRA>
@@ -510,9 +511,10 @@ cudaError_t launch_inv3(const Inv3Args& a, int nk2, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-using GeoSmall = IGeo<16, 4>;
-using GeoMid = IGeo<40, 1>;
-using GeoBig = IGeo<72, 1>;
+using GeoSmall = IGeo<16, 4, 3>;
+using GeoMid2 = IGeo<40, 2, 2>;      // two channels per tile: 20 chunks split evenly over four warps, one 80-column contraction
+using GeoMid = IGeo<40, 1, 3>;       // where the operands of two channels do not fit
+using GeoBig = IGeo<72, 1, 3>;
 
 }  // namespace
 
@@ -534,14 +536,17 @@ SpuInv3Plan spu_inv3_plan(int B, int N, int D, int sigma) {
     pl.KS = ((pl.extra ? 16 : nk2) + 3) / 4;
     pl.JP = pl.J <= 16 ? 16 : (pl.J <= 40 ? 40 : (pl.J <= 72 ? 72 : 0));
     if (!pl.JP || (pl.extra && pl.JP != 72)) return pl;
-    const size_t smem = pl.JP == 16 ? inv3_smem<GeoSmall>(pl.KS) : (pl.JP == 40 ? inv3_smem<GeoMid>(pl.KS) : inv3_smem<GeoBig>(pl.KS));
+    pl.CT = pl.JP == 16 ? 4 : 1;
+    if (pl.JP == 40 && inv3_smem<GeoMid2>(pl.KS) <= (size_t)226 * 1024) pl.CT = 2;
+    const size_t smem = pl.JP == 16 ? inv3_smem<GeoSmall>(pl.KS)
+                        : pl.JP == 40 ? (pl.CT == 2 ? inv3_smem<GeoMid2>(pl.KS) : inv3_smem<GeoMid>(pl.KS)) : inv3_smem<GeoBig>(pl.KS);
     if (smem > 226 * 1024) return pl;
     if (65536 + (size_t)pl.KS * 2 * 64 * pl.JP + (size_t)pl.JP * 8 > kSpuImgBytes) return pl;
     pl.n_ctiles = (D + kItemChannels - 1) / kItemChannels;
     const long long items = (long long)B * pl.n_ctiles;
     if (items > 0x7fffffffll) return pl;
     pl.n_items = (int)items;
-    pl.n_parts = pl.n_ctiles * (pl.JP == 16 ? 4 : 1);
+    pl.n_parts = pl.n_ctiles * pl.CT;
     pl.yop_bytes = (size_t)B * D * pl.KS * kChanBytes;
     pl.ok = 1;
     return pl;
@@ -560,7 +565,7 @@ int spu_inv3_run(const void* yop, const float* yx_re, const float* yx_im, long l
     a.img = static_cast<const unsigned char*>(img);
     const int nk2 = pl.extra ? 16 : sigma / kP + 1;
     const cudaError_t err = pl.JP == 16 ? launch_inv3<GeoSmall, false>(a, nk2, stream)
-                            : pl.JP == 40 ? launch_inv3<GeoMid, false>(a, nk2, stream)
+                            : pl.JP == 40 ? (pl.CT == 2 ? launch_inv3<GeoMid2, false>(a, nk2, stream) : launch_inv3<GeoMid, false>(a, nk2, stream))
                             : pl.extra ? launch_inv3<GeoBig, true>(a, nk2, stream) : launch_inv3<GeoBig, false>(a, nk2, stream);
     count_launch(2);
     return err == cudaSuccess ? LUVC_OK : LUVC_ERR_CUDA;
