@@ -43,8 +43,9 @@ HBM_FALLBACK_GBS = 6650.0     # used only if MEASURED_PEAKS.json is absent
 
 def ncu_traffic():
     """dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
-    profiles/ (profiles/ncu_traffic.json: kernel -> workload -> bytes, with the source version of the
-    kernel the counters were taken on; an entry is ignored once that source has changed)."""
+    profiles/ (profiles/ncu_traffic.json: kernel or kernel group -> case -> bytes, with the version of the
+    source files the counters were taken on; an entry is ignored once one of those files has changed).
+    A case is the workload number, for the prune followed by "@" and the cutoff ("4@0.05")."""
     path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
     if not os.path.exists(path):
         return {}
@@ -53,10 +54,13 @@ def ncu_traffic():
     table = json.load(open(path))
     out = {}
     for kernel, entry in table.items():
-        src = os.path.join(ROOT, entry["source"])
-        digest = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] if os.path.exists(src) else None
-        if digest == entry.get("source_sha256_16"):
-            out[kernel] = {int(k): float(v) for k, v in entry["bytes_per_launch"].items()}
+        files = entry.get("sources") or [entry["source"]]
+        h = hashlib.sha256()
+        for f in files:
+            src = os.path.join(ROOT, f)
+            h.update(open(src, "rb").read() if os.path.exists(src) else b"missing")
+        if h.hexdigest()[:16] == entry.get("source_sha256_16"):
+            out[kernel] = {str(k): float(v) for k, v in entry["bytes_per_launch"].items()}
     return out
 
 
@@ -381,7 +385,7 @@ def oim_roofline(luvc, spec, phases, peak, peak_src, traffic, matching):
     steps_ms = phases["oim_steps"]
     r = rate(iter_bytes, steps_ms, peak)
     kernel = "oim_chain_kernel" if matching == "adjacent" else "oim_bipartite_kernel"
-    t = traffic.get(kernel, {}).get(spec["id"])
+    t = traffic.get(kernel, {}).get(str(spec["id"]))
     out = {
         "kernel": "%s (one launch runs the %d merge steps of a call)" % (kernel, n_steps),
         "bound": "hbm", "achieved": r["achieved"], "peak": peak, "unit": "GB/s", "frac": r["frac"],
@@ -397,13 +401,18 @@ def oim_roofline(luvc, spec, phases, peak, peak_src, traffic, matching):
     return out
 
 
-def spu_roofline(spec, keep, phases, peak):
+def spu_roofline(spec, keep, phases, peak, traffic=None, cutoff=None):
     sb, sn, sd = spec["spu"]
     tb, selb, gb = spu_bytes(sb, sn, sd, keep)
     total_ms = phases["spu_transform"] + phases["spu_select"] + phases["spu_gather"]
     out = rate(tb + selb + gb, total_ms, peak)
+    transform = rate(tb, phases["spu_transform"], peak)
+    # DRAM bytes of the two transform kernels (forward + inverse) from the ncu capture of this case, if there is one
+    cut = cutoff if cutoff is not None else spec["cutoff"]
+    case = "%d@%g" % (spec["id"], cut if cut > 0 else 0.125)
+    transform["traffic"] = next((v[case] for v in (traffic or {}).values() if case in v), None)
     out.update({"bound": "hbm", "unit": "GB/s", "peak": peak,
-                "transform": rate(tb, phases["spu_transform"], peak),
+                "transform": transform,
                 "select": rate(selb, phases["spu_select"], peak),
                 "gather": rate(gb, phases["spu_gather"], peak)})
     return out
@@ -431,7 +440,7 @@ def per_config_report(torch, luvc, device, peak, peak_src, traffic, barrier, hav
         ph = phase_times(luvc, step, 10)
         entry = {"workload": workload_name(spec), "ms_per_step": ms, "tokens_per_s": spec["tokens"] / (ms * 1e-3),
                  "phases_ms": ph, "oim": oim_roofline(luvc, spec, ph, peak, peak_src, traffic, "adjacent"),
-                 "spu": spu_roofline(spec, spec["keep"], ph, peak)}
+                 "spu": spu_roofline(spec, spec["keep"], ph, peak, traffic)}
         c = gi.CONFIGS[k]
         sweep = []
         cutoffs = c.get("cutoffs", (0.0,))
@@ -442,7 +451,7 @@ def per_config_report(torch, luvc, device, peak, peak_src, traffic, barrier, hav
 
                 timed_steps(torch, prune, 2, 3, barrier)
                 ph2 = phase_times(luvc, prune, 6)
-                row = spu_roofline(spec, keep, ph2, peak)
+                row = spu_roofline(spec, keep, ph2, peak, traffic, cutoff)
                 row.update({"cutoff": cutoff if cutoff > 0 else 0.125, "keep": keep})
                 sweep.append(row)
         entry["spu_sweep"] = sweep
@@ -576,7 +585,7 @@ def main():
     peak, peak_src = load_peak()
     traffic = ncu_traffic()
     roofline = oim_roofline(luvc, spec, phases, peak, peak_src, traffic, args.oim_matching)
-    roofline["spu"] = spu_roofline(spec, spec["keep"], phases, peak)
+    roofline["spu"] = spu_roofline(spec, spec["keep"], phases, peak, traffic)
 
     per_config = None
     if not args.no_per_config and world == 1 and args.oim_matching == "adjacent":
