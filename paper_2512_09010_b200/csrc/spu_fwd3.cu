@@ -381,6 +381,8 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         int u = 0, item_seq = 0;
         bool ok = true;
+        float2 within[QT];
+        int within_kfe = -1;
         for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x, ++item_seq) {
             const int slice = item % a.n_slices, rest = item / a.n_slices;
             const int ctile = rest % a.n_ctiles, b = rest / a.n_ctiles;
@@ -388,10 +390,13 @@ __global__ void __launch_bounds__(kThreads, 1) spu_fwd3_kernel(const __grid_cons
             const int kfe = kf + kP * k2_lo;                         // the slice's first bin of this lane
             // twiddle of token q0 + ql: e^{-2 pi i q0 kfe / N}, exact per tile, times e^{-2 pi i ql kfe / N},
             // exact per item: two roundings per value however long the sequence is
-            float2 within[QT];
+            // (the same for every work item of a slice, so with one slice they are computed once per kernel)
+            if (kfe != within_kfe) {
 #pragma unroll
-            for (int ql = 0; ql < QT; ++ql)
-                within[ql] = root_neg((unsigned)(((unsigned long long)ql * (unsigned)kfe) % (unsigned)N), (unsigned)N);
+                for (int ql = 0; ql < QT; ++ql)
+                    within[ql] = root_neg((unsigned)(((unsigned long long)ql * (unsigned)kfe) % (unsigned)N), (unsigned)N);
+                within_kfe = kfe;
+            }
             // angle of the tile's first token, q0 kfe mod N, carried in integers (exact); N = 128 Q, so
             // e^{-2 pi i m / N} = e^{-2 pi i (m >> 7) / Q} e^{-2 pi i (m & 127) / N}: two table entries
             const int d_angle = (int)(((unsigned long long)QT * (unsigned)kfe) % (unsigned)N);
